@@ -1,0 +1,240 @@
+"""ctypes front end of the CPU oracle (TEST INFRASTRUCTURE, not part of the product).
+
+The arithmetic lives in ``rcd_oracle.c`` / ``rcd_oracle_typed.inc`` (plain C,
+single-threaded, int64 or double).  This file only compiles and loads that
+code, splits a dataset into classes (Algorithm 1, "Split the ground set V into
+L sets according to class labels"), calls the per-class routines, and joins the
+per-class blocks into one assignment vector ("Joint subset", Algorithm 1).
+
+Nothing in the CUDA library imports this module and this module imports
+nothing from the library.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+from concurrent.futures import ThreadPoolExecutor
+from typing import List, Optional, Sequence, Tuple
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = [os.path.join(_HERE, "rcd_oracle.c"), os.path.join(_HERE, "rcd_oracle_typed.inc")]
+_SO = os.path.join(_HERE, "librcd_oracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (no fast-math, no FP contraction)."""
+    newest = max(os.path.getmtime(p) for p in _SRC)
+    if force or not os.path.exists(_SO) or os.path.getmtime(_SO) < newest:
+        tmp = _SO + ".tmp.%d" % os.getpid()
+        subprocess.check_call(["gcc", "-O2", "-std=c99", "-fPIC", "-shared", "-fno-fast-math",
+                               "-ffp-contract=off", "-o", tmp, _SRC[0], "-lm"])
+        os.replace(tmp, _SO)
+    return _SO
+
+
+def _load():
+    global _lib
+    if _lib is not None:
+        return _lib
+    lib = C.CDLL(build())
+    i64, i32, dbl = C.c_int64, C.c_int32, C.c_double
+    P = C.c_void_p
+    lib.rcd_oracle_similarity_i8.argtypes = [P, i64, i64, P]
+    lib.rcd_oracle_similarity_bf16.argtypes = [P, i64, i64, P]
+    lib.rcd_oracle_quotas.argtypes = [i64, P, i32, P]
+    for suf, ret in (("i64", i64), ("f64", dbl)):
+        f = getattr(lib, "rcd_oracle_f_" + suf)
+        f.argtypes = [P, i64, P, i64]
+        f.restype = ret
+        for name in ("rcd_oracle_partition_plain_", "rcd_oracle_partition_incremental_"):
+            g = getattr(lib, name + suf)
+            g.argtypes = [P, i64, i32, P, P, P, P, P, i64]
+            g.restype = i64
+        r = getattr(lib, "rcd_oracle_replay_" + suf)
+        r.argtypes = [P, i64, i32, P, P, P, i64, dbl, P, P]
+        r.restype = i64
+        q = getattr(lib, "rcd_oracle_gains_" + suf)
+        q.argtypes = [P, i64, P, i64, P]
+        q.restype = None
+    _lib = lib
+    return lib
+
+
+def _ptr(a: np.ndarray):
+    return a.ctypes.data_as(C.c_void_p)
+
+
+def _suffix(S: np.ndarray) -> str:
+    if S.dtype == np.int64:
+        return "i64"
+    if S.dtype == np.float64:
+        return "f64"
+    raise TypeError("S must be int64 or float64, got %s" % S.dtype)
+
+
+# --------------------------------------------------------------------------- per-class pieces
+
+def similarity(X: np.ndarray) -> np.ndarray:
+    """S = X X^T for one class.  int8 -> int64 (exact); uint16 bf16 bits -> float64."""
+    lib = _load()
+    X = np.ascontiguousarray(X)
+    M, d = X.shape
+    if X.dtype == np.int8:
+        S = np.empty((M, M), dtype=np.int64)
+        lib.rcd_oracle_similarity_i8(_ptr(X), M, d, _ptr(S))
+    elif X.dtype == np.uint16:
+        S = np.empty((M, M), dtype=np.float64)
+        lib.rcd_oracle_similarity_bf16(_ptr(X), M, d, _ptr(S))
+    else:
+        raise TypeError("features must be int8 or uint16 (bf16 bits)")
+    return S
+
+
+def quotas(M: int, capacities: Sequence[float]) -> np.ndarray:
+    """Integer quotas C_{l,j} of one class of M samples (largest-remainder rule)."""
+    lib = _load()
+    r = np.ascontiguousarray(capacities, dtype=np.float64)
+    out = np.empty(len(r), dtype=np.int32)
+    lib.rcd_oracle_quotas(int(M), _ptr(r), len(r), _ptr(out))
+    return out
+
+
+def f_plain(S: np.ndarray, members: Sequence[int]):
+    """f(A) from the plain facility-location definition."""
+    lib = _load()
+    S = np.ascontiguousarray(S)
+    m = np.ascontiguousarray(members, dtype=np.int32)
+    return getattr(lib, "rcd_oracle_f_" + _suffix(S))(_ptr(S), S.shape[0], _ptr(m), len(m))
+
+
+def gains_plain(S: np.ndarray, members: Sequence[int]) -> np.ndarray:
+    """f(A u {v}) - f(A) for every v, from the plain definition."""
+    lib = _load()
+    S = np.ascontiguousarray(S)
+    m = np.ascontiguousarray(members, dtype=np.int32)
+    out = np.empty(S.shape[0], dtype=S.dtype)
+    getattr(lib, "rcd_oracle_gains_" + _suffix(S))(_ptr(S), S.shape[0], _ptr(m), len(m), _ptr(out))
+    return out
+
+
+def partition_class(S: np.ndarray, C_quota: Sequence[int], variant: str = "plain", max_picks: int = -1):
+    """Algorithm 1 on one class.  Returns (assign[M], order_j[T], order_v[T], fvals[W]).
+
+    ``max_picks >= 0`` stops the loop after that many picks (bounded timing sample)."""
+    lib = _load()
+    S = np.ascontiguousarray(S)
+    M = S.shape[0]
+    q = np.ascontiguousarray(C_quota, dtype=np.int32)
+    W = len(q)
+    assign = np.empty(M, dtype=np.int32)
+    oj = np.empty(max(M, 1), dtype=np.int32)
+    ov = np.empty(max(M, 1), dtype=np.int32)
+    fv = np.empty(W, dtype=S.dtype)
+    name = {"plain": "rcd_oracle_partition_plain_", "incremental": "rcd_oracle_partition_incremental_"}[variant]
+    T = getattr(lib, name + _suffix(S))(_ptr(S), M, W, _ptr(q), _ptr(assign), _ptr(oj), _ptr(ov), _ptr(fv),
+                                         int(max_picks))
+    return assign, oj[:T].copy(), ov[:T].copy(), fv
+
+
+def replay_class(S: np.ndarray, C_quota: Sequence[int], order_j: Sequence[int], order_v: Sequence[int],
+                 rel_tol: float):
+    """Teacher-forced check of a pick sequence.  Returns (first_bad_step or -1, stats[4], fvals[W])."""
+    lib = _load()
+    S = np.ascontiguousarray(S)
+    q = np.ascontiguousarray(C_quota, dtype=np.int32)
+    oj = np.ascontiguousarray(order_j, dtype=np.int32)
+    ov = np.ascontiguousarray(order_v, dtype=np.int32)
+    stats = np.zeros(4, dtype=np.float64)
+    fv = np.empty(len(q), dtype=S.dtype)
+    bad = getattr(lib, "rcd_oracle_replay_" + _suffix(S))(_ptr(S), S.shape[0], len(q), _ptr(q), _ptr(oj), _ptr(ov),
+                                                         len(oj), float(rel_tol), _ptr(stats), _ptr(fv))
+    return int(bad), stats, fv
+
+
+# --------------------------------------------------------------------------- whole dataset
+
+def split_by_label(labels: np.ndarray, L: int) -> List[np.ndarray]:
+    """V -> V_1..V_L; inside a class the samples keep their dataset order."""
+    groups: List[List[int]] = [[] for _ in range(L)]
+    for idx, lab in enumerate(np.asarray(labels).tolist()):
+        groups[lab].append(idx)
+    return [np.asarray(g, dtype=np.int64) for g in groups]
+
+
+class PartitionResult:
+    def __init__(self, N: int, L: int, W: int, value_dtype):
+        self.assignment = np.full(N, -1, dtype=np.int32)       # block of every sample
+        self.order = np.full(N, -1, dtype=np.int32)            # per class (class-major), global ids in pick order
+        self.order_block = np.full(N, -1, dtype=np.int32)      # block of each pick, same layout
+        self.class_offsets = np.zeros(L + 1, dtype=np.int64)
+        self.part_values = np.zeros((L, W), dtype=value_dtype)  # f(A_j^l)
+        self.quotas = np.zeros((L, W), dtype=np.int32)
+
+    @property
+    def total(self):
+        return self.part_values.sum()
+
+
+def partition(features: np.ndarray, labels: np.ndarray, capacities: Sequence[float], L: int,
+              variant: str = "incremental", threads: int = 1,
+              classes: Optional[Sequence[int]] = None, max_picks: int = -1) -> PartitionResult:
+    """Algorithm 1 over the whole dataset: classes handled one after another
+    (or one per thread: they are independent), blocks joined at the end.
+
+    ``classes`` restricts the run to some classes (others stay -1 / zero);
+    ``max_picks`` truncates every class's loop (bounded timing sample)."""
+    features = np.ascontiguousarray(features)
+    N = features.shape[0]
+    W = len(capacities)
+    vdt = np.int64 if features.dtype == np.int8 else np.float64
+    groups = split_by_label(labels, L)
+    res = PartitionResult(N, L, W, vdt)
+    res.class_offsets[1:] = np.cumsum([len(g) for g in groups])
+    todo = list(range(L)) if classes is None else list(classes)
+
+    def one(l: int):
+        ids = groups[l]
+        M = len(ids)
+        q = quotas(M, capacities)
+        if M == 0:
+            return l, q, None
+        S = similarity(features[ids])
+        return l, q, partition_class(S, q, variant, max_picks)
+
+    if threads > 1:
+        with ThreadPoolExecutor(max_workers=threads) as ex:
+            outs = list(ex.map(one, todo))
+    else:
+        outs = [one(l) for l in todo]
+    for l, q, out in outs:
+        res.quotas[l] = q
+        if out is None:
+            continue
+        assign, oj, ov, fv = out
+        ids = groups[l]
+        res.assignment[ids] = assign
+        o = int(res.class_offsets[l])
+        res.order[o:o + len(ov)] = ids[ov]
+        res.order_block[o:o + len(oj)] = oj
+        res.part_values[l] = fv
+    return res
+
+
+def objective(features: np.ndarray, labels: np.ndarray, assignment: np.ndarray, W: int, L: int) -> np.ndarray:
+    """f(A_j^l) for all (l, j), recomputed from the plain definition given an assignment."""
+    features = np.ascontiguousarray(features)
+    vdt = np.int64 if features.dtype == np.int8 else np.float64
+    out = np.zeros((L, W), dtype=vdt)
+    groups = split_by_label(labels, L)
+    for l, ids in enumerate(groups):
+        if len(ids) == 0:
+            continue
+        S = similarity(features[ids])
+        a = np.asarray(assignment)[ids]
+        for j in range(W):
+            out[l, j] = f_plain(S, np.nonzero(a == j)[0])
+    return out
