@@ -1,0 +1,178 @@
+/*
+ * rcd.h -- C ABI of the B200 (sm_100a) library for the resource-constrained
+ * submodular data partition of RCD-SGD (Algorithm 1, "Ratio-Constrained
+ * submodular partitioning", with the facility-location objective of Section 4,
+ * item 2).
+ *
+ * Conventions
+ *   - "dev" pointers are CUDA device pointers on the context's device; "host"
+ *     pointers are ordinary host memory.  The caller owns every buffer,
+ *     including the workspace; the library never frees or keeps them.
+ *   - `cuda_stream` is a cudaStream_t passed as void* (NULL = default stream).
+ *     Unless stated otherwise a call only enqueues work on that stream and
+ *     returns; outputs are valid once the stream has been synchronised.
+ *   - Argument errors are reported synchronously (nothing is launched, nothing is
+ *     written).  A CUDA runtime failure returns RCD_ERR_CUDA.  Errors detected on
+ *     the device land in a status word and are returned by rcd_sync_status().
+ *   - No exception crosses this boundary and there is no CPU fallback: a
+ *     configuration the kernels do not cover returns RCD_ERR_UNSUPPORTED.
+ *   - Not thread-safe per context: use one context per host thread.
+ *
+ * Readings of the paper fixed by this library (the paper is silent on each):
+ *   f(A) = sum_{i in V_l} max(0, max_{v' in A} S[i][v']),  f(empty) = 0;
+ *   argmin over blocks and argmax over samples break ties toward the lowest index;
+ *   quotas by largest remainder (rcd_quotas).
+ */
+#ifndef RCD_H_
+#define RCD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define RCD_API __attribute__((visibility("default")))
+#else
+#define RCD_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    RCD_OK = 0,
+    RCD_ERR_INVALID_ARG = 1,
+    RCD_ERR_UNSUPPORTED = 2,
+    RCD_ERR_WORKSPACE_TOO_SMALL = 3,
+    RCD_ERR_CUDA = 4,
+    RCD_ERR_TIMEOUT = 5,
+    RCD_ERR_INTERNAL = 6
+} rcd_status;
+
+/* Feature element type.  It also fixes the arithmetic of everything downstream:
+ *   RCD_FEAT_I8   int8 features, S = dot product in int32 (exact), gains and f in int64 (exact);
+ *   RCD_FEAT_BF16 bfloat16 features (rows L2-normalised by the caller, so the dot product is the
+ *                 cosine), S accumulated and stored in fp32, gains in fp32, f tracked in fp64.  */
+typedef enum { RCD_FEAT_I8 = 0, RCD_FEAT_BF16 = 1 } rcd_feat_dtype;
+
+typedef struct {
+    int32_t sweep_batch_max;   /* blocks whose gains one pass over S may refresh: 1,2,4 or 8; 0 = default (8) */
+    int32_t similarity_path;   /* 0 = tensor-core kernel when the shape allows, 2 = always the generic kernel */
+    int32_t profile;           /* 0 off; 1 time the phases of rcd_partition; 2 also time every sweep launch */
+    int32_t reserved[13];      /* must be 0 */
+} rcd_config;
+
+/* Timings and counters of the last rcd_partition / rcd_partition_host on a context (profile >= 1). */
+typedef struct {
+    double  total_ms;          /* whole call, first to last kernel, on the call's stream */
+    double  group_ms;          /* class split + feature gather */
+    double  similarity_ms;     /* similarity kernel(s) */
+    double  greedy_ms;         /* all greedy steps */
+    double  sweep_ms;          /* profile 2: summed duration of the sweep launches that had work */
+    int64_t sweep_launches;    /* profile 2: number of those launches */
+    int64_t sweep_bytes;       /* bytes of S and of coverage vectors those launches had to read */
+    int64_t sweep_elem_ops;    /* (element of S) x (block refreshed) pairs those launches evaluated */
+    int64_t kernel_launches;   /* kernels this library launched during the call */
+    int64_t steps;             /* greedy steps executed (= largest class size) */
+    int64_t reserved[6];
+} rcd_profile;
+
+typedef struct rcd_ctx rcd_ctx;
+
+/* ---- context ------------------------------------------------------------------------------ */
+
+/* Creates a context bound to CUDA device `cuda_device` (it owns only a few events and a small
+ * pinned staging buffer).  `cfg_or_null` NULL = defaults.  Fails with RCD_ERR_UNSUPPORTED on a
+ * device that is not compute capability 10.x, RCD_ERR_CUDA when no device can be used. */
+RCD_API rcd_status rcd_create(rcd_ctx **out, int cuda_device, const rcd_config *cfg_or_null);
+RCD_API void rcd_destroy(rcd_ctx *ctx);
+/* Text of the last error on this context (owned by the context; "" if none). NULL ctx allowed. */
+RCD_API const char *rcd_last_error(const rcd_ctx *ctx);
+RCD_API const char *rcd_version(void);
+
+/* Waits for `cuda_stream` and returns the device-side status of the last call on the context. */
+RCD_API rcd_status rcd_sync_status(rcd_ctx *ctx, void *cuda_stream);
+/* Waits for the events of the last profiled call and fills `out`. */
+RCD_API rcd_status rcd_get_profile(rcd_ctx *ctx, rcd_profile *out);
+
+/* ---- quotas (Algorithm 1: "Constraint C_{l,j} = |V_l| r_j / sum_j r_j") -------------------- */
+
+/* Host-only.  Integer quotas of one class of M samples over W blocks with capacity ratios
+ * `capacities_host[W]` (finite, > 0), by largest remainder in IEEE double: shares
+ * q_j = M*r_j/(r_0+r_1+...) are floored and the left-over units go one each to the largest
+ * fractional parts, ties to the lowest j.  sum_j quotas[j] == M.  No GPU is touched. */
+RCD_API rcd_status rcd_quotas(int64_t M, const double *capacities_host, int32_t W, int32_t *quotas_host_out);
+
+/* ---- similarity (Section 3.1 / Section 4 item 2: sim(v, v') from the feature vectors) ------ */
+
+/* S_b = X_b X_b^T for `batch` classes of equal size.
+ *   X_dev  [batch][M][d] row-major, int8 or bf16 (16-byte aligned base)
+ *   S_dev  [batch][M][ldS] row-major, int32 (I8) or fp32 (BF16); ldS >= M, ldS % 4 == 0;
+ *          columns M..ldS-1 of every row are written as 0.
+ * I8 requires 16384*d < 2^31 so that S cannot overflow int32. */
+RCD_API rcd_status rcd_similarity(rcd_ctx *ctx, const void *X_dev, rcd_feat_dtype dtype, int64_t M, int64_t d,
+                          int64_t batch, void *S_dev, int64_t ldS, void *cuda_stream);
+
+/* ---- partition (Algorithm 1 + GreedyStep, facility location) ------------------------------ */
+
+/* Upper bound of the workspace rcd_partition needs for N samples of width d in L classes none
+ * larger than M_max, W blocks.  (rcd_partition recomputes the exact need from the label counts
+ * and returns RCD_ERR_WORKSPACE_TOO_SMALL if a class was larger than promised.) */
+RCD_API rcd_status rcd_partition_workspace_bytes(rcd_ctx *ctx, rcd_feat_dtype dtype, int64_t N, int64_t d,
+                                         int32_t L, int64_t M_max, int32_t W, size_t *bytes_out);
+
+/* Partitions every class of the dataset into W blocks.
+ *   features_dev [N][d] row-major; labels_dev [N], each in [0, L) (classes may be empty and of
+ *   unequal size; inside a class samples keep their dataset order, which fixes tie-breaks);
+ *   capacities_host [W] the ratios r_j (finite, > 0).
+ * Outputs (device):
+ *   assignment_dev [N]            block of every sample, in [0, W)
+ *   order_dev_or_null [N]         class-major (ascending label); inside a class the dataset
+ *                                 indices of its samples in the order they were picked
+ *   part_values_dev_or_null [L][W] tracked f(A_j^l): int64 (I8) or double (BF16)
+ * workspace_dev: 256-byte aligned, at least rcd_partition_workspace_bytes.
+ * The call blocks once, briefly, on `cuda_stream` to read the L class sizes back (they fix the
+ * launch shapes); everything after that is only enqueued.  Per class and per pick it runs:
+ * choose the non-full block of least f; (re)compute the marginal gains
+ * sum_i max(0, S[v][i] - cover_p[i]) of every unassigned v for that block, and in the same
+ * pass over S for other non-full blocks whose stored gains are out of date (a block's gains
+ * only change when the block itself receives a sample); argmax with lowest-index ties;
+ * fold row v* into the block's coverage vector and update counts. */
+RCD_API rcd_status rcd_partition(rcd_ctx *ctx, const void *features_dev, rcd_feat_dtype dtype, int64_t N, int64_t d,
+                         const int32_t *labels_dev, int32_t L, const double *capacities_host, int32_t W,
+                         int32_t *assignment_dev, int32_t *order_dev_or_null, void *part_values_dev_or_null,
+                         void *workspace_dev, size_t workspace_bytes, void *cuda_stream);
+
+/* Same computation with HOST inputs and outputs: copies features and labels to the device
+ * (staging areas inside the workspace), runs rcd_partition, copies the results back and
+ * synchronises the stream before returning, so the host outputs are valid on return.
+ * Pinned host memory makes the copies asynchronous; pageable memory works too. */
+RCD_API rcd_status rcd_partition_host_workspace_bytes(rcd_ctx *ctx, rcd_feat_dtype dtype, int64_t N, int64_t d,
+                                              int32_t L, int64_t M_max, int32_t W, size_t *bytes_out);
+RCD_API rcd_status rcd_partition_host(rcd_ctx *ctx, const void *features_host, rcd_feat_dtype dtype, int64_t N,
+                              int64_t d, const int32_t *labels_host, int32_t L,
+                              const double *capacities_host, int32_t W, int32_t *assignment_host,
+                              int32_t *order_host_or_null, void *part_values_host_or_null,
+                              void *workspace_dev, size_t workspace_bytes, void *cuda_stream);
+
+/* ---- objective (Section 4 item 2: f(A) = sum_{v in V_l} max_{v' in A} sim(v, v')) ---------- */
+
+RCD_API rcd_status rcd_objective_workspace_bytes(rcd_ctx *ctx, rcd_feat_dtype dtype, int64_t N, int64_t d,
+                                         int32_t L, int64_t M_max, int32_t W, size_t *bytes_out);
+
+/* Recomputes f(A_j^l) for every class l and block j from the plain definition, given an
+ * assignment (values in [0, W); a negative entry means "in no block").  Independent of the
+ * greedy state: it rebuilds S and takes, per row i and block j, the maximum over the block's
+ * members.
+ *   part_values_dev [L][W]  int64 (I8) or double (BF16)
+ *   total_dev               one int64 or double: the sum over all (l, j)
+ * Blocks once on the stream, like rcd_partition, to read the class sizes. */
+RCD_API rcd_status rcd_objective(rcd_ctx *ctx, const void *features_dev, rcd_feat_dtype dtype, int64_t N, int64_t d,
+                         const int32_t *labels_dev, int32_t L, const int32_t *assignment_dev, int32_t W,
+                         void *part_values_dev, void *total_dev, void *workspace_dev,
+                         size_t workspace_bytes, void *cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RCD_H_ */

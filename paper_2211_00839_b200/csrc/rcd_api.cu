@@ -1,0 +1,525 @@
+// Host side of the C ABI: argument checks, workspace layout, quotas, and the order in which the
+// kernels of the other translation units are enqueued.
+#include "rcd_internal.h"
+
+#include <math.h>
+#include <stdarg.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <algorithm>
+#include <new>
+
+namespace rcd {
+
+rcd_status fail(rcd_ctx *ctx, rcd_status st, const char *fmt, ...)
+{
+    if (ctx) {
+        char buf[512];
+        va_list ap;
+        va_start(ap, fmt);
+        vsnprintf(buf, sizeof buf, fmt, ap);
+        va_end(ap);
+        ctx->err = buf;
+    }
+    return st;
+}
+
+rcd_status cuda_fail(rcd_ctx *ctx, cudaError_t e, const char *what)
+{
+    return fail(ctx, RCD_ERR_CUDA, "CUDA error %d (%s) in %s", (int)e, cudaGetErrorString(e), what);
+}
+
+// Bump allocator over the caller's workspace.
+struct Carver {
+    unsigned char *base;
+    size_t off = 0;
+    template <typename T> T *take(size_t count)
+    {
+        off = align_up(off);
+        T *p = base ? reinterpret_cast<T *>(base + off) : nullptr;
+        off += count * sizeof(T);
+        return p;
+    }
+};
+
+size_t layout_workspace(void *base, rcd_feat_dtype dtype, const Sizes &sz, Workspace *ws)
+{
+    Carver c{static_cast<unsigned char *>(base)};
+    const size_t L = (size_t)std::max<int32_t>(sz.L, 1), W = (size_t)std::max<int32_t>(sz.W, 1);
+    const size_t N = (size_t)std::max<int64_t>(sz.N, 1);
+    const size_t sElem = 4;                                     // int32 / fp32
+    const size_t gElem = dtype == RCD_FEAT_I8 ? 8 : 4;          // int64 / fp32
+    Workspace w{};
+    // the head does not depend on the class sizes: it is used before they are known
+    w.status = c.take<int32_t>(4);
+    w.counts = c.take<int32_t>(L);
+    w.nSweep = c.take<int32_t>(4);
+    // everything below is placed once the class sizes are known
+    w.desc = c.take<ClassDesc>(L);
+    w.chunkHist = c.take<int32_t>((size_t)std::max<int32_t>(sz.nChunks, 1) * L);
+    w.perm = c.take<int32_t>(N);
+    w.Xs = c.take<unsigned char>(N * (size_t)sz.d * feat_bytes(dtype));
+    w.S = c.take<unsigned char>((size_t)std::max<int64_t>(sz.sElems, 1) * sElem);
+    w.cover = c.take<unsigned char>((size_t)std::max<int64_t>(sz.vElems, 1) * sElem);
+    w.gains = c.take<unsigned char>((size_t)std::max<int64_t>(sz.vElems, 1) * gElem);
+    w.fval = c.take<unsigned char>(L * W * 8);
+    w.cnt = c.take<int32_t>(L * W);
+    w.quota = c.take<int32_t>(L * W);
+    w.valid = c.take<uint8_t>(L * W);
+    w.cand = c.take<int32_t>(N);
+    w.pos = c.take<int32_t>(N);
+    w.nR = c.take<int32_t>(L);
+    w.jstar = c.take<int32_t>(L);
+    w.sweepN = c.take<int32_t>(L);
+    w.sweepParts = c.take<int32_t>(L * kMaxSweepBatch);
+    w.rowCtr = c.take<int32_t>(L);
+    w.sweepList = c.take<int32_t>(2 * L);
+    w.stepBytes = c.take<unsigned long long>((size_t)sz.maxM + 1);
+    w.stepOps = c.take<unsigned long long>((size_t)sz.maxM + 1);
+    w.bytes = align_up(c.off);
+    if (ws) *ws = w;
+    return w.bytes;
+}
+
+static int32_t chunks_for(int64_t N) { return (int32_t)((N + kGroupChunk - 1) / kGroupChunk); }
+
+// Sizes for the promise "no class larger than Mmax".
+static Sizes bound_sizes(int64_t N, int64_t d, int32_t L, int64_t Mmax, int32_t W)
+{
+    Sizes sz{};
+    sz.N = N; sz.d = d; sz.L = L; sz.W = W;
+    if (Mmax > N) Mmax = N;
+    sz.maxM = Mmax;
+    sz.sElems = N * (int64_t)pad4(Mmax);                  // sum M_l * ld_l <= N * pad4(Mmax)
+    sz.vElems = (int64_t)W * (N + 3LL * L);               // sum W * ld_l,  ld_l <= M_l + 3
+    sz.nChunks = chunks_for(N);
+    return sz;
+}
+
+static rcd_status check_common(rcd_ctx *ctx, rcd_feat_dtype dtype, int64_t N, int64_t d, int32_t L, int32_t W)
+{
+    if (!ctx) return RCD_ERR_INVALID_ARG;
+    if (dtype != RCD_FEAT_I8 && dtype != RCD_FEAT_BF16) return fail(ctx, RCD_ERR_INVALID_ARG, "unknown feature dtype %d", (int)dtype);
+    if (N < 0 || N > 0x7fffffffLL) return fail(ctx, RCD_ERR_INVALID_ARG, "N=%lld out of range", (long long)N);
+    if (d <= 0) return fail(ctx, RCD_ERR_INVALID_ARG, "d=%lld must be positive", (long long)d);
+    if (L <= 0) return fail(ctx, RCD_ERR_INVALID_ARG, "L=%d must be positive", L);
+    if (W <= 0) return fail(ctx, RCD_ERR_INVALID_ARG, "W=%d must be positive", W);
+    if (W > 1024) return fail(ctx, RCD_ERR_UNSUPPORTED, "W=%d: at most 1024 blocks are supported", W);
+    if (dtype == RCD_FEAT_I8 && 16384LL * d > 0x7fffffffLL)
+        return fail(ctx, RCD_ERR_UNSUPPORTED, "d=%lld: an int8 dot product could overflow int32", (long long)d);
+    return RCD_OK;
+}
+
+static rcd_status check_capacities(rcd_ctx *ctx, const double *cap, int32_t W)
+{
+    if (!cap) return fail(ctx, RCD_ERR_INVALID_ARG, "capacities is null");
+    for (int32_t j = 0; j < W; ++j)
+        if (!(cap[j] > 0.0) || !std::isfinite(cap[j]))
+            return fail(ctx, RCD_ERR_INVALID_ARG, "capacity %d is not a finite positive number", j);
+    return RCD_OK;
+}
+
+// Largest-remainder quotas.  Plain IEEE double operations in a fixed order.
+static void quotas_host(int64_t M, const double *r, int32_t W, int32_t *out)
+{
+    volatile double total = 0.0;
+    for (int32_t j = 0; j < W; ++j) total = total + r[j];
+    std::vector<double> rem((size_t)W);
+    int64_t used = 0;
+    for (int32_t j = 0; j < W; ++j) {
+        volatile double scaled = (double)M * r[j];
+        volatile double share = scaled / total;
+        double whole = floor(share);
+        out[j] = (int32_t)whole;
+        rem[j] = share - whole;
+        used += out[j];
+    }
+    for (int64_t extra = M - used; extra > 0; --extra) {
+        int32_t pick = -1;
+        for (int32_t j = 0; j < W; ++j)
+            if (rem[j] >= 0.0 && (pick < 0 || rem[j] > rem[pick])) pick = j;
+        out[pick] += 1;
+        rem[pick] = -1.0;
+    }
+    for (int64_t over = used - M; over > 0; --over) {      // a share rounded up to an integer: give one back
+        int32_t pick = -1;
+        for (int32_t j = 0; j < W; ++j)
+            if (out[j] > 0 && rem[j] >= 0.0 && (pick < 0 || rem[j] <= rem[pick])) pick = j;
+        out[pick] -= 1;
+        rem[pick] = -1.0;
+    }
+}
+
+// Shared front half of rcd_partition and rcd_objective: class sizes, descriptors, workspace
+// layout, stable split, feature gather, similarity.
+struct Prepared {
+    Sizes sz{};
+    Workspace ws{};
+    std::vector<ClassDesc> desc;
+};
+
+static rcd_status prepare(rcd_ctx *ctx, const void *features, rcd_feat_dtype dtype, int64_t N, int64_t d,
+                          const int32_t *labels, int32_t L, int32_t W, void *workspace, size_t workspaceBytes,
+                          cudaStream_t st, Prepared *out)
+{
+    if (((uintptr_t)workspace) % kAlign != 0) return fail(ctx, RCD_ERR_INVALID_ARG, "workspace must be 256-byte aligned");
+    // head of the workspace: status, counts
+    Sizes head{};
+    head.N = N; head.d = d; head.L = L; head.W = W; head.nChunks = chunks_for(N);
+    Workspace hw{};
+    Sizes tiny = head;
+    layout_workspace(workspace, dtype, tiny, &hw);
+    size_t headBytes = (size_t)((unsigned char *)hw.desc - (unsigned char *)workspace);
+    if (workspaceBytes < headBytes) return fail(ctx, RCD_ERR_WORKSPACE_TOO_SMALL, "workspace smaller than its %zu-byte head", headBytes);
+    if ((size_t)L > ctx->hostStageInts) return fail(ctx, RCD_ERR_UNSUPPORTED, "L=%d exceeds the %zu classes the context can stage", L, ctx->hostStageInts);
+
+    RCD_CUDA(ctx, cudaMemsetAsync(hw.status, 0, 4 * sizeof(int32_t), st));
+    RCD_CUDA(ctx, cudaMemsetAsync(hw.counts, 0, (size_t)L * sizeof(int32_t), st));
+    rcd_status rs = launch_count_labels(ctx, labels, N, L, hw.counts, hw.status, st);
+    if (rs != RCD_OK) return rs;
+    RCD_CUDA(ctx, cudaMemcpyAsync(ctx->hostStage, hw.counts, (size_t)L * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+    RCD_CUDA(ctx, cudaMemcpyAsync(ctx->hostStage + L, hw.status, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+    RCD_CUDA(ctx, cudaStreamSynchronize(st));
+    if (ctx->hostStage[L] & kDevBadLabel) return fail(ctx, RCD_ERR_INVALID_ARG, "a label lies outside [0, %d)", L);
+
+    Prepared &P = *out;
+    P.desc.resize((size_t)L);
+    Sizes sz = head;
+    int64_t row = 0, sOff = 0, vOff = 0, maxM = 0;
+    for (int32_t l = 0; l < L; ++l) {
+        ClassDesc c{};
+        c.M = ctx->hostStage[l];
+        c.ld = pad4(c.M);
+        c.row0 = (int32_t)row;
+        c.sOff = sOff;
+        c.vOff = vOff;
+        row += c.M;
+        sOff += (int64_t)c.M * c.ld;
+        vOff += (int64_t)W * c.ld;
+        maxM = std::max<int64_t>(maxM, c.M);
+        P.desc[(size_t)l] = c;
+    }
+    if (row != N) return fail(ctx, RCD_ERR_INTERNAL, "class sizes sum to %lld, expected %lld", (long long)row, (long long)N);
+    sz.sElems = sOff; sz.vElems = vOff; sz.maxM = maxM;
+    size_t need = layout_workspace(workspace, dtype, sz, &P.ws);
+    if (need > workspaceBytes)
+        return fail(ctx, RCD_ERR_WORKSPACE_TOO_SMALL, "workspace has %zu bytes, the class sizes found need %zu", workspaceBytes, need);
+    P.sz = sz;
+    ctx->statusDev = P.ws.status;
+
+    RCD_CUDA(ctx, cudaMemcpyAsync(P.ws.desc, P.desc.data(), (size_t)L * sizeof(ClassDesc), cudaMemcpyHostToDevice, st));
+    rs = launch_stable_split(ctx, labels, N, L, sz.nChunks, P.ws.chunkHist, P.ws.desc, P.ws.perm, st);
+    if (rs != RCD_OK) return rs;
+    rs = launch_gather_rows(ctx, features, P.ws.perm, N, d * (int64_t)feat_bytes(dtype), P.ws.Xs, st);
+    if (rs != RCD_OK) return rs;
+    if (ctx->cfg.profile >= 1) RCD_CUDA(ctx, cudaEventRecord(ctx->evPhase[1], st));
+    SimClasses cls{};
+    cls.src.table = P.ws.desc;
+    cls.L = L;
+    cls.maxM = maxM;
+    for (const auto &c : P.desc) cls.tiles128 += (int64_t)((c.M + 127) / 128) * ((c.M + 127) / 128);
+    rs = launch_similarity(ctx, P.ws.Xs, dtype, N, d, cls, P.ws.S, st);
+    if (rs != RCD_OK) return rs;
+    if (ctx->cfg.profile >= 1) RCD_CUDA(ctx, cudaEventRecord(ctx->evPhase[2], st));
+    return RCD_OK;
+}
+
+}  // namespace rcd
+
+using namespace rcd;
+
+extern "C" {
+
+const char *rcd_version(void) { return "rcd-b200 0.1 (sm_100a)"; }
+
+const char *rcd_last_error(const rcd_ctx *ctx) { return ctx ? ctx->err.c_str() : ""; }
+
+rcd_status rcd_create(rcd_ctx **out, int cuda_device, const rcd_config *cfg)
+{
+    if (!out) return RCD_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (cfg) {
+        if (cfg->sweep_batch_max != 0 && cfg->sweep_batch_max != 1 && cfg->sweep_batch_max != 2 &&
+            cfg->sweep_batch_max != 4 && cfg->sweep_batch_max != 8)
+            return RCD_ERR_INVALID_ARG;
+        if (cfg->similarity_path != 0 && cfg->similarity_path != 2) return RCD_ERR_INVALID_ARG;
+        if (cfg->profile < 0 || cfg->profile > 2) return RCD_ERR_INVALID_ARG;
+        for (int i = 0; i < 13; ++i) if (cfg->reserved[i] != 0) return RCD_ERR_INVALID_ARG;
+    }
+    int count = 0;
+    if (cudaGetDeviceCount(&count) != cudaSuccess || cuda_device < 0 || cuda_device >= count) {
+        cudaGetLastError();
+        return RCD_ERR_CUDA;
+    }
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, cuda_device) != cudaSuccess) return RCD_ERR_CUDA;
+    if (prop.major != 10) return RCD_ERR_UNSUPPORTED;     // the kernels are built for sm_100a only
+    if (cudaSetDevice(cuda_device) != cudaSuccess) return RCD_ERR_CUDA;
+    rcd_ctx *ctx = new (std::nothrow) rcd_ctx();
+    if (!ctx) return RCD_ERR_INTERNAL;
+    ctx->device = cuda_device;
+    ctx->smCount = prop.multiProcessorCount;
+    ctx->maxSmemOptin = (int)prop.sharedMemPerBlockOptin;
+    if (cfg) ctx->cfg = *cfg;
+    ctx->hostStageInts = 1 << 20;
+    if (cudaMallocHost((void **)&ctx->hostStage, (ctx->hostStageInts + 16) * sizeof(int32_t)) != cudaSuccess) {
+        delete ctx;
+        return RCD_ERR_CUDA;
+    }
+    for (auto &e : ctx->evPhase)
+        if (cudaEventCreate(&e) != cudaSuccess) { rcd_destroy(ctx); return RCD_ERR_CUDA; }
+    *out = ctx;
+    return RCD_OK;
+}
+
+void rcd_destroy(rcd_ctx *ctx)
+{
+    if (!ctx) return;
+    cudaSetDevice(ctx->device);
+    for (auto &e : ctx->evPhase) if (e) cudaEventDestroy(e);
+    for (auto &e : ctx->evSweep) cudaEventDestroy(e);
+    if (ctx->hostStage) cudaFreeHost(ctx->hostStage);
+    delete ctx;
+}
+
+rcd_status rcd_sync_status(rcd_ctx *ctx, void *cuda_stream)
+{
+    if (!ctx) return RCD_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    RCD_CUDA(ctx, cudaStreamSynchronize(st));
+    if (!ctx->statusDev) return RCD_OK;
+    int32_t word = 0;
+    RCD_CUDA(ctx, cudaMemcpy(&word, ctx->statusDev, sizeof word, cudaMemcpyDeviceToHost));
+    if (word == 0) return RCD_OK;
+    if (word & kDevBadLabel) return fail(ctx, RCD_ERR_INVALID_ARG, "device status %d: label out of range", word);
+    return fail(ctx, RCD_ERR_INTERNAL, "device status %d: greedy state inconsistent", word);
+}
+
+rcd_status rcd_get_profile(rcd_ctx *ctx, rcd_profile *out)
+{
+    if (!ctx || !out) return RCD_ERR_INVALID_ARG;
+    memset(out, 0, sizeof *out);
+    out->kernel_launches = ctx->kernelLaunches;
+    out->steps = ctx->steps;
+    if (!ctx->phaseValid) return RCD_OK;
+    RCD_CUDA(ctx, cudaEventSynchronize(ctx->evPhase[4]));
+    float ms = 0.f;
+    RCD_CUDA(ctx, cudaEventElapsedTime(&ms, ctx->evPhase[0], ctx->evPhase[4])); out->total_ms = ms;
+    RCD_CUDA(ctx, cudaEventElapsedTime(&ms, ctx->evPhase[0], ctx->evPhase[1])); out->group_ms = ms;
+    RCD_CUDA(ctx, cudaEventElapsedTime(&ms, ctx->evPhase[1], ctx->evPhase[2])); out->similarity_ms = ms;
+    RCD_CUDA(ctx, cudaEventElapsedTime(&ms, ctx->evPhase[2], ctx->evPhase[3])); out->greedy_ms = ms;
+    if (ctx->stepBytesDev && ctx->steps > 0) {
+        std::vector<unsigned long long> bytes((size_t)ctx->steps + 1), ops((size_t)ctx->steps + 1);
+        RCD_CUDA(ctx, cudaMemcpy(bytes.data(), ctx->stepBytesDev, bytes.size() * sizeof(unsigned long long), cudaMemcpyDeviceToHost));
+        RCD_CUDA(ctx, cudaMemcpy(ops.data(), ctx->stepOpsDev, ops.size() * sizeof(unsigned long long), cudaMemcpyDeviceToHost));
+        for (int64_t t = 0; t < ctx->steps; ++t) {
+            if (bytes[(size_t)t] == 0) continue;
+            out->sweep_bytes += (int64_t)bytes[(size_t)t];
+            out->sweep_elem_ops += (int64_t)ops[(size_t)t];
+            out->sweep_launches += 1;
+            if (ctx->sweepEventsUsed >= 2 * (t + 1)) {
+                RCD_CUDA(ctx, cudaEventElapsedTime(&ms, ctx->evSweep[(size_t)(2 * t)], ctx->evSweep[(size_t)(2 * t + 1)]));
+                out->sweep_ms += ms;
+            }
+        }
+    }
+    return RCD_OK;
+}
+
+rcd_status rcd_quotas(int64_t M, const double *capacities_host, int32_t W, int32_t *quotas_host_out)
+{
+    if (M < 0 || M > 0x7fffffffLL || W <= 0 || !capacities_host || !quotas_host_out) return RCD_ERR_INVALID_ARG;
+    for (int32_t j = 0; j < W; ++j)
+        if (!(capacities_host[j] > 0.0) || !std::isfinite(capacities_host[j])) return RCD_ERR_INVALID_ARG;
+    quotas_host(M, capacities_host, W, quotas_host_out);
+    return RCD_OK;
+}
+
+rcd_status rcd_similarity(rcd_ctx *ctx, const void *X_dev, rcd_feat_dtype dtype, int64_t M, int64_t d,
+                          int64_t batch, void *S_dev, int64_t ldS, void *cuda_stream)
+{
+    rcd_status rs = check_common(ctx, dtype, 0, d, 1, 1);
+    if (rs != RCD_OK) return rs;
+    if (M < 0 || batch < 0 || M > 0x7fffffffLL) return fail(ctx, RCD_ERR_INVALID_ARG, "M or batch negative");
+    if (M == 0 || batch == 0) return RCD_OK;
+    if (!X_dev || !S_dev) return fail(ctx, RCD_ERR_INVALID_ARG, "null device pointer");
+    if (ldS != pad4(M)) return fail(ctx, RCD_ERR_INVALID_ARG, "ldS must be M rounded up to a multiple of 4 (%d), got %lld", pad4(M), (long long)ldS);
+    if (M * batch > 0x7fffffffLL) return fail(ctx, RCD_ERR_INVALID_ARG, "M*batch too large");
+    if (((uintptr_t)X_dev) % 16 || ((uintptr_t)S_dev) % 16) return fail(ctx, RCD_ERR_INVALID_ARG, "X and S must be 16-byte aligned");
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    RCD_CUDA(ctx, cudaSetDevice(ctx->device));
+    SimClasses cls{};
+    cls.src.table = nullptr;
+    cls.src.uniM = (int32_t)M;
+    cls.src.uniLd = (int32_t)ldS;
+    cls.L = (int32_t)batch;
+    cls.maxM = M;
+    cls.tiles128 = batch * ((M + 127) / 128) * ((M + 127) / 128);
+    ctx->kernelLaunches = 0;
+    return launch_similarity(ctx, X_dev, dtype, M * batch, d, cls, S_dev, st);
+}
+
+rcd_status rcd_partition_workspace_bytes(rcd_ctx *ctx, rcd_feat_dtype dtype, int64_t N, int64_t d, int32_t L,
+                                         int64_t M_max, int32_t W, size_t *bytes_out)
+{
+    rcd_status rs = check_common(ctx, dtype, N, d, L, W);
+    if (rs != RCD_OK) return rs;
+    if (!bytes_out || M_max < 0) return fail(ctx, RCD_ERR_INVALID_ARG, "bad M_max or null output");
+    Sizes sz = bound_sizes(N, d, L, M_max, W);
+    *bytes_out = layout_workspace(nullptr, dtype, sz, nullptr);
+    return RCD_OK;
+}
+
+rcd_status rcd_partition(rcd_ctx *ctx, const void *features_dev, rcd_feat_dtype dtype, int64_t N, int64_t d,
+                         const int32_t *labels_dev, int32_t L, const double *capacities_host, int32_t W,
+                         int32_t *assignment_dev, int32_t *order_dev_or_null, void *part_values_dev_or_null,
+                         void *workspace_dev, size_t workspace_bytes, void *cuda_stream)
+{
+    rcd_status rs = check_common(ctx, dtype, N, d, L, W);
+    if (rs != RCD_OK) return rs;
+    rs = check_capacities(ctx, capacities_host, W);
+    if (rs != RCD_OK) return rs;
+    if (N > 0 && (!features_dev || !labels_dev || !assignment_dev)) return fail(ctx, RCD_ERR_INVALID_ARG, "null device pointer");
+    if (!workspace_dev) return fail(ctx, RCD_ERR_INVALID_ARG, "workspace is null");
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    RCD_CUDA(ctx, cudaSetDevice(ctx->device));
+    ctx->kernelLaunches = 0;
+    ctx->steps = 0;
+    ctx->phaseValid = false;
+    ctx->stepBytesDev = nullptr;
+    ctx->stepOpsDev = nullptr;
+    ctx->sweepEventsUsed = 0;
+    const bool prof = ctx->cfg.profile >= 1;
+    if (prof) RCD_CUDA(ctx, cudaEventRecord(ctx->evPhase[0], st));
+
+    Prepared P;
+    rs = prepare(ctx, features_dev, dtype, N, d, labels_dev, L, W, workspace_dev, workspace_bytes, st, &P);
+    if (rs != RCD_OK) return rs;
+
+    std::vector<int32_t> quota((size_t)L * W);
+    for (int32_t l = 0; l < L; ++l) quotas_host(P.desc[(size_t)l].M, capacities_host, W, quota.data() + (size_t)l * W);
+    RCD_CUDA(ctx, cudaMemcpyAsync(P.ws.quota, quota.data(), quota.size() * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+
+    rs = launch_greedy(ctx, dtype, P.sz, P.ws, P.desc, assignment_dev, order_dev_or_null, st);
+    if (rs != RCD_OK) return rs;
+    if (prof) RCD_CUDA(ctx, cudaEventRecord(ctx->evPhase[3], st));
+    if (part_values_dev_or_null) {
+        if (P.sz.maxM == 0) RCD_CUDA(ctx, cudaMemsetAsync(part_values_dev_or_null, 0, (size_t)L * W * 8, st));
+        else RCD_CUDA(ctx, cudaMemcpyAsync(part_values_dev_or_null, P.ws.fval, (size_t)L * W * 8, cudaMemcpyDeviceToDevice, st));
+    }
+    if (prof) {
+        RCD_CUDA(ctx, cudaEventRecord(ctx->evPhase[4], st));
+        ctx->phaseValid = true;
+    }
+    return RCD_OK;
+}
+
+// Host-buffer variant: staging areas for features, labels and the three outputs sit behind the
+// device workspace proper.
+static size_t host_tail_bytes(rcd_feat_dtype dtype, int64_t N, int64_t d, int32_t L, int32_t W)
+{
+    const size_t featB = align_up((size_t)std::max<int64_t>(N, 1) * (size_t)d * feat_bytes(dtype));
+    const size_t vecB = align_up((size_t)std::max<int64_t>(N, 1) * 4);
+    const size_t valB = align_up((size_t)L * W * 8);
+    return featB + 3 * vecB + valB;
+}
+
+rcd_status rcd_partition_host_workspace_bytes(rcd_ctx *ctx, rcd_feat_dtype dtype, int64_t N, int64_t d, int32_t L,
+                                              int64_t M_max, int32_t W, size_t *bytes_out)
+{
+    rcd_status rs = check_common(ctx, dtype, N, d, L, W);
+    if (rs != RCD_OK) return rs;
+    if (!bytes_out || M_max < 0) return fail(ctx, RCD_ERR_INVALID_ARG, "bad M_max or null output");
+    Sizes sz = bound_sizes(N, d, L, M_max, W);
+    *bytes_out = layout_workspace(nullptr, dtype, sz, nullptr) + host_tail_bytes(dtype, N, d, L, W) + kAlign;
+    return RCD_OK;
+}
+
+rcd_status rcd_partition_host(rcd_ctx *ctx, const void *features_host, rcd_feat_dtype dtype, int64_t N, int64_t d,
+                              const int32_t *labels_host, int32_t L, const double *capacities_host, int32_t W,
+                              int32_t *assignment_host, int32_t *order_host_or_null, void *part_values_host_or_null,
+                              void *workspace_dev, size_t workspace_bytes, void *cuda_stream)
+{
+    rcd_status rs = check_common(ctx, dtype, N, d, L, W);
+    if (rs != RCD_OK) return rs;
+    rs = check_capacities(ctx, capacities_host, W);
+    if (rs != RCD_OK) return rs;
+    if (N > 0 && (!features_host || !labels_host || !assignment_host)) return fail(ctx, RCD_ERR_INVALID_ARG, "null host pointer");
+    if (!workspace_dev || ((uintptr_t)workspace_dev) % kAlign) return fail(ctx, RCD_ERR_INVALID_ARG, "workspace null or not 256-byte aligned");
+    // The staging areas are placed from the END of the workspace so that the inner workspace can
+    // use whatever the true class sizes need.
+    const size_t featB = align_up((size_t)std::max<int64_t>(N, 1) * (size_t)d * feat_bytes(dtype));
+    const size_t vecB = align_up((size_t)std::max<int64_t>(N, 1) * 4);
+    const size_t tail = host_tail_bytes(dtype, N, d, L, W);
+    if (workspace_bytes < tail + kAlign) return fail(ctx, RCD_ERR_WORKSPACE_TOO_SMALL, "workspace smaller than the staging areas (%zu bytes)", tail);
+    size_t innerBytes = (workspace_bytes - tail) / kAlign * kAlign;
+    unsigned char *base = (unsigned char *)workspace_dev;
+    unsigned char *feat = base + innerBytes;
+    int32_t *lab = (int32_t *)(feat + featB);
+    int32_t *asg = (int32_t *)((unsigned char *)lab + vecB);
+    int32_t *ord = (int32_t *)((unsigned char *)asg + vecB);
+    void *val = (unsigned char *)ord + vecB;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    RCD_CUDA(ctx, cudaSetDevice(ctx->device));
+    if (N > 0) {
+        RCD_CUDA(ctx, cudaMemcpyAsync(feat, features_host, (size_t)N * (size_t)d * feat_bytes(dtype), cudaMemcpyHostToDevice, st));
+        RCD_CUDA(ctx, cudaMemcpyAsync(lab, labels_host, (size_t)N * 4, cudaMemcpyHostToDevice, st));
+    }
+    rs = rcd_partition(ctx, feat, dtype, N, d, lab, L, capacities_host, W, asg, order_host_or_null ? ord : nullptr,
+                       part_values_host_or_null ? val : nullptr, workspace_dev, innerBytes, st);
+    if (rs != RCD_OK) return rs;
+    if (N > 0) {
+        RCD_CUDA(ctx, cudaMemcpyAsync(assignment_host, asg, (size_t)N * 4, cudaMemcpyDeviceToHost, st));
+        if (order_host_or_null) RCD_CUDA(ctx, cudaMemcpyAsync(order_host_or_null, ord, (size_t)N * 4, cudaMemcpyDeviceToHost, st));
+    }
+    if (part_values_host_or_null)
+        RCD_CUDA(ctx, cudaMemcpyAsync(part_values_host_or_null, val, (size_t)L * W * 8, cudaMemcpyDeviceToHost, st));
+    return rcd_sync_status(ctx, st);
+}
+
+// Objective scratch: per class and row block, W partial sums.
+static size_t objective_scratch_bytes(int32_t L, int64_t Mmax, int32_t W)
+{
+    size_t blocks = (size_t)((Mmax + 63) / 64);
+    return align_up(std::max<size_t>(1, (size_t)L * blocks * (size_t)W * 8));
+}
+
+rcd_status rcd_objective_workspace_bytes(rcd_ctx *ctx, rcd_feat_dtype dtype, int64_t N, int64_t d, int32_t L,
+                                         int64_t M_max, int32_t W, size_t *bytes_out)
+{
+    rcd_status rs = check_common(ctx, dtype, N, d, L, W);
+    if (rs != RCD_OK) return rs;
+    if (!bytes_out || M_max < 0) return fail(ctx, RCD_ERR_INVALID_ARG, "bad M_max or null output");
+    Sizes sz = bound_sizes(N, d, L, M_max, W);
+    *bytes_out = layout_workspace(nullptr, dtype, sz, nullptr) + objective_scratch_bytes(L, std::min(M_max, N), W);
+    return RCD_OK;
+}
+
+rcd_status rcd_objective(rcd_ctx *ctx, const void *features_dev, rcd_feat_dtype dtype, int64_t N, int64_t d,
+                         const int32_t *labels_dev, int32_t L, const int32_t *assignment_dev, int32_t W,
+                         void *part_values_dev, void *total_dev, void *workspace_dev, size_t workspace_bytes,
+                         void *cuda_stream)
+{
+    rcd_status rs = check_common(ctx, dtype, N, d, L, W);
+    if (rs != RCD_OK) return rs;
+    if (!part_values_dev || !total_dev) return fail(ctx, RCD_ERR_INVALID_ARG, "null output pointer");
+    if (N > 0 && (!features_dev || !labels_dev || !assignment_dev)) return fail(ctx, RCD_ERR_INVALID_ARG, "null device pointer");
+    if (!workspace_dev) return fail(ctx, RCD_ERR_INVALID_ARG, "workspace is null");
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    RCD_CUDA(ctx, cudaSetDevice(ctx->device));
+    const int savedProfile = ctx->cfg.profile;
+    ctx->cfg.profile = 0;
+    Prepared P;
+    rs = prepare(ctx, features_dev, dtype, N, d, labels_dev, L, W, workspace_dev, workspace_bytes, st, &P);
+    ctx->cfg.profile = savedProfile;
+    if (rs != RCD_OK) return rs;
+    size_t scratchB = objective_scratch_bytes(L, P.sz.maxM, W);
+    if (P.ws.bytes + scratchB > workspace_bytes)
+        return fail(ctx, RCD_ERR_WORKSPACE_TOO_SMALL, "workspace has %zu bytes, objective needs %zu", workspace_bytes, P.ws.bytes + scratchB);
+    void *scratch = (unsigned char *)workspace_dev + P.ws.bytes;
+    return launch_objective(ctx, dtype, P.sz, P.ws.desc, P.desc, P.ws.S, P.ws.perm, assignment_dev, part_values_dev,
+                            total_dev, scratch, st);
+}
+
+}  // extern "C"

@@ -1,0 +1,570 @@
+// The greedy loop of Algorithm 1 with the facility-location objective, all classes in lockstep.
+//
+// Per class the device keeps, for every block p: a coverage vector cover_p[i] =
+// max(0, max_{v' in A_p} S[i][v']), the tracked value f_p = sum_i cover_p[i], the count and the
+// quota, and a row of stored marginal gains G_p[v] = sum_i max(0, S[v][i] - cover_p[i])
+// (GreedyStep's f(A_p u {v}) - f(A_p); S is symmetric).  G_p stays correct until block p itself
+// receives a sample, so a pass over S is only needed when the chosen block's row is out of date,
+// and that pass refreshes up to `sweep_batch_max` out-of-date blocks at once.
+//
+// One greedy step t = two launches:
+//   sweep_kernel   persistent CTAs (one per SM) pull row groups of every class that scheduled a
+//                  sweep; each warp streams its rows of S with 128-bit loads against the coverage
+//                  vectors staged in shared memory, reduces with warp shuffles, writes G.
+//   select_kernel  one CTA per class: argmax of G_{j*} over the unassigned samples (warp-shuffle
+//                  reduction, lowest index on ties), coverage / value / count update, removal of
+//                  v* from the candidate list, choice of the next block j* (least f among the
+//                  non-full blocks, lowest index on ties) and scheduling of the next sweep.
+#include "rcd_internal.h"
+
+#include <limits.h>
+
+namespace rcd {
+
+template <typename SV> struct Arith;
+template <> struct Arith<int32_t> {
+    using GV = long long;   // gains
+    using FV = long long;   // tracked f
+    static constexpr bool kInt = true;
+};
+template <> struct Arith<float> {
+    using GV = float;
+    using FV = double;
+    static constexpr bool kInt = false;
+};
+
+template <typename SV>
+struct GreedyParams {
+    using GV = typename Arith<SV>::GV;
+    using FV = typename Arith<SV>::FV;
+    const ClassDesc *desc;
+    const SV *S;
+    SV *cover;
+    GV *gains;
+    FV *fval;
+    int32_t *cnt;
+    const int32_t *quota;
+    uint8_t *valid;
+    int32_t *cand;
+    int32_t *pos;
+    int32_t *nR;
+    int32_t *jstar;
+    int32_t *sweepN;
+    int32_t *sweepParts;
+    int32_t *rowCtr;
+    int32_t *sweepList;
+    int32_t *nSweep;
+    unsigned long long *stepBytes;
+    unsigned long long *stepOps;
+    int32_t *status;
+    const int32_t *perm;
+    int32_t *assignment;
+    int32_t *order;         // may be null
+    int32_t L, W;
+    int32_t batchMax;       // 1, 2, 4 or 8
+    int32_t smemBytes;      // dynamic shared memory of the sweep kernel
+    int32_t segIters;       // int path: chunk iterations a 32-bit partial sum can take without overflow
+};
+
+__host__ __device__ inline int rows_per_group(int P) { return P == 8 ? 4 : 8; }
+
+// ---------------------------------------------------------------------------------------------
+// Choice of the next block and of the blocks the next sweep refreshes.  Run by warp 0 of the
+// class's CTA after a __syncthreads().
+template <typename SV>
+__device__ void plan_next(const GreedyParams<SV> &prm, int l, int nextStep)
+{
+    using FV = typename Arith<SV>::FV;
+    const int lane = threadIdx.x & 31;
+    if ((threadIdx.x >> 5) != 0) return;
+    const int W = prm.W;
+    const int nR = prm.nR[l];
+    const ClassDesc c = prm.desc[l];
+    FV *f = prm.fval + (int64_t)l * W;
+    int32_t *cnt = prm.cnt + (int64_t)l * W;
+    const int32_t *quota = prm.quota + (int64_t)l * W;
+    uint8_t *valid = prm.valid + (int64_t)l * W;
+
+    if (nR == 0) {
+        if (lane == 0) { prm.jstar[l] = -1; prm.sweepN[l] = 0; }
+        return;
+    }
+    // j* = argmin over non-full blocks of f, ties -> lowest index
+    FV bestF = 0;
+    int bestP = INT_MAX;
+    int nStale = 0;
+    for (int p = lane; p < W; p += 32) {
+        if (cnt[p] < quota[p]) {
+            FV fp = f[p];
+            if (bestP == INT_MAX || fp < bestF) { bestF = fp; bestP = p; }
+            if (!valid[p]) ++nStale;
+        }
+    }
+    for (int off = 16; off > 0; off >>= 1) {
+        FV oF = __shfl_xor_sync(0xffffffffu, bestF, off);
+        int oP = __shfl_xor_sync(0xffffffffu, bestP, off);
+        nStale += __shfl_xor_sync(0xffffffffu, nStale, off);
+        if (oP != INT_MAX && (bestP == INT_MAX || oF < bestF || (oF == bestF && oP < bestP))) { bestF = oF; bestP = oP; }
+    }
+    if (bestP == INT_MAX) {
+        if (lane == 0) { prm.jstar[l] = -1; prm.sweepN[l] = 0; atomicOr(prm.status, kDevNoCandidate); }
+        return;
+    }
+    const int jstar = bestP;
+    if (valid[jstar]) {
+        if (lane == 0) { prm.jstar[l] = jstar; prm.sweepN[l] = 0; }
+        return;
+    }
+    // how many blocks one pass can refresh: power of two, bounded by the configuration, by the
+    // shared memory that holds their coverage vectors and by the number of out-of-date blocks
+    int cap = prm.batchMax;
+    while (cap > 1 && (int64_t)cap * c.ld * (int64_t)sizeof(SV) > prm.smemBytes) cap >>= 1;
+    int P = 1;
+    while (P * 2 <= cap && P * 2 <= nStale) P *= 2;
+    int32_t *parts = prm.sweepParts + (int64_t)l * kMaxSweepBatch;
+    if (lane == 0) { parts[0] = jstar; valid[jstar] = 1; }
+    __syncwarp();
+    for (int k = 1; k < P; ++k) {
+        // next out-of-date non-full block of least f: the one most likely to be chosen soon
+        FV qF = 0;
+        int qP = INT_MAX;
+        for (int p = lane; p < W; p += 32) {
+            if (cnt[p] < quota[p] && !valid[p]) {
+                FV fp = f[p];
+                if (qP == INT_MAX || fp < qF) { qF = fp; qP = p; }
+            }
+        }
+        for (int off = 16; off > 0; off >>= 1) {
+            FV oF = __shfl_xor_sync(0xffffffffu, qF, off);
+            int oP = __shfl_xor_sync(0xffffffffu, qP, off);
+            if (oP != INT_MAX && (qP == INT_MAX || oF < qF || (oF == qF && oP < qP))) { qF = oF; qP = oP; }
+        }
+        if (lane == 0) { parts[k] = qP; valid[qP] = 1; }
+        __syncwarp();
+    }
+    if (lane == 0) {
+        prm.jstar[l] = jstar;
+        prm.sweepN[l] = P;
+        prm.rowCtr[l] = 0;
+        int par = nextStep & 1;
+        int slot = atomicAdd(&prm.nSweep[par], 1);
+        prm.sweepList[(int64_t)par * prm.L + slot] = l;
+        atomicAdd(&prm.stepBytes[nextStep], (unsigned long long)((int64_t)nR * c.ld + (int64_t)P * c.ld) * sizeof(SV));
+        atomicAdd(&prm.stepOps[nextStep], (unsigned long long)((int64_t)nR * c.M * P));
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+template <typename SV>
+__global__ void __launch_bounds__(kSelectThreads, 4) init_kernel(GreedyParams<SV> prm)
+{
+    using FV = typename Arith<SV>::FV;
+    const int l = blockIdx.x;
+    const ClassDesc c = prm.desc[l];
+    const int W = prm.W;
+    SV *cover = prm.cover + c.vOff;
+    for (int64_t i = threadIdx.x; i < (int64_t)W * c.ld; i += blockDim.x) cover[i] = 0;
+    for (int v = threadIdx.x; v < c.M; v += blockDim.x) {
+        prm.cand[c.row0 + v] = v;
+        prm.pos[c.row0 + v] = v;
+    }
+    for (int p = threadIdx.x; p < W; p += blockDim.x) {
+        prm.cnt[(int64_t)l * W + p] = 0;
+        prm.fval[(int64_t)l * W + p] = (FV)0;
+        prm.valid[(int64_t)l * W + p] = 0;
+    }
+    if (threadIdx.x == 0) prm.nR[l] = c.M;
+    __syncthreads();
+    plan_next(prm, l, 0);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Streaming 128-bit load that does not allocate in L1 (S is read once per pass; the L1 is left to
+// nothing in particular, the coverage vectors sit in shared memory).
+__device__ __forceinline__ int4 ld_stream(const int4 *p)
+{
+    int4 v;
+    asm("ld.global.nc.L1::no_allocate.v4.s32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+
+// Sum NA per-lane partials over the 32 lanes so that lane k ends with the total of partial
+// k / (32/NA): each step hands half of the values to the partner lane (xor offset) and adds the
+// partner's copy of the half that stays, then plain butterflies finish the remaining offsets.
+// The order of additions is fixed, so fp32 results are reproducible.
+template <typename T, int N>
+struct WarpMultiReduce {
+    static __device__ __forceinline__ T run(T (&v)[N], int off, int lane)
+    {
+        T w[N / 2];
+        const bool up = (lane & off) != 0;
+#pragma unroll
+        for (int i = 0; i < N / 2; ++i) {
+            T send = up ? v[i] : v[i + N / 2];
+            T keep = up ? v[i + N / 2] : v[i];
+            w[i] = keep + __shfl_xor_sync(0xffffffffu, send, off);
+        }
+        return WarpMultiReduce<T, N / 2>::run(w, off >> 1, lane);
+    }
+};
+template <typename T>
+struct WarpMultiReduce<T, 1> {
+    static __device__ __forceinline__ T run(T (&v)[1], int off, int lane)
+    {
+        T x = v[0];
+        for (; off > 0; off >>= 1) x += __shfl_xor_sync(0xffffffffu, x, off);
+        return x;
+    }
+};
+
+// One class, P blocks: warps pull groups of R rows until the class's rows are exhausted.
+template <typename SV, int P, int R>
+__device__ __forceinline__ void sweep_class(const GreedyParams<SV> &prm, int l, const ClassDesc &c, int nR,
+                                            const int4 *shCover, const long long *shF, const int32_t *parts)
+{
+    using GV = typename Arith<SV>::GV;
+    constexpr int NA = P * R;
+    const int lane = threadIdx.x & 31;
+    const int ld4 = c.ld >> 2;
+    const int nGroups = (nR + R - 1) / R;
+    const SV *Sl = prm.S + c.sOff;
+    const int32_t *cand = prm.cand + c.row0;
+    GV *G = prm.gains + c.vOff;
+
+    for (;;) {
+        int g = 0;
+        if (lane == 0) g = atomicAdd(&prm.rowCtr[l], 1);
+        g = __shfl_sync(0xffffffffu, g, 0);
+        if (g >= nGroups) break;
+        const int k0 = g * R;
+        int vrow[R];
+        const int4 *rp[R];
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            int k = k0 + r;
+            vrow[r] = cand[k < nR ? k : nR - 1];
+            rp[r] = reinterpret_cast<const int4 *>(Sl + (int64_t)vrow[r] * c.ld);
+        }
+        GV total = 0;
+        if constexpr (Arith<SV>::kInt) {
+            // sum_i max(S[v][i], cover[i]) in unsigned 32-bit partials (every term is in [0, 2^31)),
+            // widened to 64 bits every segIters iterations; the gain is that sum minus f_p.
+            unsigned long long tot = 0;
+            const int segLen = prm.segIters * 32;
+            for (int c0 = 0; c0 < ld4; c0 += segLen) {
+                uint32_t acc[NA];
+#pragma unroll
+                for (int i = 0; i < NA; ++i) acc[i] = 0u;
+                const int cEnd = min(ld4, c0 + segLen);
+#pragma unroll 2
+                for (int cc = c0 + lane; cc < cEnd; cc += 32) {
+                    int4 s[R];
+#pragma unroll
+                    for (int r = 0; r < R; ++r) s[r] = ld_stream(rp[r] + cc);
+#pragma unroll
+                    for (int p = 0; p < P; ++p) {
+                        const int4 m = shCover[p * ld4 + cc];
+#pragma unroll
+                        for (int r = 0; r < R; ++r)
+                            acc[r * P + p] += ((uint32_t)max(s[r].x, m.x) + (uint32_t)max(s[r].y, m.y)) +
+                                              ((uint32_t)max(s[r].z, m.z) + (uint32_t)max(s[r].w, m.w));
+                    }
+                }
+                unsigned long long wide[NA / 2];
+                {
+                    const bool up = (lane & 16) != 0;
+#pragma unroll
+                    for (int i = 0; i < NA / 2; ++i) {
+                        uint32_t send = up ? acc[i] : acc[i + NA / 2];
+                        uint32_t keep = up ? acc[i + NA / 2] : acc[i];
+                        wide[i] = (unsigned long long)keep + (unsigned long long)__shfl_xor_sync(0xffffffffu, send, 16);
+                    }
+                }
+                tot += WarpMultiReduce<unsigned long long, NA / 2>::run(wide, 8, lane);
+            }
+            total = (GV)tot;
+        } else {
+            float acc[NA];
+#pragma unroll
+            for (int i = 0; i < NA; ++i) acc[i] = 0.f;
+#pragma unroll 2
+            for (int cc = lane; cc < ld4; cc += 32) {
+                int4 s[R];
+#pragma unroll
+                for (int r = 0; r < R; ++r) s[r] = ld_stream(rp[r] + cc);
+#pragma unroll
+                for (int p = 0; p < P; ++p) {
+                    const int4 mi = shCover[p * ld4 + cc];
+                    const float m0 = __int_as_float(mi.x), m1 = __int_as_float(mi.y);
+                    const float m2 = __int_as_float(mi.z), m3 = __int_as_float(mi.w);
+#pragma unroll
+                    for (int r = 0; r < R; ++r) {
+                        float a = acc[r * P + p];
+                        a += fmaxf(__int_as_float(s[r].x) - m0, 0.f);
+                        a += fmaxf(__int_as_float(s[r].y) - m1, 0.f);
+                        a += fmaxf(__int_as_float(s[r].z) - m2, 0.f);
+                        a += fmaxf(__int_as_float(s[r].w) - m3, 0.f);
+                        acc[r * P + p] = a;
+                    }
+                }
+            }
+            total = WarpMultiReduce<float, NA>::run(acc, 16, lane);
+        }
+        // lane k holds partial k / (32/NA) = r * P + p
+        constexpr int kShare = 32 / NA;
+        if ((lane % kShare) == 0) {
+            const int idx = lane / kShare;
+            const int r = idx / P, p = idx % P;
+            if (k0 + r < nR) {
+                GV gain;
+                if constexpr (Arith<SV>::kInt) gain = total - shF[p];
+                else gain = total;
+                int row = 0;
+#pragma unroll
+                for (int q = 0; q < R; ++q) if (q == r) row = vrow[q];
+                G[(int64_t)parts[p] * c.ld + row] = gain;
+            }
+        }
+    }
+}
+
+template <typename SV>
+__global__ void __launch_bounds__(kSweepThreads, 1) sweep_kernel(GreedyParams<SV> prm, int step)
+{
+    extern __shared__ int4 shCover[];
+    __shared__ long long shF[kMaxSweepBatch];
+    __shared__ int32_t shParts[kMaxSweepBatch];
+    __shared__ int shGo;
+    const int par = step & 1;
+    const int nS = prm.nSweep[par];
+    if (blockIdx.x == 0 && threadIdx.x == 0) prm.nSweep[par ^ 1] = 0;   // list the coming select fills
+    if (nS == 0) return;
+    const int start = (int)(((int64_t)blockIdx.x * nS) / gridDim.x);
+    for (int k = 0; k < nS; ++k) {
+        int s = start + k;
+        if (s >= nS) s -= nS;
+        const int l = prm.sweepList[(int64_t)par * prm.L + s];
+        const ClassDesc c = prm.desc[l];
+        const int nR = prm.nR[l];
+        const int P = prm.sweepN[l];
+        const int R = rows_per_group(P);
+        const int nGroups = (nR + R - 1) / R;
+        if (threadIdx.x == 0) shGo = (*(volatile int32_t *)&prm.rowCtr[l] < nGroups) ? 1 : 0;
+        __syncthreads();
+        const int go = shGo;
+        if (go) {
+            const int ld4 = c.ld >> 2;
+            const int32_t *parts = prm.sweepParts + (int64_t)l * kMaxSweepBatch;
+            const int4 *cov = reinterpret_cast<const int4 *>(prm.cover + c.vOff);
+            for (int i = threadIdx.x; i < P * ld4; i += blockDim.x) {
+                int p = i / ld4, cc = i - p * ld4;
+                shCover[i] = cov[(int64_t)parts[p] * ld4 + cc];
+            }
+            if (threadIdx.x < P) {
+                shParts[threadIdx.x] = parts[threadIdx.x];
+                if constexpr (Arith<SV>::kInt) shF[threadIdx.x] = prm.fval[(int64_t)l * prm.W + parts[threadIdx.x]];
+            }
+            __syncthreads();
+            switch (P) {
+            case 1: sweep_class<SV, 1, 8>(prm, l, c, nR, shCover, shF, shParts); break;
+            case 2: sweep_class<SV, 2, 8>(prm, l, c, nR, shCover, shF, shParts); break;
+            case 4: sweep_class<SV, 4, 8>(prm, l, c, nR, shCover, shF, shParts); break;
+            default: sweep_class<SV, 8, 4>(prm, l, c, nR, shCover, shF, shParts); break;
+            }
+        }
+        __syncthreads();
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+template <typename SV>
+__global__ void __launch_bounds__(kSelectThreads, 4) select_kernel(GreedyParams<SV> prm, int step)
+{
+    using GV = typename Arith<SV>::GV;
+    using FV = typename Arith<SV>::FV;
+    __shared__ GV shG[kSelectThreads / 32];
+    __shared__ int shV[kSelectThreads / 32];
+    __shared__ int shPick;
+    const int l = blockIdx.x;
+    const int nR = prm.nR[l];
+    if (nR == 0) return;
+    const int j = prm.jstar[l];
+    if (j < 0) return;
+    const ClassDesc c = prm.desc[l];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int32_t *cand = prm.cand + c.row0;
+    int32_t *pos = prm.pos + c.row0;
+    const GV *G = prm.gains + c.vOff + (int64_t)j * c.ld;
+
+    // v* = argmax over the unassigned samples, ties -> lowest class-local index (GreedyStep)
+    GV bestG = 0;
+    int bestV = INT_MAX;
+    for (int k = threadIdx.x; k < nR; k += blockDim.x) {
+        int v = cand[k];
+        GV g = G[v];
+        if (bestV == INT_MAX || g > bestG || (g == bestG && v < bestV)) { bestG = g; bestV = v; }
+    }
+    for (int off = 16; off > 0; off >>= 1) {
+        GV oG = __shfl_xor_sync(0xffffffffu, bestG, off);
+        int oV = __shfl_xor_sync(0xffffffffu, bestV, off);
+        if (oV != INT_MAX && (bestV == INT_MAX || oG > bestG || (oG == bestG && oV < bestV))) { bestG = oG; bestV = oV; }
+    }
+    if (lane == 0) { shG[warp] = bestG; shV[warp] = bestV; }
+    __syncthreads();
+    if (warp == 0) {
+        bestG = lane < kSelectThreads / 32 ? shG[lane] : (GV)0;
+        bestV = lane < kSelectThreads / 32 ? shV[lane] : INT_MAX;
+        for (int off = 16; off > 0; off >>= 1) {
+            GV oG = __shfl_xor_sync(0xffffffffu, bestG, off);
+            int oV = __shfl_xor_sync(0xffffffffu, bestV, off);
+            if (oV != INT_MAX && (bestV == INT_MAX || oG > bestG || (oG == bestG && oV < bestV))) { bestG = oG; bestV = oV; }
+        }
+        if (lane == 0) {
+            shPick = bestV;
+            shG[0] = bestG;
+        }
+    }
+    __syncthreads();
+    const int vstar = shPick;
+    const GV gstar = shG[0];
+    if (vstar == INT_MAX || vstar < 0 || vstar >= c.M) {
+        if (threadIdx.x == 0) atomicOr(prm.status, kDevBadState);
+        return;
+    }
+    // cover_j <- max(cover_j, S[v*][.])
+    {
+        const int ld4 = c.ld >> 2;
+        int4 *cov = reinterpret_cast<int4 *>(prm.cover + c.vOff + (int64_t)j * c.ld);
+        const int4 *row = reinterpret_cast<const int4 *>(prm.S + c.sOff + (int64_t)vstar * c.ld);
+        for (int i = threadIdx.x; i < ld4; i += blockDim.x) {
+            int4 a = cov[i], b = row[i];
+            if constexpr (Arith<SV>::kInt) {
+                a.x = max(a.x, b.x); a.y = max(a.y, b.y); a.z = max(a.z, b.z); a.w = max(a.w, b.w);
+            } else {
+                a.x = __float_as_int(fmaxf(__int_as_float(a.x), __int_as_float(b.x)));
+                a.y = __float_as_int(fmaxf(__int_as_float(a.y), __int_as_float(b.y)));
+                a.z = __float_as_int(fmaxf(__int_as_float(a.z), __int_as_float(b.z)));
+                a.w = __float_as_int(fmaxf(__int_as_float(a.w), __int_as_float(b.w)));
+            }
+            cov[i] = a;
+        }
+    }
+    if (threadIdx.x == 0) {
+        const int64_t at = (int64_t)l * prm.W + j;
+        prm.fval[at] += (FV)gstar;
+        prm.cnt[at] += 1;
+        prm.valid[at] = 0;
+        const int global = prm.perm[c.row0 + vstar];
+        prm.assignment[global] = j;
+        if (prm.order) prm.order[c.row0 + (c.M - nR)] = global;
+        const int k = pos[vstar];
+        const int lastV = cand[nR - 1];
+        cand[k] = lastV;
+        pos[lastV] = k;
+        prm.nR[l] = nR - 1;
+    }
+    __syncthreads();
+    plan_next(prm, l, step + 1);
+}
+
+// ---------------------------------------------------------------------------------------------
+template <typename SV>
+static rcd_status run_greedy(rcd_ctx *ctx, const Sizes &sz, const Workspace &ws,
+                             const std::vector<ClassDesc> &descHost, int32_t *assignment, int32_t *order,
+                             cudaStream_t st)
+{
+    using GV = typename Arith<SV>::GV;
+    using FV = typename Arith<SV>::FV;
+    GreedyParams<SV> prm;
+    prm.desc = ws.desc;
+    prm.S = (const SV *)ws.S;
+    prm.cover = (SV *)ws.cover;
+    prm.gains = (GV *)ws.gains;
+    prm.fval = (FV *)ws.fval;
+    prm.cnt = ws.cnt;
+    prm.quota = ws.quota;
+    prm.valid = ws.valid;
+    prm.cand = ws.cand;
+    prm.pos = ws.pos;
+    prm.nR = ws.nR;
+    prm.jstar = ws.jstar;
+    prm.sweepN = ws.sweepN;
+    prm.sweepParts = ws.sweepParts;
+    prm.rowCtr = ws.rowCtr;
+    prm.sweepList = ws.sweepList;
+    prm.nSweep = ws.nSweep;
+    prm.stepBytes = ws.stepBytes;
+    prm.stepOps = ws.stepOps;
+    prm.status = ws.status;
+    prm.perm = ws.perm;
+    prm.assignment = assignment;
+    prm.order = order;
+    prm.L = sz.L;
+    prm.W = sz.W;
+    int batch = ctx->cfg.sweep_batch_max;
+    if (batch <= 0) batch = kMaxSweepBatch;
+    prm.batchMax = batch;
+
+    int maxLd = 0;
+    for (const auto &c : descHost) if (c.ld > maxLd) maxLd = c.ld;
+    const int64_t smemCap = (int64_t)ctx->maxSmemOptin - 2048;     // static shared + margin
+    int64_t smem = (int64_t)batch * maxLd * (int64_t)sizeof(SV);
+    if (smem > smemCap) smem = smemCap;
+    if ((int64_t)maxLd * (int64_t)sizeof(SV) > smem)
+        return fail(ctx, RCD_ERR_UNSUPPORTED,
+                    "class of %d samples: one coverage vector (%lld bytes) exceeds the %lld bytes of shared memory",
+                    maxLd, (long long)maxLd * (long long)sizeof(SV), (long long)smem);
+    if (smem < 16) smem = 16;
+    prm.smemBytes = (int32_t)smem;
+    // 32-bit partial sums take terms below 16384*d each, four per chunk iteration
+    {
+        int64_t bound = 16384LL * sz.d;
+        int64_t it = 0xffffffffLL / (4 * bound);
+        if (it < 1) return fail(ctx, RCD_ERR_UNSUPPORTED, "feature width %lld too large for 32-bit partial sums", (long long)sz.d);
+        if (it > 1 << 20) it = 1 << 20;
+        prm.segIters = (int32_t)it;
+    }
+    RCD_CUDA(ctx, cudaFuncSetAttribute(sweep_kernel<SV>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+
+    RCD_CUDA(ctx, cudaMemsetAsync(ws.nSweep, 0, 2 * sizeof(int32_t), st));
+    RCD_CUDA(ctx, cudaMemsetAsync(ws.stepBytes, 0, (size_t)(sz.maxM + 1) * sizeof(unsigned long long), st));
+    RCD_CUDA(ctx, cudaMemsetAsync(ws.stepOps, 0, (size_t)(sz.maxM + 1) * sizeof(unsigned long long), st));
+    init_kernel<SV><<<sz.L, kSelectThreads, 0, st>>>(prm);
+    ctx->kernelLaunches++;
+    RCD_CUDA(ctx, cudaGetLastError());
+
+    const bool perSweep = ctx->cfg.profile >= 2;
+    if (perSweep) {
+        while ((int64_t)ctx->evSweep.size() < 2 * sz.maxM) {
+            cudaEvent_t e;
+            RCD_CUDA(ctx, cudaEventCreate(&e));
+            ctx->evSweep.push_back(e);
+        }
+    }
+    ctx->sweepEventsUsed = 0;
+    for (int64_t t = 0; t < sz.maxM; ++t) {
+        if (perSweep) RCD_CUDA(ctx, cudaEventRecord(ctx->evSweep[2 * t], st));
+        sweep_kernel<SV><<<ctx->smCount, kSweepThreads, (size_t)smem, st>>>(prm, (int)t);
+        if (perSweep) RCD_CUDA(ctx, cudaEventRecord(ctx->evSweep[2 * t + 1], st));
+        select_kernel<SV><<<sz.L, kSelectThreads, 0, st>>>(prm, (int)t);
+        ctx->kernelLaunches += 2;
+    }
+    if (perSweep) ctx->sweepEventsUsed = 2 * sz.maxM;
+    RCD_CUDA(ctx, cudaGetLastError());
+    ctx->steps = sz.maxM;
+    ctx->stepBytesDev = ws.stepBytes;
+    ctx->stepOpsDev = ws.stepOps;
+    return RCD_OK;
+}
+
+rcd_status launch_greedy(rcd_ctx *ctx, rcd_feat_dtype dtype, const Sizes &sz, const Workspace &ws,
+                         const std::vector<ClassDesc> &descHost, int32_t *assignment, int32_t *order,
+                         cudaStream_t st)
+{
+    if (sz.L == 0 || sz.maxM == 0) return RCD_OK;
+    if (dtype == RCD_FEAT_I8) return run_greedy<int32_t>(ctx, sz, ws, descHost, assignment, order, st);
+    return run_greedy<float>(ctx, sz, ws, descHost, assignment, order, st);
+}
+
+}  // namespace rcd

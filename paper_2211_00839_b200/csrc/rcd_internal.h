@@ -1,0 +1,167 @@
+// Internal declarations shared by the library's translation units (not part of the ABI).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stddef.h>
+#include <string>
+#include <vector>
+
+#include "rcd.h"
+
+namespace rcd {
+
+constexpr int kMaxSweepBatch = 8;          // blocks refreshed by one pass over S
+constexpr int kSweepThreads = 512;         // sweep CTA: 16 warps, one CTA per SM
+constexpr int kSelectThreads = 256;        // pick/update CTA: one per class
+constexpr size_t kAlign = 256;
+
+// Device-side status bits (OR-ed into the status word).
+enum : int {
+    kDevOk = 0,
+    kDevBadLabel = 1,          // a label outside [0, L)
+    kDevNoCandidate = 2,       // a class had samples left but no block could take one
+    kDevBadState = 4,          // internal consistency check failed
+};
+
+// One class, as the kernels see it.  Built on the host once the class sizes are known.
+struct ClassDesc {
+    int32_t M;        // samples in the class
+    int32_t ld;       // row pitch of S and of the per-block vectors, in elements (M rounded up to 4)
+    int32_t row0;     // first row of the class in class-sorted sample order
+    int32_t pad_;
+    int64_t sOff;     // element offset of S_l
+    int64_t vOff;     // element offset of the class's [W][ld] arrays (coverage, gains)
+};
+
+// Where a kernel finds the descriptor of class l: a table in device memory, or (table == null)
+// `L` classes of equal size laid out back to back.
+struct DescSource {
+    const ClassDesc *table;
+    int32_t uniM, uniLd;
+    __host__ __device__ ClassDesc get(int l) const
+    {
+        if (table) return table[l];
+        ClassDesc c;
+        c.M = uniM; c.ld = uniLd; c.row0 = l * uniM; c.pad_ = 0;
+        c.sOff = (int64_t)l * uniM * uniLd; c.vOff = 0;
+        return c;
+    }
+};
+
+// The classes a similarity launch covers.
+struct SimClasses {
+    DescSource src;
+    int32_t L;
+    int64_t maxM;
+    int64_t tiles128;       // sum over classes of ceil(M/128)^2 (tensor-core tile count)
+};
+
+// Pointers into the caller's workspace for one rcd_partition call.
+struct Workspace {
+    // grouping
+    int32_t *counts;        // [L]
+    int32_t *chunkHist;     // [nChunks][L]
+    int32_t *perm;          // [N] class-sorted position -> dataset index
+    void *Xs;               // [N][d] features in class-sorted order
+    // per class
+    ClassDesc *desc;        // [L]
+    void *S;                // similarity matrices
+    void *cover;            // [sum W*ld] coverage vectors (int32 / float)
+    void *gains;            // [sum W*ld] stored gains (int64 / float)
+    void *fval;             // [L][W] tracked f (int64 / double)
+    int32_t *cnt;           // [L][W]
+    int32_t *quota;         // [L][W]
+    uint8_t *valid;         // [L][W] 1 = stored gains of that block are current
+    int32_t *cand;          // [N] unassigned samples of each class (class-local ids), compact
+    int32_t *pos;           // [N] position of each sample in cand
+    int32_t *nR;            // [L] unassigned count
+    int32_t *jstar;         // [L] block chosen for the next pick (-1: none)
+    int32_t *sweepN;        // [L] blocks to refresh in the next sweep (0: none)
+    int32_t *sweepParts;    // [L][kMaxSweepBatch]
+    int32_t *rowCtr;        // [L] ticket counter over row groups of the running sweep
+    int32_t *sweepList;     // [2][L] classes that sweep in the next step (double-buffered by step parity)
+    int32_t *nSweep;        // [2]
+    unsigned long long *stepBytes;   // [steps+1] bytes the sweep of step t has to read
+    unsigned long long *stepOps;     // [steps+1] element x block pairs of that sweep
+    int32_t *status;        // [1]
+    size_t bytes;           // total bytes laid out
+};
+
+struct Sizes {
+    int64_t N, d;
+    int32_t L, W;
+    int64_t sElems;         // sum M_l * ld_l
+    int64_t vElems;         // sum W * ld_l
+    int64_t maxM;
+    int32_t nChunks;
+};
+
+constexpr int kGroupChunk = 1024;           // samples per chunk of the stable class split
+
+inline size_t feat_bytes(rcd_feat_dtype t) { return t == RCD_FEAT_I8 ? 1 : 2; }
+inline size_t align_up(size_t x, size_t a = kAlign) { return (x + a - 1) / a * a; }
+inline int32_t pad4(int64_t m) { return (int32_t)((m + 3) / 4 * 4); }
+
+// Lays the workspace out at `base` (may be null to measure).  Returns total bytes.
+size_t layout_workspace(void *base, rcd_feat_dtype dtype, const Sizes &sz, Workspace *ws);
+
+}  // namespace rcd
+
+struct rcd_ctx {
+    int device = 0;
+    int smCount = 0;
+    int maxSmemOptin = 0;
+    rcd_config cfg{};
+    std::string err;
+    int32_t *hostStage = nullptr;       // pinned, counts / status read-back
+    size_t hostStageInts = 0;
+    // profiling
+    cudaEvent_t evPhase[5]{};           // start, after group, after similarity, after greedy, end
+    bool phaseValid = false;
+    std::vector<cudaEvent_t> evSweep;   // 2 per step
+    int64_t sweepEventsUsed = 0;
+    int64_t kernelLaunches = 0;
+    int64_t steps = 0;
+    const unsigned long long *stepBytesDev = nullptr;
+    const unsigned long long *stepOpsDev = nullptr;
+    const int32_t *statusDev = nullptr;
+};
+
+namespace rcd {
+
+rcd_status fail(rcd_ctx *ctx, rcd_status st, const char *fmt, ...);
+rcd_status cuda_fail(rcd_ctx *ctx, cudaError_t e, const char *what);
+
+#define RCD_CUDA(ctx, call)                                            \
+    do {                                                               \
+        cudaError_t e__ = (call);                                      \
+        if (e__ != cudaSuccess) return ::rcd::cuda_fail(ctx, e__, #call); \
+    } while (0)
+
+// ---- launchers implemented in the .cu files (all asynchronous on `st`) ----
+
+// class split
+rcd_status launch_count_labels(rcd_ctx *ctx, const int32_t *labels, int64_t N, int32_t L, int32_t *counts,
+                               int32_t *status, cudaStream_t st);
+rcd_status launch_stable_split(rcd_ctx *ctx, const int32_t *labels, int64_t N, int32_t L, int32_t nChunks,
+                               int32_t *chunkHist, const ClassDesc *descDev, int32_t *perm, cudaStream_t st);
+rcd_status launch_gather_rows(rcd_ctx *ctx, const void *X, const int32_t *perm, int64_t N, int64_t rowBytes,
+                              void *Xs, cudaStream_t st);
+
+// similarity: S_l = Xs_l Xs_l^T for every class described by desc
+rcd_status launch_similarity(rcd_ctx *ctx, const void *Xs, rcd_feat_dtype dtype, int64_t Ntot, int64_t d,
+                             const SimClasses &cls, void *S, cudaStream_t st);
+
+// greedy loop
+rcd_status launch_greedy(rcd_ctx *ctx, rcd_feat_dtype dtype, const Sizes &sz, const Workspace &ws,
+                         const std::vector<ClassDesc> &descHost, int32_t *assignment, int32_t *order,
+                         cudaStream_t st);
+
+// objective from an assignment
+rcd_status launch_objective(rcd_ctx *ctx, rcd_feat_dtype dtype, const Sizes &sz, const ClassDesc *descDev,
+                            const std::vector<ClassDesc> &descHost, const void *S, const int32_t *perm,
+                            const int32_t *assignment, void *partValues, void *total, void *scratch,
+                            cudaStream_t st);
+
+}  // namespace rcd

@@ -1,0 +1,293 @@
+"""Parity of the CUDA library (through its C ABI) against the CPU oracle, on the same seeded inputs.
+
+int8 features: bit-exact (assignment, pick order, int64 objective).
+bf16 features: objective within 1e-4 relative; picks equal to the oracle's wherever the
+oracle's top-two candidates differ by more than 1e-3 relative (teacher-forced replay).
+"""
+import numpy as np
+import pytest
+
+pytestmark = pytest.mark.gpu
+
+OBJ_RTOL = 1e-4      # final objective, float configs
+PICK_RTOL = 1e-3     # a pick may differ from the oracle's only inside this relative gap
+
+
+@pytest.fixture(scope="module")
+def rcd():
+    import torch
+    assert torch.cuda.is_available()
+    from paper_2211_00839_b200 import binding
+    return binding
+
+
+@pytest.fixture(scope="module")
+def orc():
+    from oracle import rcd_oracle
+    return rcd_oracle
+
+
+def to_device(rcd, wl):
+    import torch
+    dev = torch.device("cuda", 0)
+    X = rcd.features_to_torch(wl.features, device=dev)
+    y = torch.from_numpy(wl.labels).to(dev)
+    return X, y
+
+
+def run_partition(rcd, wl, **cfg):
+    import torch
+    with rcd.Context(0, **cfg) as ctx:
+        X, y = to_device(rcd, wl)
+        a, o, v = ctx.rcd_partition(X, y, wl.capacities, wl.L)
+        ctx.sync_status()
+        return a.cpu().numpy(), o.cpu().numpy(), v.cpu().numpy()
+
+
+# ----------------------------------------------------------------------------- similarity
+
+@pytest.mark.parametrize("M,d,batch", [(200, 64, 2), (257, 100, 1), (130, 37, 3), (1, 5, 1), (515, 512, 1)])
+@pytest.mark.parametrize("path", [0, 2])
+def test_similarity_int8_exact(rcd, orc, M, d, batch, path):
+    import torch
+    rng = np.random.default_rng(M * 1000 + d)
+    X = rng.integers(-128, 128, size=(batch, M, d)).astype(np.int8)
+    with rcd.Context(0, similarity_path=path) as ctx:
+        S = ctx.rcd_similarity(torch.from_numpy(X).cuda())
+        torch.cuda.synchronize()
+        S = S.cpu().numpy()
+    ld = (M + 3) // 4 * 4
+    assert S.shape == (batch, M, ld)
+    for b in range(batch):
+        want = orc.similarity(X[b])
+        assert np.array_equal(S[b, :, :M].astype(np.int64), want)
+        assert np.all(S[b, :, M:] == 0)
+
+
+@pytest.mark.parametrize("M,d,batch", [(200, 64, 2), (257, 104, 1), (131, 37, 2), (515, 2048, 1)])
+@pytest.mark.parametrize("path", [0, 2])
+def test_similarity_bf16_close(rcd, orc, M, d, batch, path):
+    import torch
+    from paper_2211_00839_b200.workloads import fp32_to_bf16_bits
+    rng = np.random.default_rng(M * 7 + d)
+    x = np.abs(rng.standard_normal((batch, M, d))).astype(np.float32)
+    x /= np.linalg.norm(x, axis=2, keepdims=True)
+    bits = fp32_to_bf16_bits(x)
+    with rcd.Context(0, similarity_path=path) as ctx:
+        S = ctx.rcd_similarity(rcd.features_to_torch(bits.reshape(batch * M, d)).view(batch, M, d).cuda())
+        torch.cuda.synchronize()
+        S = S.cpu().numpy()
+    for b in range(batch):
+        want = orc.similarity(bits[b])
+        # fp32 accumulation of d products of magnitude <= 1/d-ish: absolute error far below 1e-5
+        assert np.allclose(S[b, :, :M], want, rtol=2e-5, atol=2e-6)
+        assert np.all(S[b, :, M:] == 0)
+
+
+# ----------------------------------------------------------------------------- partition, int8: bit-exact
+
+def check_exact(rcd, orc, wl, variant="incremental", **cfg):
+    a, o, v = run_partition(rcd, wl, **cfg)
+    ref = orc.partition(wl.features, wl.labels, wl.capacities, wl.L, variant=variant)
+    assert np.array_equal(a, ref.assignment)
+    assert np.array_equal(o, ref.order)
+    assert np.array_equal(v, ref.part_values)
+    return a, o, v, ref
+
+
+@pytest.mark.parametrize("batch", [1, 2, 4, 8])
+def test_partition_c1_exact(rcd, orc, batch):
+    from paper_2211_00839_b200.workloads import make_workload
+    wl = make_workload("C1")
+    a, o, v, ref = check_exact(rcd, orc, wl, variant="plain", sweep_batch_max=batch)
+    for l in range(wl.L):
+        ids = np.nonzero(wl.labels == l)[0]
+        assert np.bincount(a[ids], minlength=wl.W).tolist() == [25, 25, 50, 100]
+
+
+@pytest.mark.parametrize("seed", [0, 1])
+def test_partition_int8_ragged_classes(rcd, orc, seed):
+    """Unequal class sizes (several tiles and a ragged tail), an empty class, a class smaller than W,
+    a feature width that is not a multiple of 4."""
+    from paper_2211_00839_b200.workloads import Workload, make_mixture
+    rng = np.random.default_rng(40 + seed)
+    sizes = [333, 0, 5, 1030, 1, 257]
+    d = 75
+    feats, labels = [], []
+    for l, M in enumerate(sizes):
+        x = make_mixture(rng, M, d, 4, "dirichlet", "gauss", 4.0) if M else np.zeros((0, d), np.float32)
+        feats.append(np.clip(np.rint(x), -127, 127).astype(np.int8))
+        labels.append(np.full(M, l, np.int32))
+    feats = np.concatenate(feats)
+    labels = np.concatenate(labels)
+    perm = rng.permutation(len(labels))
+    caps = np.array([1, 2.5, 1, 4, 0.5, 3, 1, 1, 2], dtype=np.float64)
+    wl = Workload("ragged", "int8", np.ascontiguousarray(feats[perm]), np.ascontiguousarray(labels[perm]), caps,
+                  len(sizes), len(caps))
+    for batch in (8, 1):
+        check_exact(rcd, orc, wl, sweep_batch_max=batch)
+
+
+def test_partition_int8_ties_and_duplicates(rcd, orc):
+    """Duplicate rows and one-hot rows: every argmax / argmin tie must fall to the lowest index."""
+    from paper_2211_00839_b200.workloads import Workload
+    rng = np.random.default_rng(3)
+    base = rng.integers(-5, 6, size=(12, 16)).astype(np.int8)
+    feats = np.concatenate([base[rng.integers(0, 12, size=90)], 9 * np.eye(30, 16, dtype=np.int8)])
+    labels = np.concatenate([np.zeros(90, np.int32), np.ones(30, np.int32)])
+    wl = Workload("ties", "int8", feats, labels, np.array([1.0, 1.0, 2.0]), 2, 3)
+    check_exact(rcd, orc, wl, variant="plain")
+
+
+def test_partition_c2_reduced_exact(rcd, orc):
+    from paper_2211_00839_b200.workloads import make_workload
+    wl = make_workload("C2", L=3, M=1200)
+    check_exact(rcd, orc, wl)
+
+
+def test_partition_c5_reduced_exact(rcd, orc):
+    from paper_2211_00839_b200.workloads import make_workload
+    wl = make_workload("C5", L=6, M=700, d=256)
+    check_exact(rcd, orc, wl)
+
+
+def test_partition_is_reproducible(rcd):
+    from paper_2211_00839_b200.workloads import make_workload
+    wl = make_workload("C3", L=2, M=600, d=128)
+    r1 = run_partition(rcd, wl)
+    r2 = run_partition(rcd, wl)
+    for x, y in zip(r1, r2):
+        assert np.array_equal(x, y)
+
+
+# ----------------------------------------------------------------------------- partition, bf16: tolerance rule
+
+def check_float(rcd, orc, wl, **cfg):
+    a, o, v = run_partition(rcd, wl, **cfg)
+    free = orc.partition(wl.features, wl.labels, wl.capacities, wl.L, variant="incremental")
+    groups = orc.split_by_label(wl.labels, wl.L)
+    total_replayed = 0.0
+    for l, ids in enumerate(groups):
+        M = len(ids)
+        if M == 0:
+            continue
+        q = orc.quotas(M, wl.capacities)
+        assert np.bincount(a[ids], minlength=wl.W).tolist() == q.tolist()
+        off = int(free.class_offsets[l])
+        picked = o[off:off + M]
+        assert sorted(picked.tolist()) == sorted(ids.tolist())
+        local = np.searchsorted(ids, picked).astype(np.int32)
+        S = orc.similarity(wl.features[ids])
+        bad, stats, fv = orc.replay_class(S, q, a[picked], local, PICK_RTOL)
+        assert bad == -1, "class %d: pick %d outside the %g gap (stats %s)" % (l, bad, PICK_RTOL, stats)
+        # tracked (fp32 gains summed in fp64) vs the oracle's value of the same picks
+        assert np.allclose(v[l], fv, rtol=OBJ_RTOL, atol=1e-9)
+        total_replayed += fv.sum()
+        # free-running oracle: identical picks up to the first step whose top-two gap is inside the tolerance
+        ref_picked = free.order[off:off + M]
+        same = (picked == ref_picked) & (a[picked] == free.order_block[off:off + M])
+        if not same.all():
+            first = int(np.argmin(same))
+            bad0, stats0, _ = orc.replay_class(S, q, a[picked][:first + 1], local[:first + 1], 0.0)
+            assert bad0 == first and max(stats0[2], stats0[3]) <= PICK_RTOL
+    assert abs(v.sum() - total_replayed) <= OBJ_RTOL * abs(total_replayed)
+    assert abs(v.sum() - free.total) <= 5e-3 * abs(free.total)     # different near-tie branches stay close
+    return a, o, v
+
+
+def test_partition_c3_reduced_float(rcd, orc):
+    from paper_2211_00839_b200.workloads import make_workload
+    wl = make_workload("C3", L=2, M=900, d=512)
+    check_float(rcd, orc, wl)
+
+
+@pytest.mark.parametrize("batch", [1, 8])
+def test_partition_c4_reduced_float(rcd, orc, batch):
+    from paper_2211_00839_b200.workloads import make_workload
+    wl = make_workload("C4", L=5, M=500, d=256)
+    check_float(rcd, orc, wl, sweep_batch_max=batch)
+
+
+# ----------------------------------------------------------------------------- objective
+
+@pytest.mark.parametrize("name,L,M,d", [("C1", 2, 200, 64), ("C5", 3, 300, 128), ("C4", 3, 250, 96)])
+def test_objective_matches_plain_definition(rcd, orc, name, L, M, d):
+    import torch
+    from paper_2211_00839_b200.workloads import make_workload
+    wl = make_workload(name, L=L, M=M, d=d)
+    rng = np.random.default_rng(5)
+    assignment = rng.integers(-1, wl.W, size=wl.N).astype(np.int32)     # arbitrary, -1 = in no block
+    with rcd.Context(0) as ctx:
+        X, y = to_device(rcd, wl)
+        vals, total = ctx.rcd_objective(X, y, torch.from_numpy(assignment).cuda(), wl.W, wl.L)
+        ctx.sync_status()
+        vals, total = vals.cpu().numpy(), total.cpu().numpy()
+    want = orc.objective(wl.features, wl.labels, assignment, wl.W, wl.L)
+    if wl.dtype == "int8":
+        assert np.array_equal(vals, want) and total[0] == want.sum()
+    else:
+        assert np.allclose(vals, want, rtol=1e-5, atol=1e-7)
+        assert total[0] == pytest.approx(want.sum(), rel=1e-5)
+
+
+def test_tracked_values_equal_recomputed_objective(rcd):
+    import torch
+    from paper_2211_00839_b200.workloads import make_workload
+    wl = make_workload("C2", L=2, M=800)
+    with rcd.Context(0) as ctx:
+        X, y = to_device(rcd, wl)
+        a, o, v = ctx.rcd_partition(X, y, wl.capacities, wl.L)
+        vals, total = ctx.rcd_objective(X, y, a, wl.W, wl.L)
+        ctx.sync_status()
+        assert torch.equal(v, vals) and int(total[0]) == int(v.sum())
+
+
+# ----------------------------------------------------------------------------- host-buffer entry point, errors
+
+def test_partition_host_matches_device_entry(rcd, orc):
+    import torch
+    from paper_2211_00839_b200.workloads import make_workload
+    wl = make_workload("C1")
+    ref = orc.partition(wl.features, wl.labels, wl.capacities, wl.L, variant="plain")
+    with rcd.Context(0) as ctx:
+        X = rcd.features_to_torch(wl.features, pin=True)
+        y = torch.from_numpy(wl.labels).pin_memory()
+        a, o, v = ctx.rcd_partition_host(X, y, wl.capacities, wl.L)
+        assert np.array_equal(a.numpy(), ref.assignment)
+        assert np.array_equal(o.numpy(), ref.order)
+        assert np.array_equal(v.numpy(), ref.part_values)
+
+
+def test_argument_errors_are_reported(rcd):
+    import torch
+    from paper_2211_00839_b200.workloads import make_workload
+    wl = make_workload("C1")
+    with rcd.Context(0) as ctx:
+        X, y = to_device(rcd, wl)
+        with pytest.raises(rcd.RcdError) as e:
+            ctx.rcd_partition(X, y, [1.0, -1.0], wl.L)
+        assert e.value.status == 1
+        with pytest.raises(rcd.RcdError) as e:
+            ctx.rcd_partition(X, y, [1.0, float("nan")], wl.L)
+        assert e.value.status == 1
+        with pytest.raises(rcd.RcdError) as e:       # a label outside [0, L)
+            ctx.rcd_partition(X, y, wl.capacities, 1)
+        assert e.value.status == 1
+        with pytest.raises(rcd.RcdError) as e:       # class larger than promised -> workspace too small
+            ctx._ws = None
+            ctx.rcd_partition(X, y, wl.capacities, wl.L, M_max=10)
+        assert e.value.status == 3
+        # and the context still works afterwards
+        a, o, v = ctx.rcd_partition(X, y, wl.capacities, wl.L)
+        ctx.sync_status()
+        assert int(a.min()) >= 0 and int(a.max()) < wl.W
+
+
+def test_empty_input(rcd):
+    import torch
+    with rcd.Context(0) as ctx:
+        X = torch.empty((0, 16), dtype=torch.int8, device="cuda")
+        y = torch.empty((0,), dtype=torch.int32, device="cuda")
+        a, o, v = ctx.rcd_partition(X, y, [1.0, 2.0], 3)
+        ctx.sync_status()
+        assert a.numel() == 0 and v.shape == (3, 2) and int(v.abs().sum()) == 0
