@@ -172,6 +172,28 @@ RCD_API rcd_status rcd_objective(rcd_ctx *ctx, const void *features_dev, rcd_fea
                          void *part_values_dev, void *total_dev, void *workspace_dev,
                          size_t workspace_bytes, void *cuda_stream);
 
+/* ---- objective of one class without any allocation (no counterpart in the paper) ----------- */
+
+/* The paper has nothing corresponding to this entry point: it exists for callers that cannot
+ * allocate device memory (code running inside a fixed, pre-carved memory budget or in a region
+ * where touching the CUDA allocator is not allowed) and so cannot supply the workspace that
+ * rcd_objective needs.  It computes f(A_j) for the W blocks of ONE class from a similarity
+ * matrix the caller already has (for instance from rcd_similarity), using a 1 MiB scratch array
+ * that is built into the library instead of a workspace.
+ *   S_dev           [M][ldS] row-major, int32 (RCD_FEAT_I8) or fp32 (RCD_FEAT_BF16), ldS >= M
+ *   assignment_dev  [M] block of each sample of the class, in [0, W); negative = in no block
+ *   part_values_dev [W] int64 / double;  total_dev one int64 / double (their sum)
+ * Limits: W <= 1024 and ceil(M/64) * W * 8 <= 1048576 bytes, otherwise RCD_ERR_UNSUPPORTED with
+ * the sizes in rcd_last_error.  The array is held by every GPU that loads the library until the
+ * process exits.  All calls on a device share it: calls whose kernels overlap on the GPU race,
+ * so keep them on one stream or order them with events.  It keeps the previous call's partial
+ * sums; every slot a call reads has been written by that call first, so nothing needs clearing.
+ * The first call on each device looks up the array's device address; make that first call
+ * outside any stream capture.  No cudaMalloc/cudaFree or allocating routine is called. */
+RCD_API rcd_status rcd_objective_class_static(rcd_ctx *ctx, const void *S_dev, rcd_feat_dtype dtype, int64_t M,
+                                      int64_t ldS, const int32_t *assignment_dev, int32_t W,
+                                      void *part_values_dev, void *total_dev, void *cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

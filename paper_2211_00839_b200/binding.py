@@ -30,7 +30,7 @@ STATUS_NAMES = {0: "RCD_OK", 1: "RCD_ERR_INVALID_ARG", 2: "RCD_ERR_UNSUPPORTED",
 EXPORTS = ["rcd_create", "rcd_destroy", "rcd_last_error", "rcd_version", "rcd_sync_status", "rcd_get_profile",
            "rcd_quotas", "rcd_similarity", "rcd_partition_workspace_bytes", "rcd_partition",
            "rcd_partition_host_workspace_bytes", "rcd_partition_host", "rcd_objective_workspace_bytes",
-           "rcd_objective"]
+           "rcd_objective", "rcd_objective_class_static"]
 
 
 class RcdError(RuntimeError):
@@ -74,6 +74,7 @@ def _load() -> C.CDLL:
     lib.rcd_partition.argtypes = [vp, vp, C.c_int, i64, i64, vp, i32, vp, i32, vp, vp, vp, vp, sz, vp]
     lib.rcd_partition_host.argtypes = [vp, vp, C.c_int, i64, i64, vp, i32, vp, i32, vp, vp, vp, vp, sz, vp]
     lib.rcd_objective.argtypes = [vp, vp, C.c_int, i64, i64, vp, i32, vp, i32, vp, vp, vp, sz, vp]
+    lib.rcd_objective_class_static.argtypes = [vp, vp, C.c_int, i64, i64, vp, i32, vp, vp, vp]
     for name in EXPORTS:
         f = getattr(lib, name)
         if name not in ("rcd_destroy", "rcd_last_error", "rcd_version"):
@@ -293,6 +294,21 @@ class Context:
                                       C.c_void_p(values.data_ptr()), C.c_void_p(total.data_ptr()),
                                       C.c_void_p(ws.data_ptr()), ws.numel(), self._stream()))
         return values, total
+
+
+def rcd_objective_class_static(ctx: Context, S, assignment, W: int, part_values, total):
+    """Block values of one class from its similarity matrix, for callers that cannot allocate.
+
+    Everything is passed in: ``S`` [M, ld] int32 / float32, ``assignment`` [M] int32, and the
+    outputs ``part_values`` [W] and ``total`` [1] (int64 for int32 S, float64 for float32 S), all
+    device tensors the caller already owns.  This wrapper allocates nothing either."""
+    torch = _torch()
+    M, ld = S.shape
+    code = RCD_FEAT_I8 if S.dtype == torch.int32 else RCD_FEAT_BF16
+    ctx._check(lib.rcd_objective_class_static(ctx._h, C.c_void_p(S.data_ptr()), code, M, ld,
+                                              C.c_void_p(assignment.data_ptr()), W,
+                                              C.c_void_p(part_values.data_ptr()), C.c_void_p(total.data_ptr()),
+                                              ctx._stream()))
 
 
 def rcd_similarity(ctx: Context, X):
