@@ -73,6 +73,7 @@ size_t layout_workspace(void *base, rcd_feat_dtype dtype, const Sizes &sz, Works
     w.jstar = c.take<int32_t>(L);
     w.sweepN = c.take<int32_t>(L);
     w.sweepParts = c.take<int32_t>(L * kMaxSweepBatch);
+    w.sweepCS = c.take<int32_t>(L);
     w.rowCtr = c.take<int32_t>(L);
     w.sweepList = c.take<int32_t>(2 * L);
     w.stepBytes = c.take<unsigned long long>((size_t)sz.maxM + 1);

@@ -8,9 +8,10 @@
 // and that pass refreshes up to `sweep_batch_max` out-of-date blocks at once.
 //
 // One greedy step t = two launches:
-//   sweep_kernel   persistent CTAs (one per SM) pull row groups of every class that scheduled a
-//                  sweep; each warp streams its rows of S with 128-bit loads against the coverage
-//                  vectors staged in shared memory, reduces with warp shuffles, writes G.
+//   sweep_kernel   persistent CTAs (one per SM) serve every class that scheduled a sweep; teams
+//                  of 1-16 warps pull groups of rows, each warp streams its 128-column chunks of
+//                  those rows with 128-bit loads against the coverage vectors staged in shared
+//                  memory, reduces with warp shuffles, and the team writes G.
 //   select_kernel  one CTA per class: argmax of G_{j*} over the unassigned samples (warp-shuffle
 //                  reduction, lowest index on ties), coverage / value / count update, removal of
 //                  v* from the candidate list, choice of the next block j* (least f among the
@@ -18,6 +19,7 @@
 #include "rcd_internal.h"
 
 #include <limits.h>
+#include <type_traits>
 
 namespace rcd {
 
@@ -51,6 +53,7 @@ struct GreedyParams {
     int32_t *jstar;
     int32_t *sweepN;
     int32_t *sweepParts;
+    int32_t *sweepCS;       // warps that share one row group in the next sweep (1, 2, 4, 8 or 16)
     int32_t *rowCtr;
     int32_t *sweepList;
     int32_t *nSweep;
@@ -64,6 +67,7 @@ struct GreedyParams {
     int32_t batchMax;       // 1, 2, 4 or 8
     int32_t smemBytes;      // dynamic shared memory of the sweep kernel
     int32_t segIters;       // int path: chunk iterations a 32-bit partial sum can take without overflow
+    int32_t sweepWarps;     // warps of one sweep launch (CTAs x 16)
 };
 
 __host__ __device__ inline int rows_per_group(int P) { return P == 8 ? 4 : 8; }
@@ -119,12 +123,15 @@ __device__ void plan_next(const GreedyParams<SV> &prm, int l, int nextStep)
     // shared memory that holds their coverage vectors and by the number of out-of-date blocks
     int cap = prm.batchMax;
     while (cap > 1 && (int64_t)cap * c.ld * (int64_t)sizeof(SV) > prm.smemBytes) cap >>= 1;
+    // n blocks are refreshed; the kernel is instantiated for P = 1, 2, 4, 8 lists, so the list is
+    // padded with copies of j* up to the next power of two (same bytes read, identical values written)
+    const int n = nStale < cap ? nStale : cap;
     int P = 1;
-    while (P * 2 <= cap && P * 2 <= nStale) P *= 2;
+    while (P < n) P *= 2;
     int32_t *parts = prm.sweepParts + (int64_t)l * kMaxSweepBatch;
     if (lane == 0) { parts[0] = jstar; valid[jstar] = 1; }
     __syncwarp();
-    for (int k = 1; k < P; ++k) {
+    for (int k = 1; k < n; ++k) {
         // next out-of-date non-full block of least f: the one most likely to be chosen soon
         FV qF = 0;
         int qP = INT_MAX;
@@ -142,15 +149,25 @@ __device__ void plan_next(const GreedyParams<SV> &prm, int l, int nextStep)
         if (lane == 0) { parts[k] = qP; valid[qP] = 1; }
         __syncwarp();
     }
+    if (lane == 0) for (int k = n; k < P; ++k) parts[k] = jstar;
+    // warps per row group: enough that the row groups of the classes expected to sweep together
+    // (about L / P of them) cover every warp of the launch, at least one 128-column chunk per warp
+    const int R = rows_per_group(P);
+    const int64_t nGroups = (nR + R - 1) / R;
+    const int64_t together = prm.L / P > 1 ? prm.L / P : 1;
+    const int chunks = (c.ld + 127) / 128;
+    int CS = 1;
+    while (CS < 16 && 2 * CS <= chunks && 2 * CS * together * nGroups <= prm.sweepWarps) CS *= 2;
     if (lane == 0) {
         prm.jstar[l] = jstar;
         prm.sweepN[l] = P;
+        prm.sweepCS[l] = CS;
         prm.rowCtr[l] = 0;
         int par = nextStep & 1;
         int slot = atomicAdd(&prm.nSweep[par], 1);
         prm.sweepList[(int64_t)par * prm.L + slot] = l;
-        atomicAdd(&prm.stepBytes[nextStep], (unsigned long long)((int64_t)nR * c.ld + (int64_t)P * c.ld) * sizeof(SV));
-        atomicAdd(&prm.stepOps[nextStep], (unsigned long long)((int64_t)nR * c.M * P));
+        atomicAdd(&prm.stepBytes[nextStep], (unsigned long long)((int64_t)nR * c.ld + (int64_t)n * c.ld) * sizeof(SV));
+        atomicAdd(&prm.stepOps[nextStep], (unsigned long long)((int64_t)nR * c.M * n));
     }
 }
 
@@ -179,14 +196,20 @@ __global__ void __launch_bounds__(kSelectThreads, 4) init_kernel(GreedyParams<SV
 }
 
 // ---------------------------------------------------------------------------------------------
-// Streaming 128-bit load that does not allocate in L1 (S is read once per pass; the L1 is left to
-// nothing in particular, the coverage vectors sit in shared memory).
+// Streaming 128-bit load that does not allocate in L1 (S is read once per pass; the coverage
+// vectors sit in shared memory).
 __device__ __forceinline__ int4 ld_stream(const int4 *p)
 {
     int4 v;
     asm("ld.global.nc.L1::no_allocate.v4.s32 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+        : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
     return v;
+}
+
+// Barrier over the `threads` threads of one team of warps (named barriers 1..15; 0 is the CTA's).
+__device__ __forceinline__ void team_sync(int id, int threads)
+{
+    asm volatile("bar.sync %0, %1;" :: "r"(id), "r"(threads) : "memory");
 }
 
 // Sum NA per-lane partials over the 32 lanes so that lane k ends with the total of partial
@@ -218,24 +241,68 @@ struct WarpMultiReduce<T, 1> {
     }
 };
 
-// One class, P blocks: warps pull groups of R rows until the class's rows are exhausted.
 template <typename SV, int P, int R>
-__device__ __forceinline__ void sweep_class(const GreedyParams<SV> &prm, int l, const ClassDesc &c, int nR,
-                                            const int4 *shCover, const long long *shF, const int32_t *parts)
+__device__ __forceinline__ void accumulate_chunk(const int4 (&s)[R], const int4 *shCover, int ld4, int cc,
+                                                 typename std::conditional<Arith<SV>::kInt, uint32_t, float>::type (&acc)[P * R])
+{
+#pragma unroll
+    for (int p = 0; p < P; ++p) {
+        const int4 m = shCover[p * ld4 + cc];
+        if constexpr (Arith<SV>::kInt) {
+#pragma unroll
+            for (int r = 0; r < R; ++r)
+                acc[r * P + p] += ((uint32_t)max(s[r].x, m.x) + (uint32_t)max(s[r].y, m.y)) +
+                                  ((uint32_t)max(s[r].z, m.z) + (uint32_t)max(s[r].w, m.w));
+        } else {
+            const float m0 = __int_as_float(m.x), m1 = __int_as_float(m.y);
+            const float m2 = __int_as_float(m.z), m3 = __int_as_float(m.w);
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                float a = acc[r * P + p];
+                a += fmaxf(__int_as_float(s[r].x) - m0, 0.f);
+                a += fmaxf(__int_as_float(s[r].y) - m1, 0.f);
+                a += fmaxf(__int_as_float(s[r].z) - m2, 0.f);
+                a += fmaxf(__int_as_float(s[r].w) - m3, 0.f);
+                acc[r * P + p] = a;
+            }
+        }
+    }
+}
+
+// One class, P blocks.  The CTA's 16 warps form teams of CS warps; a team pulls a group of R rows
+// from the class's ticket counter and its warps take interleaved 128-column chunks of those rows,
+// so that a sweep with few rows left still spreads over every warp of the GPU.  Per-warp partial
+// sums meet in shared memory and are added in warp order (fixed, reproducible).
+template <typename SV, int P, int R>
+__device__ __forceinline__ void sweep_class(const GreedyParams<SV> &prm, int l, const ClassDesc &c, int nR, int CS,
+                                            const int4 *shCover, const long long *shF, const int32_t *parts,
+                                            int *shTicket, typename Arith<SV>::GV *shPart)
 {
     using GV = typename Arith<SV>::GV;
+    using AccT = typename std::conditional<Arith<SV>::kInt, uint32_t, float>::type;
     constexpr int NA = P * R;
-    const int lane = threadIdx.x & 31;
+    constexpr bool kPrefetch = (R <= 4);          // second register buffer only where it fits
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int team = warp / CS, wIn = warp - team * CS;
+    const int teamThreads = CS * 32, barId = 1 + team;
     const int ld4 = c.ld >> 2;
     const int nGroups = (nR + R - 1) / R;
+    const int stride = CS * 32;
     const SV *Sl = prm.S + c.sOff;
     const int32_t *cand = prm.cand + c.row0;
     GV *G = prm.gains + c.vOff;
+    GV *myPart = shPart + (team * CS) * 32;       // [CS][32] for this team (teams are CS-aligned)
 
     for (;;) {
         int g = 0;
-        if (lane == 0) g = atomicAdd(&prm.rowCtr[l], 1);
-        g = __shfl_sync(0xffffffffu, g, 0);
+        if (CS == 1) {
+            if (lane == 0) g = atomicAdd(&prm.rowCtr[l], 1);
+            g = __shfl_sync(0xffffffffu, g, 0);
+        } else {
+            if (wIn == 0 && lane == 0) shTicket[team] = atomicAdd(&prm.rowCtr[l], 1);
+            team_sync(barId, teamThreads);
+            g = shTicket[team];
+        }
         if (g >= nGroups) break;
         const int k0 = g * R;
         int vrow[R];
@@ -246,29 +313,43 @@ __device__ __forceinline__ void sweep_class(const GreedyParams<SV> &prm, int l, 
             vrow[r] = cand[k < nR ? k : nR - 1];
             rp[r] = reinterpret_cast<const int4 *>(Sl + (int64_t)vrow[r] * c.ld);
         }
-        GV total = 0;
+        GV total;
+        const int first = wIn * 32 + lane;
         if constexpr (Arith<SV>::kInt) {
             // sum_i max(S[v][i], cover[i]) in unsigned 32-bit partials (every term is in [0, 2^31)),
             // widened to 64 bits every segIters iterations; the gain is that sum minus f_p.
             unsigned long long tot = 0;
-            const int segLen = prm.segIters * 32;
-            for (int c0 = 0; c0 < ld4; c0 += segLen) {
-                uint32_t acc[NA];
+            // every lane runs every segment (the shuffles below need the whole warp), whether or
+            // not its own columns reach into it
+            const int segLen = prm.segIters * stride;
+            for (int base = 0; base < ld4; base += segLen) {
+                AccT acc[NA];
 #pragma unroll
                 for (int i = 0; i < NA; ++i) acc[i] = 0u;
-                const int cEnd = min(ld4, c0 + segLen);
-#pragma unroll 2
-                for (int cc = c0 + lane; cc < cEnd; cc += 32) {
-                    int4 s[R];
+                const int c0 = base + first;
+                const int cEnd = min(ld4, base + segLen);
+                if constexpr (kPrefetch) {
+                    int4 cur[R], nxt[R];
+                    if (c0 < cEnd) {
 #pragma unroll
-                    for (int r = 0; r < R; ++r) s[r] = ld_stream(rp[r] + cc);
+                        for (int r = 0; r < R; ++r) cur[r] = ld_stream(rp[r] + c0);
+                    }
+                    for (int cc = c0; cc < cEnd; cc += stride) {
+                        const int cn = cc + stride;
+                        if (cn < cEnd) {
 #pragma unroll
-                    for (int p = 0; p < P; ++p) {
-                        const int4 m = shCover[p * ld4 + cc];
+                            for (int r = 0; r < R; ++r) nxt[r] = ld_stream(rp[r] + cn);
+                        }
+                        accumulate_chunk<SV, P, R>(cur, shCover, ld4, cc, acc);
 #pragma unroll
-                        for (int r = 0; r < R; ++r)
-                            acc[r * P + p] += ((uint32_t)max(s[r].x, m.x) + (uint32_t)max(s[r].y, m.y)) +
-                                              ((uint32_t)max(s[r].z, m.z) + (uint32_t)max(s[r].w, m.w));
+                        for (int r = 0; r < R; ++r) cur[r] = nxt[r];
+                    }
+                } else {
+                    for (int cc = c0; cc < cEnd; cc += stride) {
+                        int4 s[R];
+#pragma unroll
+                        for (int r = 0; r < R; ++r) s[r] = ld_stream(rp[r] + cc);
+                        accumulate_chunk<SV, P, R>(s, shCover, ld4, cc, acc);
                     }
                 }
                 unsigned long long wide[NA / 2];
@@ -285,35 +366,47 @@ __device__ __forceinline__ void sweep_class(const GreedyParams<SV> &prm, int l, 
             }
             total = (GV)tot;
         } else {
-            float acc[NA];
+            AccT acc[NA];
 #pragma unroll
             for (int i = 0; i < NA; ++i) acc[i] = 0.f;
-#pragma unroll 2
-            for (int cc = lane; cc < ld4; cc += 32) {
-                int4 s[R];
+            if constexpr (kPrefetch) {
+                int4 cur[R], nxt[R];
+                if (first < ld4) {
 #pragma unroll
-                for (int r = 0; r < R; ++r) s[r] = ld_stream(rp[r] + cc);
+                    for (int r = 0; r < R; ++r) cur[r] = ld_stream(rp[r] + first);
+                }
+                for (int cc = first; cc < ld4; cc += stride) {
+                    const int cn = cc + stride;
+                    if (cn < ld4) {
 #pragma unroll
-                for (int p = 0; p < P; ++p) {
-                    const int4 mi = shCover[p * ld4 + cc];
-                    const float m0 = __int_as_float(mi.x), m1 = __int_as_float(mi.y);
-                    const float m2 = __int_as_float(mi.z), m3 = __int_as_float(mi.w);
-#pragma unroll
-                    for (int r = 0; r < R; ++r) {
-                        float a = acc[r * P + p];
-                        a += fmaxf(__int_as_float(s[r].x) - m0, 0.f);
-                        a += fmaxf(__int_as_float(s[r].y) - m1, 0.f);
-                        a += fmaxf(__int_as_float(s[r].z) - m2, 0.f);
-                        a += fmaxf(__int_as_float(s[r].w) - m3, 0.f);
-                        acc[r * P + p] = a;
+                        for (int r = 0; r < R; ++r) nxt[r] = ld_stream(rp[r] + cn);
                     }
+                    accumulate_chunk<SV, P, R>(cur, shCover, ld4, cc, acc);
+#pragma unroll
+                    for (int r = 0; r < R; ++r) cur[r] = nxt[r];
+                }
+            } else {
+                for (int cc = first; cc < ld4; cc += stride) {
+                    int4 s[R];
+#pragma unroll
+                    for (int r = 0; r < R; ++r) s[r] = ld_stream(rp[r] + cc);
+                    accumulate_chunk<SV, P, R>(s, shCover, ld4, cc, acc);
                 }
             }
             total = WarpMultiReduce<float, NA>::run(acc, 16, lane);
         }
-        // lane k holds partial k / (32/NA) = r * P + p
+        // lane k holds partial k / (32/NA) = r * P + p of this warp's columns
+        if (CS > 1) {
+            myPart[wIn * 32 + lane] = total;
+            team_sync(barId, teamThreads);
+            if (wIn == 0) {
+                GV sum = myPart[lane];
+                for (int w = 1; w < CS; ++w) sum += myPart[w * 32 + lane];
+                total = sum;
+            }
+        }
         constexpr int kShare = 32 / NA;
-        if ((lane % kShare) == 0) {
+        if (wIn == 0 && (lane % kShare) == 0) {
             const int idx = lane / kShare;
             const int r = idx / P, p = idx % P;
             if (k0 + r < nR) {
@@ -332,10 +425,15 @@ __device__ __forceinline__ void sweep_class(const GreedyParams<SV> &prm, int l, 
 template <typename SV>
 __global__ void __launch_bounds__(kSweepThreads, 1) sweep_kernel(GreedyParams<SV> prm, int step)
 {
+    using GV = typename Arith<SV>::GV;
     extern __shared__ int4 shCover[];
     __shared__ long long shF[kMaxSweepBatch];
     __shared__ int32_t shParts[kMaxSweepBatch];
+    __shared__ int shTicket[kSweepThreads / 32];
+    __shared__ GV shPart[kSweepThreads];
     __shared__ int shGo;
+    cudaGridDependencySynchronize();              // the previous launch (select / init) has finished
+    cudaTriggerProgrammaticLaunchCompletion();
     const int par = step & 1;
     const int nS = prm.nSweep[par];
     if (blockIdx.x == 0 && threadIdx.x == 0) prm.nSweep[par ^ 1] = 0;   // list the coming select fills
@@ -348,6 +446,7 @@ __global__ void __launch_bounds__(kSweepThreads, 1) sweep_kernel(GreedyParams<SV
         const ClassDesc c = prm.desc[l];
         const int nR = prm.nR[l];
         const int P = prm.sweepN[l];
+        const int CS = prm.sweepCS[l];
         const int R = rows_per_group(P);
         const int nGroups = (nR + R - 1) / R;
         if (threadIdx.x == 0) shGo = (*(volatile int32_t *)&prm.rowCtr[l] < nGroups) ? 1 : 0;
@@ -367,10 +466,10 @@ __global__ void __launch_bounds__(kSweepThreads, 1) sweep_kernel(GreedyParams<SV
             }
             __syncthreads();
             switch (P) {
-            case 1: sweep_class<SV, 1, 8>(prm, l, c, nR, shCover, shF, shParts); break;
-            case 2: sweep_class<SV, 2, 8>(prm, l, c, nR, shCover, shF, shParts); break;
-            case 4: sweep_class<SV, 4, 8>(prm, l, c, nR, shCover, shF, shParts); break;
-            default: sweep_class<SV, 8, 4>(prm, l, c, nR, shCover, shF, shParts); break;
+            case 1: sweep_class<SV, 1, 8>(prm, l, c, nR, CS, shCover, shF, shParts, shTicket, shPart); break;
+            case 2: sweep_class<SV, 2, 8>(prm, l, c, nR, CS, shCover, shF, shParts, shTicket, shPart); break;
+            case 4: sweep_class<SV, 4, 8>(prm, l, c, nR, CS, shCover, shF, shParts, shTicket, shPart); break;
+            default: sweep_class<SV, 8, 4>(prm, l, c, nR, CS, shCover, shF, shParts, shTicket, shPart); break;
             }
         }
         __syncthreads();
@@ -386,6 +485,8 @@ __global__ void __launch_bounds__(kSelectThreads, 4) select_kernel(GreedyParams<
     __shared__ GV shG[kSelectThreads / 32];
     __shared__ int shV[kSelectThreads / 32];
     __shared__ int shPick;
+    cudaGridDependencySynchronize();              // the sweep of this step has finished
+    cudaTriggerProgrammaticLaunchCompletion();
     const int l = blockIdx.x;
     const int nR = prm.nR[l];
     if (nR == 0) return;
@@ -469,6 +570,24 @@ __global__ void __launch_bounds__(kSelectThreads, 4) select_kernel(GreedyParams<
 }
 
 // ---------------------------------------------------------------------------------------------
+// Launch with programmatic stream serialization: the next kernel's CTAs may be placed while this
+// one drains; every kernel starts with cudaGridDependencySynchronize(), so data dependencies hold.
+template <typename... KArgs, typename... Args>
+static cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 template <typename SV>
 static rcd_status run_greedy(rcd_ctx *ctx, const Sizes &sz, const Workspace &ws,
                              const std::vector<ClassDesc> &descHost, int32_t *assignment, int32_t *order,
@@ -491,6 +610,7 @@ static rcd_status run_greedy(rcd_ctx *ctx, const Sizes &sz, const Workspace &ws,
     prm.jstar = ws.jstar;
     prm.sweepN = ws.sweepN;
     prm.sweepParts = ws.sweepParts;
+    prm.sweepCS = ws.sweepCS;
     prm.rowCtr = ws.rowCtr;
     prm.sweepList = ws.sweepList;
     prm.nSweep = ws.nSweep;
@@ -505,6 +625,7 @@ static rcd_status run_greedy(rcd_ctx *ctx, const Sizes &sz, const Workspace &ws,
     int batch = ctx->cfg.sweep_batch_max;
     if (batch <= 0) batch = kMaxSweepBatch;
     prm.batchMax = batch;
+    prm.sweepWarps = ctx->smCount * (kSweepThreads / 32);
 
     int maxLd = 0;
     for (const auto &c : descHost) if (c.ld > maxLd) maxLd = c.ld;
@@ -545,9 +666,9 @@ static rcd_status run_greedy(rcd_ctx *ctx, const Sizes &sz, const Workspace &ws,
     ctx->sweepEventsUsed = 0;
     for (int64_t t = 0; t < sz.maxM; ++t) {
         if (perSweep) RCD_CUDA(ctx, cudaEventRecord(ctx->evSweep[2 * t], st));
-        sweep_kernel<SV><<<ctx->smCount, kSweepThreads, (size_t)smem, st>>>(prm, (int)t);
+        RCD_CUDA(ctx, launch_pdl(sweep_kernel<SV>, dim3(ctx->smCount), dim3(kSweepThreads), (size_t)smem, st, prm, (int)t));
         if (perSweep) RCD_CUDA(ctx, cudaEventRecord(ctx->evSweep[2 * t + 1], st));
-        select_kernel<SV><<<sz.L, kSelectThreads, 0, st>>>(prm, (int)t);
+        RCD_CUDA(ctx, launch_pdl(select_kernel<SV>, dim3(sz.L), dim3(kSelectThreads), 0, st, prm, (int)t));
         ctx->kernelLaunches += 2;
     }
     if (perSweep) ctx->sweepEventsUsed = 2 * sz.maxM;

@@ -79,6 +79,7 @@ struct Workspace {
     int32_t *jstar;         // [L] block chosen for the next pick (-1: none)
     int32_t *sweepN;        // [L] blocks to refresh in the next sweep (0: none)
     int32_t *sweepParts;    // [L][kMaxSweepBatch]
+    int32_t *sweepCS;       // [L] warps per row group in the next sweep
     int32_t *rowCtr;        // [L] ticket counter over row groups of the running sweep
     int32_t *sweepList;     // [2][L] classes that sweep in the next step (double-buffered by step parity)
     int32_t *nSweep;        // [2]
