@@ -68,40 +68,53 @@ struct GreedyParams {
     int32_t smemBytes;      // dynamic shared memory of the sweep kernel
     int32_t segIters;       // int path: chunk iterations a 32-bit partial sum can take without overflow
     int32_t sweepWarps;     // warps of one sweep launch (CTAs x 16)
+    uint32_t one;           // the value 1, opaque to the compiler (see accumulate_chunk)
 };
 
 __host__ __device__ inline int rows_per_group(int P) { return P == 8 ? 4 : 8; }
 
 // ---------------------------------------------------------------------------------------------
-// Choice of the next block and of the blocks the next sweep refreshes.  Run by warp 0 of the
-// class's CTA after a __syncthreads().
+// Choice of the next block and of the blocks the next sweep refreshes.  Called by every thread of
+// the class's CTA after a __syncthreads(); the block values and flags are staged in shared memory
+// once, then warp 0 decides.
+constexpr int kMaxBlocks = 1024;
+template <typename FV>
+struct PlanShared {
+    FV f[kMaxBlocks];
+    uint8_t open[kMaxBlocks];      // bit 0: block is not full, bit 1: its stored gains are out of date
+};
+
 template <typename SV>
-__device__ void plan_next(const GreedyParams<SV> &prm, int l, int nextStep)
+__device__ void plan_next(const GreedyParams<SV> &prm, int l, int nextStep, PlanShared<typename Arith<SV>::FV> &sh)
 {
     using FV = typename Arith<SV>::FV;
     const int lane = threadIdx.x & 31;
-    if ((threadIdx.x >> 5) != 0) return;
     const int W = prm.W;
     const int nR = prm.nR[l];
-    const ClassDesc c = prm.desc[l];
-    FV *f = prm.fval + (int64_t)l * W;
-    int32_t *cnt = prm.cnt + (int64_t)l * W;
-    const int32_t *quota = prm.quota + (int64_t)l * W;
     uint8_t *valid = prm.valid + (int64_t)l * W;
-
     if (nR == 0) {
-        if (lane == 0) { prm.jstar[l] = -1; prm.sweepN[l] = 0; }
+        if (threadIdx.x == 0) { prm.jstar[l] = -1; prm.sweepN[l] = 0; }
         return;
     }
+    for (int p = threadIdx.x; p < W; p += blockDim.x) {
+        const int64_t at = (int64_t)l * W + p;
+        sh.f[p] = prm.fval[at];
+        sh.open[p] = (uint8_t)((prm.cnt[at] < prm.quota[at] ? 1 : 0) | (valid[p] ? 0 : 2));
+    }
+    __syncthreads();
+    if ((threadIdx.x >> 5) != 0) return;
+    const ClassDesc c = prm.desc[l];
+
     // j* = argmin over non-full blocks of f, ties -> lowest index
     FV bestF = 0;
     int bestP = INT_MAX;
     int nStale = 0;
     for (int p = lane; p < W; p += 32) {
-        if (cnt[p] < quota[p]) {
-            FV fp = f[p];
+        const uint8_t o = sh.open[p];
+        if (o & 1) {
+            const FV fp = sh.f[p];
             if (bestP == INT_MAX || fp < bestF) { bestF = fp; bestP = p; }
-            if (!valid[p]) ++nStale;
+            if (o & 2) ++nStale;
         }
     }
     for (int off = 16; off > 0; off >>= 1) {
@@ -115,29 +128,29 @@ __device__ void plan_next(const GreedyParams<SV> &prm, int l, int nextStep)
         return;
     }
     const int jstar = bestP;
-    if (valid[jstar]) {
+    if (!(sh.open[jstar] & 2)) {
         if (lane == 0) { prm.jstar[l] = jstar; prm.sweepN[l] = 0; }
         return;
     }
-    // how many blocks one pass can refresh: power of two, bounded by the configuration, by the
-    // shared memory that holds their coverage vectors and by the number of out-of-date blocks
+    // how many blocks one pass can refresh: bounded by the configuration, by the shared memory
+    // that holds their coverage vectors and by the number of out-of-date blocks
     int cap = prm.batchMax;
     while (cap > 1 && (int64_t)cap * c.ld * (int64_t)sizeof(SV) > prm.smemBytes) cap >>= 1;
-    // n blocks are refreshed; the kernel is instantiated for P = 1, 2, 4, 8 lists, so the list is
+    // n blocks are refreshed; the kernel is instantiated for lists of 1, 2, 4, 8, so the list is
     // padded with copies of j* up to the next power of two (same bytes read, identical values written)
     const int n = nStale < cap ? nStale : cap;
     int P = 1;
     while (P < n) P *= 2;
     int32_t *parts = prm.sweepParts + (int64_t)l * kMaxSweepBatch;
-    if (lane == 0) { parts[0] = jstar; valid[jstar] = 1; }
+    if (lane == 0) { parts[0] = jstar; valid[jstar] = 1; sh.open[jstar] = 1; }
     __syncwarp();
     for (int k = 1; k < n; ++k) {
         // next out-of-date non-full block of least f: the one most likely to be chosen soon
         FV qF = 0;
         int qP = INT_MAX;
         for (int p = lane; p < W; p += 32) {
-            if (cnt[p] < quota[p] && !valid[p]) {
-                FV fp = f[p];
+            if (sh.open[p] == 3) {
+                const FV fp = sh.f[p];
                 if (qP == INT_MAX || fp < qF) { qF = fp; qP = p; }
             }
         }
@@ -146,7 +159,7 @@ __device__ void plan_next(const GreedyParams<SV> &prm, int l, int nextStep)
             int oP = __shfl_xor_sync(0xffffffffu, qP, off);
             if (oP != INT_MAX && (qP == INT_MAX || oF < qF || (oF == qF && oP < qP))) { qF = oF; qP = oP; }
         }
-        if (lane == 0) { parts[k] = qP; valid[qP] = 1; }
+        if (lane == 0) { parts[k] = qP; valid[qP] = 1; sh.open[qP] = 1; }
         __syncwarp();
     }
     if (lane == 0) for (int k = n; k < P; ++k) parts[k] = jstar;
@@ -176,6 +189,7 @@ template <typename SV>
 __global__ void __launch_bounds__(kSelectThreads, 4) init_kernel(GreedyParams<SV> prm)
 {
     using FV = typename Arith<SV>::FV;
+    __shared__ PlanShared<FV> shPlan;
     const int l = blockIdx.x;
     const ClassDesc c = prm.desc[l];
     const int W = prm.W;
@@ -192,7 +206,7 @@ __global__ void __launch_bounds__(kSelectThreads, 4) init_kernel(GreedyParams<SV
     }
     if (threadIdx.x == 0) prm.nR[l] = c.M;
     __syncthreads();
-    plan_next(prm, l, 0);
+    plan_next(prm, l, 0, shPlan);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -241,8 +255,17 @@ struct WarpMultiReduce<T, 1> {
     }
 };
 
+// acc + x computed as x * one + acc: an integer multiply-add issues on the FMA pipe, so the adds
+// of the integer path do not compete with the max operations for the ALU pipe.
+__device__ __forceinline__ uint32_t add_on_fma_pipe(uint32_t x, uint32_t one, uint32_t acc)
+{
+    uint32_t r;
+    asm("mad.lo.u32 %0, %1, %2, %3;" : "=r"(r) : "r"(x), "r"(one), "r"(acc));
+    return r;
+}
+
 template <typename SV, int P, int R>
-__device__ __forceinline__ void accumulate_chunk(const int4 (&s)[R], const int4 *shCover, int ld4, int cc,
+__device__ __forceinline__ void accumulate_chunk(uint32_t one, const int4 (&s)[R], const int4 *shCover, int ld4, int cc,
                                                  typename std::conditional<Arith<SV>::kInt, uint32_t, float>::type (&acc)[P * R])
 {
 #pragma unroll
@@ -250,9 +273,14 @@ __device__ __forceinline__ void accumulate_chunk(const int4 (&s)[R], const int4 
         const int4 m = shCover[p * ld4 + cc];
         if constexpr (Arith<SV>::kInt) {
 #pragma unroll
-            for (int r = 0; r < R; ++r)
-                acc[r * P + p] += ((uint32_t)max(s[r].x, m.x) + (uint32_t)max(s[r].y, m.y)) +
-                                  ((uint32_t)max(s[r].z, m.z) + (uint32_t)max(s[r].w, m.w));
+            for (int r = 0; r < R; ++r) {
+                uint32_t a = acc[r * P + p];
+                a = add_on_fma_pipe((uint32_t)max(s[r].x, m.x), one, a);
+                a = add_on_fma_pipe((uint32_t)max(s[r].y, m.y), one, a);
+                a = add_on_fma_pipe((uint32_t)max(s[r].z, m.z), one, a);
+                a = add_on_fma_pipe((uint32_t)max(s[r].w, m.w), one, a);
+                acc[r * P + p] = a;
+            }
         } else {
             const float m0 = __int_as_float(m.x), m1 = __int_as_float(m.y);
             const float m2 = __int_as_float(m.z), m3 = __int_as_float(m.w);
@@ -340,7 +368,7 @@ __device__ __forceinline__ void sweep_class(const GreedyParams<SV> &prm, int l, 
 #pragma unroll
                             for (int r = 0; r < R; ++r) nxt[r] = ld_stream(rp[r] + cn);
                         }
-                        accumulate_chunk<SV, P, R>(cur, shCover, ld4, cc, acc);
+                        accumulate_chunk<SV, P, R>(prm.one, cur, shCover, ld4, cc, acc);
 #pragma unroll
                         for (int r = 0; r < R; ++r) cur[r] = nxt[r];
                     }
@@ -349,7 +377,7 @@ __device__ __forceinline__ void sweep_class(const GreedyParams<SV> &prm, int l, 
                         int4 s[R];
 #pragma unroll
                         for (int r = 0; r < R; ++r) s[r] = ld_stream(rp[r] + cc);
-                        accumulate_chunk<SV, P, R>(s, shCover, ld4, cc, acc);
+                        accumulate_chunk<SV, P, R>(prm.one, s, shCover, ld4, cc, acc);
                     }
                 }
                 unsigned long long wide[NA / 2];
@@ -381,7 +409,7 @@ __device__ __forceinline__ void sweep_class(const GreedyParams<SV> &prm, int l, 
 #pragma unroll
                         for (int r = 0; r < R; ++r) nxt[r] = ld_stream(rp[r] + cn);
                     }
-                    accumulate_chunk<SV, P, R>(cur, shCover, ld4, cc, acc);
+                    accumulate_chunk<SV, P, R>(prm.one, cur, shCover, ld4, cc, acc);
 #pragma unroll
                     for (int r = 0; r < R; ++r) cur[r] = nxt[r];
                 }
@@ -390,7 +418,7 @@ __device__ __forceinline__ void sweep_class(const GreedyParams<SV> &prm, int l, 
                     int4 s[R];
 #pragma unroll
                     for (int r = 0; r < R; ++r) s[r] = ld_stream(rp[r] + cc);
-                    accumulate_chunk<SV, P, R>(s, shCover, ld4, cc, acc);
+                    accumulate_chunk<SV, P, R>(prm.one, s, shCover, ld4, cc, acc);
                 }
             }
             total = WarpMultiReduce<float, NA>::run(acc, 16, lane);
@@ -478,10 +506,11 @@ __global__ void __launch_bounds__(kSweepThreads, 1) sweep_kernel(GreedyParams<SV
 
 // ---------------------------------------------------------------------------------------------
 template <typename SV>
-__global__ void __launch_bounds__(kSelectThreads, 4) select_kernel(GreedyParams<SV> prm, int step)
+__global__ void __launch_bounds__(kSelectThreads, 2) select_kernel(GreedyParams<SV> prm, int step)
 {
     using GV = typename Arith<SV>::GV;
     using FV = typename Arith<SV>::FV;
+    __shared__ PlanShared<FV> shPlan;
     __shared__ GV shG[kSelectThreads / 32];
     __shared__ int shV[kSelectThreads / 32];
     __shared__ int shPick;
@@ -497,14 +526,17 @@ __global__ void __launch_bounds__(kSelectThreads, 4) select_kernel(GreedyParams<
     int32_t *cand = prm.cand + c.row0;
     int32_t *pos = prm.pos + c.row0;
     const GV *G = prm.gains + c.vOff + (int64_t)j * c.ld;
+    const int lastV = cand[nR - 1];               // needed by the removal below; fetched early
 
-    // v* = argmax over the unassigned samples, ties -> lowest class-local index (GreedyStep)
+    // v* = argmax over the unassigned samples, ties -> lowest class-local index (GreedyStep).
+    // Walks all samples with independent, coalesced loads (pos[v] < 0 marks an assigned sample).
     GV bestG = 0;
     int bestV = INT_MAX;
-    for (int k = threadIdx.x; k < nR; k += blockDim.x) {
-        int v = cand[k];
-        GV g = G[v];
-        if (bestV == INT_MAX || g > bestG || (g == bestG && v < bestV)) { bestG = g; bestV = v; }
+#pragma unroll 4
+    for (int v = threadIdx.x; v < c.M; v += kSelectThreads) {
+        const GV g = G[v];
+        const int ps = pos[v];
+        if (ps >= 0 && (bestV == INT_MAX || g > bestG)) { bestG = g; bestV = v; }
     }
     for (int off = 16; off > 0; off >>= 1) {
         GV oG = __shfl_xor_sync(0xffffffffu, bestG, off);
@@ -533,12 +565,28 @@ __global__ void __launch_bounds__(kSelectThreads, 4) select_kernel(GreedyParams<
         if (threadIdx.x == 0) atomicOr(prm.status, kDevBadState);
         return;
     }
+    // bookkeeping by the last warp while the others fold row v* into the coverage vector
+    if (threadIdx.x == kSelectThreads - 32) {
+        const int64_t at = (int64_t)l * prm.W + j;
+        prm.fval[at] += (FV)gstar;
+        prm.cnt[at] += 1;
+        prm.valid[at] = 0;
+        const int global = prm.perm[c.row0 + vstar];
+        prm.assignment[global] = j;
+        if (prm.order) prm.order[c.row0 + (c.M - nR)] = global;
+        const int k = pos[vstar];
+        cand[k] = lastV;
+        pos[lastV] = k;
+        pos[vstar] = -1;
+        prm.nR[l] = nR - 1;
+    }
     // cover_j <- max(cover_j, S[v*][.])
     {
         const int ld4 = c.ld >> 2;
         int4 *cov = reinterpret_cast<int4 *>(prm.cover + c.vOff + (int64_t)j * c.ld);
         const int4 *row = reinterpret_cast<const int4 *>(prm.S + c.sOff + (int64_t)vstar * c.ld);
-        for (int i = threadIdx.x; i < ld4; i += blockDim.x) {
+#pragma unroll 2
+        for (int i = threadIdx.x; i < ld4; i += kSelectThreads) {
             int4 a = cov[i], b = row[i];
             if constexpr (Arith<SV>::kInt) {
                 a.x = max(a.x, b.x); a.y = max(a.y, b.y); a.z = max(a.z, b.z); a.w = max(a.w, b.w);
@@ -551,22 +599,8 @@ __global__ void __launch_bounds__(kSelectThreads, 4) select_kernel(GreedyParams<
             cov[i] = a;
         }
     }
-    if (threadIdx.x == 0) {
-        const int64_t at = (int64_t)l * prm.W + j;
-        prm.fval[at] += (FV)gstar;
-        prm.cnt[at] += 1;
-        prm.valid[at] = 0;
-        const int global = prm.perm[c.row0 + vstar];
-        prm.assignment[global] = j;
-        if (prm.order) prm.order[c.row0 + (c.M - nR)] = global;
-        const int k = pos[vstar];
-        const int lastV = cand[nR - 1];
-        cand[k] = lastV;
-        pos[lastV] = k;
-        prm.nR[l] = nR - 1;
-    }
     __syncthreads();
-    plan_next(prm, l, step + 1);
+    plan_next(prm, l, step + 1, shPlan);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -626,6 +660,7 @@ static rcd_status run_greedy(rcd_ctx *ctx, const Sizes &sz, const Workspace &ws,
     if (batch <= 0) batch = kMaxSweepBatch;
     prm.batchMax = batch;
     prm.sweepWarps = ctx->smCount * (kSweepThreads / 32);
+    prm.one = 1u;
 
     int maxLd = 0;
     for (const auto &c : descHost) if (c.ld > maxLd) maxLd = c.ld;

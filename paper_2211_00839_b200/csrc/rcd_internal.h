@@ -13,7 +13,7 @@ namespace rcd {
 
 constexpr int kMaxSweepBatch = 8;          // blocks refreshed by one pass over S
 constexpr int kSweepThreads = 512;         // sweep CTA: 16 warps, one CTA per SM
-constexpr int kSelectThreads = 256;        // pick/update CTA: one per class
+constexpr int kSelectThreads = 512;        // pick/update CTA: one per class
 constexpr size_t kAlign = 256;
 
 // Device-side status bits (OR-ed into the status word).
