@@ -74,15 +74,16 @@ typedef struct {
     int64_t sweep_elem_ops;    /* (element of S) x (block refreshed) pairs those launches evaluated */
     int64_t kernel_launches;   /* kernels this library launched during the call */
     int64_t steps;             /* greedy steps executed (= largest class size) */
-    int64_t reserved[6];
+    int64_t similarity_tc_launches; /* similarity launches of the last call that ran on the tensor cores */
+    int64_t reserved[5];
 } rcd_profile;
 
 typedef struct rcd_ctx rcd_ctx;
 
 /* ---- context ------------------------------------------------------------------------------ */
 
-/* Creates a context bound to CUDA device `cuda_device` (it owns only a few events and a small
- * pinned staging buffer).  `cfg_or_null` NULL = defaults.  Fails with RCD_ERR_UNSUPPORTED on a
+/* Creates a context bound to CUDA device `cuda_device` (it owns only a few events, a small pinned
+ * staging buffer and a 256-byte device status block).  `cfg_or_null` NULL = defaults.  Fails with RCD_ERR_UNSUPPORTED on a
  * device that is not compute capability 10.x, RCD_ERR_CUDA when no device can be used. */
 RCD_API rcd_status rcd_create(rcd_ctx **out, int cuda_device, const rcd_config *cfg_or_null);
 RCD_API void rcd_destroy(rcd_ctx *ctx);

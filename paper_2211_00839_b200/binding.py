@@ -48,7 +48,7 @@ class RcdProfile(C.Structure):
     _fields_ = [("total_ms", C.c_double), ("group_ms", C.c_double), ("similarity_ms", C.c_double),
                 ("greedy_ms", C.c_double), ("sweep_ms", C.c_double), ("sweep_launches", C.c_int64),
                 ("sweep_bytes", C.c_int64), ("sweep_elem_ops", C.c_int64), ("kernel_launches", C.c_int64),
-                ("steps", C.c_int64), ("reserved", C.c_int64 * 6)]
+                ("steps", C.c_int64), ("similarity_tc_launches", C.c_int64), ("reserved", C.c_int64 * 5)]
 
 
 def _load() -> C.CDLL:

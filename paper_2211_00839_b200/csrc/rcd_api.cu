@@ -268,6 +268,10 @@ rcd_status rcd_create(rcd_ctx **out, int cuda_device, const rcd_config *cfg)
         delete ctx;
         return RCD_ERR_CUDA;
     }
+    if (cudaMalloc((void **)&ctx->statusOwn, 256) != cudaSuccess || cudaMemset(ctx->statusOwn, 0, 256) != cudaSuccess) {
+        rcd_destroy(ctx);
+        return RCD_ERR_CUDA;
+    }
     for (auto &e : ctx->evPhase)
         if (cudaEventCreate(&e) != cudaSuccess) { rcd_destroy(ctx); return RCD_ERR_CUDA; }
     *out = ctx;
@@ -281,6 +285,7 @@ void rcd_destroy(rcd_ctx *ctx)
     for (auto &e : ctx->evPhase) if (e) cudaEventDestroy(e);
     for (auto &e : ctx->evSweep) cudaEventDestroy(e);
     if (ctx->hostStage) cudaFreeHost(ctx->hostStage);
+    if (ctx->statusOwn) cudaFree(ctx->statusOwn);
     delete ctx;
 }
 
@@ -294,6 +299,7 @@ rcd_status rcd_sync_status(rcd_ctx *ctx, void *cuda_stream)
     RCD_CUDA(ctx, cudaMemcpy(&word, ctx->statusDev, sizeof word, cudaMemcpyDeviceToHost));
     if (word == 0) return RCD_OK;
     if (word & kDevBadLabel) return fail(ctx, RCD_ERR_INVALID_ARG, "device status %d: label out of range", word);
+    if (word & kDevTimeout) return fail(ctx, RCD_ERR_TIMEOUT, "device status %d: a bounded wait inside a kernel ran out", word);
     return fail(ctx, RCD_ERR_INTERNAL, "device status %d: greedy state inconsistent", word);
 }
 
@@ -303,6 +309,7 @@ rcd_status rcd_get_profile(rcd_ctx *ctx, rcd_profile *out)
     memset(out, 0, sizeof *out);
     out->kernel_launches = ctx->kernelLaunches;
     out->steps = ctx->steps;
+    out->similarity_tc_launches = ctx->tcLaunches;
     if (!ctx->phaseValid) return RCD_OK;
     RCD_CUDA(ctx, cudaEventSynchronize(ctx->evPhase[4]));
     float ms = 0.f;
@@ -358,6 +365,9 @@ rcd_status rcd_similarity(rcd_ctx *ctx, const void *X_dev, rcd_feat_dtype dtype,
     cls.maxM = M;
     cls.tiles128 = batch * ((M + 127) / 128) * ((M + 127) / 128);
     ctx->kernelLaunches = 0;
+    ctx->tcLaunches = 0;
+    ctx->statusDev = ctx->statusOwn;
+    RCD_CUDA(ctx, cudaMemsetAsync(ctx->statusOwn, 0, sizeof(int32_t), st));
     return launch_similarity(ctx, X_dev, dtype, M * batch, d, cls, S_dev, st);
 }
 
@@ -386,6 +396,7 @@ rcd_status rcd_partition(rcd_ctx *ctx, const void *features_dev, rcd_feat_dtype 
     cudaStream_t st = (cudaStream_t)cuda_stream;
     RCD_CUDA(ctx, cudaSetDevice(ctx->device));
     ctx->kernelLaunches = 0;
+    ctx->tcLaunches = 0;
     ctx->steps = 0;
     ctx->phaseValid = false;
     ctx->stepBytesDev = nullptr;

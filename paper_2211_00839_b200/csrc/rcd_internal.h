@@ -22,6 +22,7 @@ enum : int {
     kDevBadLabel = 1,          // a label outside [0, L)
     kDevNoCandidate = 2,       // a class had samples left but no block could take one
     kDevBadState = 4,          // internal consistency check failed
+    kDevTimeout = 8,           // a bounded wait inside a kernel ran out
 };
 
 // One class, as the kernels see it.  Built on the host once the class sizes are known.
@@ -116,6 +117,7 @@ struct rcd_ctx {
     rcd_config cfg{};
     std::string err;
     int32_t *hostStage = nullptr;       // pinned, counts / status read-back
+    int32_t *statusOwn = nullptr;       // device status word for calls that take no workspace
     size_t hostStageInts = 0;
     // profiling
     cudaEvent_t evPhase[5]{};           // start, after group, after similarity, after greedy, end
@@ -123,6 +125,7 @@ struct rcd_ctx {
     std::vector<cudaEvent_t> evSweep;   // 2 per step
     int64_t sweepEventsUsed = 0;
     int64_t kernelLaunches = 0;
+    int64_t tcLaunches = 0;
     int64_t steps = 0;
     const unsigned long long *stepBytesDev = nullptr;
     const unsigned long long *stepOpsDev = nullptr;

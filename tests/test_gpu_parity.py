@@ -54,7 +54,9 @@ def test_similarity_int8_exact(rcd, orc, M, d, batch, path):
     X = rng.integers(-128, 128, size=(batch, M, d)).astype(np.int8)
     with rcd.Context(0, similarity_path=path) as ctx:
         S = ctx.rcd_similarity(torch.from_numpy(X).cuda())
-        torch.cuda.synchronize()
+        ctx.sync_status()
+        # rows that are 16-byte multiples of at least 128 bytes must take the tensor-core kernel
+        assert ctx.profile()["similarity_tc_launches"] == (1 if path == 0 and d % 16 == 0 and d >= 128 else 0)
         S = S.cpu().numpy()
     ld = (M + 3) // 4 * 4
     assert S.shape == (batch, M, ld)
@@ -75,7 +77,8 @@ def test_similarity_bf16_close(rcd, orc, M, d, batch, path):
     bits = fp32_to_bf16_bits(x)
     with rcd.Context(0, similarity_path=path) as ctx:
         S = ctx.rcd_similarity(rcd.features_to_torch(bits.reshape(batch * M, d)).view(batch, M, d).cuda())
-        torch.cuda.synchronize()
+        ctx.sync_status()
+        assert ctx.profile()["similarity_tc_launches"] == (1 if path == 0 and (2 * d) % 16 == 0 and 2 * d >= 128 else 0)
         S = S.cpu().numpy()
     for b in range(batch):
         want = orc.similarity(bits[b])
