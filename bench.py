@@ -242,11 +242,11 @@ def run_ours(args):
     # roofline of the dominant kernel (the gain sweep): one extra pass with an event pair around
     # every sweep launch; algorithmic bytes = rows of S of the unassigned samples + the coverage
     # vectors of the blocks refreshed, as scheduled on the device
+    peaks = load_peaks()
     ctx2 = rcd.Context(local, sweep_batch_max=args.sweep_batch, profile=2)
     ctx2.rcd_partition(Xd, yd, wl.capacities, wl.L, M_max=M)
     ctx2.sync_status()
     p2 = ctx2.profile()
-    peaks = load_peaks()
     sweep_s = p2["sweep_ms"] * 1e-3
     achieved = p2["sweep_bytes"] / sweep_s / 1e9 if sweep_s > 0 else 0.0
     roofline = {"bound": "hbm", "kernel": "sweep_kernel", "achieved": achieved, "peak": peaks["hbm_gbs"],
@@ -257,10 +257,19 @@ def run_ours(args):
                 "bytes_per_launch": p2["sweep_bytes"] / max(1, p2["sweep_launches"]),
                 "elem_block_ops_per_s": p2["sweep_elem_ops"] / sweep_s if sweep_s > 0 else 0.0,
                 "sweep_share_of_step": p2["sweep_ms"] / p2["total_ms"] if p2["total_ms"] > 0 else None}
+    # similarity GEMM: a dense contraction on the tensor cores.  Peak for its dtype: the measured bf16
+    # cuBLAS peak, times 2 for int8 (nominal int8 : bf16 ratio of the part); it also has to write 4*M^2
+    # bytes per class, which is the tighter bound at d = 512.
     sim_flops = 2.0 * wl.L * M * M * wl.d
     sim_s = prof["similarity_ms"] * 1e-3
-    similarity = {"ms": prof["similarity_ms"], "tflops": sim_flops / sim_s / 1e12 if sim_s > 0 else None,
-                  "bytes_written_gbs": 4.0 * wl.L * M * M / sim_s / 1e9 if sim_s > 0 else None}
+    tensor_peak = peaks["bf16_tflops"] * (2.0 if wl.dtype == "int8" else 1.0)
+    sim_tflops = sim_flops / sim_s / 1e12 if sim_s > 0 else None
+    sim_gbs = 4.0 * wl.L * M * M / sim_s / 1e9 if sim_s > 0 else None
+    similarity = {"ms": prof["similarity_ms"], "tensor_core_launches": int(prof["similarity_tc_launches"]),
+                  "tflops": sim_tflops, "tensor_peak_tflops": tensor_peak,
+                  "frac_of_tensor_peak": sim_tflops / tensor_peak if sim_tflops else None,
+                  "bytes_written_gbs": sim_gbs, "frac_of_hbm_peak": sim_gbs / peaks["hbm_gbs"] if sim_gbs else None,
+                  "peak_source": peaks["source"] + (" bf16 x2 (nominal int8:bf16 ratio)" if wl.dtype == "int8" else " bf16")}
 
     result = {"metric": "samples partitioned/sec", "value": value, "unit": "samples/s", "n_gpus": world,
               "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps,
