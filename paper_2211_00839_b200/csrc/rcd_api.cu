@@ -57,6 +57,7 @@ size_t layout_workspace(void *base, rcd_feat_dtype dtype, const Sizes &sz, Works
     w.nSweep = c.take<int32_t>(4);
     // everything below is placed once the class sizes are known
     w.desc = c.take<ClassDesc>(L);
+    w.tilePrefix = c.take<int32_t>(L + 1);
     w.chunkHist = c.take<int32_t>((size_t)std::max<int32_t>(sz.nChunks, 1) * L);
     w.perm = c.take<int32_t>(N);
     w.Xs = c.take<unsigned char>(N * (size_t)sz.d * feat_bytes(dtype));
@@ -219,7 +220,20 @@ static rcd_status prepare(rcd_ctx *ctx, const void *features, rcd_feat_dtype dty
     cls.src.table = P.ws.desc;
     cls.L = L;
     cls.maxM = maxM;
-    for (const auto &c : P.desc) cls.tiles128 += (int64_t)((c.M + 127) / 128) * ((c.M + 127) / 128);
+    {
+        std::vector<int32_t> prefix((size_t)L + 1);
+        int64_t run = 0;
+        for (int32_t l = 0; l < L; ++l) {
+            prefix[(size_t)l] = (int32_t)run;
+            const int64_t nt = (P.desc[(size_t)l].M + 127) / 128;
+            run += nt * (nt + 1) / 2;
+            if (run > 0x7fffffffLL) return fail(ctx, RCD_ERR_UNSUPPORTED, "too many similarity tiles");
+        }
+        prefix[(size_t)L] = (int32_t)run;
+        cls.upperTiles = run;
+        cls.tilePrefixDev = P.ws.tilePrefix;
+        RCD_CUDA(ctx, cudaMemcpyAsync(P.ws.tilePrefix, prefix.data(), prefix.size() * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+    }
     rs = launch_similarity(ctx, P.ws.Xs, dtype, N, d, cls, P.ws.S, st);
     if (rs != RCD_OK) return rs;
     if (ctx->cfg.profile >= 1) RCD_CUDA(ctx, cudaEventRecord(ctx->evPhase[2], st));
@@ -363,7 +377,9 @@ rcd_status rcd_similarity(rcd_ctx *ctx, const void *X_dev, rcd_feat_dtype dtype,
     cls.src.uniLd = (int32_t)ldS;
     cls.L = (int32_t)batch;
     cls.maxM = M;
-    cls.tiles128 = batch * ((M + 127) / 128) * ((M + 127) / 128);
+    cls.tilePrefixDev = nullptr;
+    cls.uniTiles = (int32_t)(((M + 127) / 128) * ((M + 127) / 128 + 1) / 2);
+    cls.upperTiles = batch * (int64_t)cls.uniTiles;
     ctx->kernelLaunches = 0;
     ctx->tcLaunches = 0;
     ctx->statusDev = ctx->statusOwn;

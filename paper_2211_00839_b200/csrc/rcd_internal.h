@@ -55,7 +55,10 @@ struct SimClasses {
     DescSource src;
     int32_t L;
     int64_t maxM;
-    int64_t tiles128;       // sum over classes of ceil(M/128)^2 (tensor-core tile count)
+    // tensor-core kernel: 128 x 128 tiles on or above the diagonal, listed class after class
+    const int32_t *tilePrefixDev;   // [L+1] first tile index of every class (null: equal classes)
+    int32_t uniTiles;               // tiles per class when the classes are equal
+    int64_t upperTiles;             // tiles in all
 };
 
 // Pointers into the caller's workspace for one rcd_partition call.
@@ -67,6 +70,7 @@ struct Workspace {
     void *Xs;               // [N][d] features in class-sorted order
     // per class
     ClassDesc *desc;        // [L]
+    int32_t *tilePrefix;    // [L+1] first upper-triangle tile of every class (tensor-core similarity)
     void *S;                // similarity matrices
     void *cover;            // [sum W*ld] coverage vectors (int32 / float)
     void *gains;            // [sum W*ld] stored gains (int64 / float)

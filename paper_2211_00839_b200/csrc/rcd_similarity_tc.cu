@@ -1,12 +1,15 @@
 // Tensor-core similarity kernel for sm_100a:  S_l = X_l X_l^T  per class (Section 3.1: similarities
 // from the feature vectors; int8 -> int32 exact, bf16 -> fp32).
 //
-// One CTA computes one 128 x 128 tile of one class.  Both operands are rows of the class-sorted
-// feature matrix (K-major), brought in 128-byte k-slabs by TMA (cp.async.bulk.tensor, 128-byte
-// swizzle, out-of-range rows and columns filled with zeros) into a 2-stage shared-memory ring;
-// one thread issues tcgen05.mma (kind::i8 or kind::f16 with bf16 inputs) with the accumulator in
-// tensor memory; four warps read the accumulator back with tcgen05.ld, transpose 32 x 32 blocks
-// through shared memory and write S with coalesced 128-bit stores (pad columns as zeros).
+// Persistent CTAs (one per SM) walk the 128 x 128 tiles on or above the diagonal of every class;
+// S is symmetric, so each off-diagonal tile is computed once and written twice (itself and its
+// mirror image), which halves the tensor work and the operand traffic.  Both operands are rows of
+// the class-sorted feature matrix (K-major), brought in 128-byte k-slabs by TMA (cp.async.bulk.tensor,
+// 128-byte swizzle, out-of-range rows and columns filled with zeros) into a 4-stage shared-memory
+// ring; one thread issues tcgen05.mma (kind::i8, or kind::f16 with bf16 inputs) into one of two
+// accumulator buffers in tensor memory, so the next tile's MMAs run while four warps read the
+// previous accumulator back with tcgen05.ld, transpose 32 x 32 blocks through shared memory and
+// write S with coalesced 128-bit stores (pad columns as zeros).
 //
 // Warp roles: 0 = TMA producer, 1 = TMEM allocation + MMA issue, 2..5 = epilogue.
 // Every wait on an mbarrier is bounded: on expiry the CTA records kDevTimeout in the status
@@ -23,17 +26,18 @@ namespace {
 constexpr int kTileM = 128;
 constexpr int kTileN = 128;
 constexpr int kSlabBytes = 128;                         // k-slab per stage and operand row
-constexpr int kStages = 2;                              // two CTAs per SM overlap each other's epilogue
+constexpr int kStages = 4;
 constexpr int kOperandBytes = kTileM * kSlabBytes;      // 16 KB
 constexpr int kStageBytes = 2 * kOperandBytes;          // A + B
 constexpr int kTcThreads = 192;
-constexpr int kTmemCols = 128;
+constexpr int kTmemCols = 256;                           // two accumulator buffers of 128 columns
 constexpr uint32_t kSpinLimit = 1u << 22;               // polls of ~64 ns: a quarter of a second
 
 struct __align__(8) TcShared {
     uint64_t full[kStages];
     uint64_t empty[kStages];
-    uint64_t accReady;
+    uint64_t accFull[2];
+    uint64_t accEmpty[2];
     uint32_t tmemBase;
     int32_t abort;
 };
@@ -121,9 +125,43 @@ __device__ __forceinline__ void tmem_load_32cols(uint32_t taddr, uint32_t (&v)[3
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" :: "r"(smem_addr(bar)) : "memory");
+}
+
+// Tile idx of the launch -> (class, row tile, column tile).  Only tiles on or above the diagonal
+// are listed (S is symmetric); a class with nt row tiles owns nt*(nt+1)/2 consecutive indices.
+struct TileCoord { int l, tm, tn; };
+__device__ __forceinline__ TileCoord decode_tile(const DescSource &src, const int32_t *__restrict__ prefix, int L, int uniTiles, int idx)
+{
+    TileCoord t;
+    int local;
+    if (prefix) {
+        int lo = 0, hi = L;                              // prefix[lo] <= idx < prefix[hi]
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (prefix[mid] <= idx) lo = mid; else hi = mid;
+        }
+        t.l = lo;
+        local = idx - prefix[lo];
+    } else {
+        t.l = idx / uniTiles;
+        local = idx - t.l * uniTiles;
+    }
+    const ClassDesc c = src.get(t.l);
+    int rowLen = (c.M + kTileM - 1) / kTileM;
+    t.tm = 0;
+    while (local >= rowLen) { local -= rowLen; --rowLen; ++t.tm; }
+    t.tn = t.tm + local;
+    return t;
+}
+
 template <bool kInt8>
-__global__ void __launch_bounds__(kTcThreads, 2) sim_tc_kernel(const __grid_constant__ CUtensorMap map, DescSource src, int32_t L,
-                                                              int32_t numSlabs, uint32_t *__restrict__ S, int32_t *status)
+__global__ void __launch_bounds__(kTcThreads, 1) sim_tc_kernel(const __grid_constant__ CUtensorMap map, DescSource src, int32_t L,
+                                                              const int32_t *__restrict__ tilePrefix, int32_t uniTiles,
+                                                              int32_t totalTiles, int32_t numSlabs, uint32_t *__restrict__ S,
+                                                              int32_t *status)
 {
     extern __shared__ unsigned char smemRaw[];
     // operand stages need 1024-byte alignment for the 128-byte swizzle pattern
@@ -133,119 +171,153 @@ __global__ void __launch_bounds__(kTcThreads, 2) sim_tc_kernel(const __grid_cons
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
-    {
-        const int l = blockIdx.z;                        // one tile per CTA; the launcher keeps L <= 65535
-        if (l >= L) return;
-        const ClassDesc c = src.get(l);
-        const int tilesM = (c.M + kTileM - 1) / kTileM;
-        const int tilesN = (c.ld + kTileN - 1) / kTileN;
-        if ((int)blockIdx.y >= tilesM || (int)blockIdx.x >= tilesN) return;       // uniform for the CTA
-        const int rowA = blockIdx.y * kTileM, rowB = blockIdx.x * kTileN;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(&sh.accFull[b], 1); mbar_init(&sh.accEmpty[b], 4); }
+        sh.abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" :: "r"(smem_addr(&sh.tmemBase)), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmemBase = sh.tmemBase;
 
-        if (threadIdx.x == 0) {
-            for (int s = 0; s < kStages; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], 1); }
-            mbar_init(&sh.accReady, 1);
-            sh.abort = 0;
-            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        }
-        if (warp == 1) {
-            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" :: "r"(smem_addr(&sh.tmemBase)), "r"(kTmemCols) : "memory");
-            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-        }
-        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-        __syncthreads();
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const uint32_t tmemD = sh.tmemBase;
-
-        if (warp == 0) {
-            // ---------------- TMA producer ----------------
-            if (lane == 0) {
-                int issued = 0;
-                for (int kb = 0; kb < numSlabs; ++kb) {
-                    const int s = kb % kStages;
-                    const uint32_t round = (uint32_t)(kb / kStages);
-                    if (!mbar_wait(&sh.empty[s], (round & 1) ^ 1, &sh)) break;
+    if (warp == 0) {
+        // ---------------- TMA producer ----------------
+        if (lane == 0) {
+            uint32_t it = 0;                             // k-slabs issued so far, over all tiles
+            bool ok = true;
+            for (int idx = blockIdx.x; idx < totalTiles && ok; idx += gridDim.x) {
+                const TileCoord t = decode_tile(src, tilePrefix, L, uniTiles, idx);
+                const ClassDesc c = src.get(t.l);
+                const int rowA = c.row0 + t.tm * kTileM, rowB = c.row0 + t.tn * kTileN;
+                const bool diag = (t.tm == t.tn);        // A and B are the same rows: one copy serves both
+                for (int kb = 0; kb < numSlabs; ++kb, ++it) {
+                    const int s = it % kStages;
+                    if (!mbar_wait(&sh.empty[s], ((it / kStages) & 1) ^ 1, &sh)) { ok = false; break; }
                     unsigned char *a = tiles + (size_t)s * kStageBytes;
-                    mbar_expect_tx(&sh.full[s], kStageBytes);
+                    mbar_expect_tx(&sh.full[s], diag ? kOperandBytes : kStageBytes);
                     const int k0 = kb * (kInt8 ? kSlabBytes : kSlabBytes / 2);         // element coordinate
-                    tma_load_2d(a, &map, k0, c.row0 + rowA, &sh.full[s]);
-                    tma_load_2d(a + kOperandBytes, &map, k0, c.row0 + rowB, &sh.full[s]);
-                    issued = kb + 1;
-                }
-                // after an abort: let the copies already issued land before the CTA leaves
-                if (*(volatile int32_t *)&sh.abort) {
-                    for (int kb = (issued > kStages ? issued - kStages : 0); kb < issued; ++kb) {
-                        const int s = kb % kStages;
-                        for (uint32_t spin = 0; spin < kSpinLimit && !mbar_test(&sh.full[s], (uint32_t)(kb / kStages) & 1); ++spin) __nanosleep(64);
-                    }
+                    tma_load_2d(a, &map, k0, rowA, &sh.full[s]);
+                    if (!diag) tma_load_2d(a + kOperandBytes, &map, k0, rowB, &sh.full[s]);
                 }
             }
-        } else if (warp == 1) {
-            // ---------------- MMA issuer ----------------
-            if (lane == 0) {
-                // instruction descriptor: D format, A/B format, K-major operands, N and M of the tile
-                const uint32_t idesc = (kInt8 ? (2u << 4) | (1u << 7) | (1u << 10)       // S32 accumulate, S8 x S8
-                                              : (1u << 4) | (1u << 7) | (1u << 10))      // F32 accumulate, BF16 x BF16
-                                       | ((uint32_t)(kTileN >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
-                bool ok = true;
-                for (int kb = 0; kb < numSlabs && ok; ++kb) {
-                    const int s = kb % kStages;
-                    const uint32_t round = (uint32_t)(kb / kStages);
-                    ok = mbar_wait(&sh.full[s], round & 1, &sh);
-                    if (!ok) break;
+            // after an abort: let the copies already issued land before the CTA leaves
+            if (*(volatile int32_t *)&sh.abort) {
+                for (uint32_t k = (it > (uint32_t)kStages ? it - kStages : 0); k < it; ++k) {
+                    const int s = k % kStages;
+                    for (uint32_t spin = 0; spin < kSpinLimit && !mbar_test(&sh.full[s], (k / kStages) & 1); ++spin) __nanosleep(64);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer ----------------
+        if (lane == 0) {
+            // instruction descriptor: D format, A/B format, K-major operands, N and M of the tile
+            const uint32_t idesc = (kInt8 ? (2u << 4) | (1u << 7) | (1u << 10)       // S32 accumulate, S8 x S8
+                                          : (1u << 4) | (1u << 7) | (1u << 10))      // F32 accumulate, BF16 x BF16
+                                   | ((uint32_t)(kTileN >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
+            uint32_t it = 0, nt = 0;
+            bool ok = true;
+            for (int idx = blockIdx.x; idx < totalTiles && ok; idx += gridDim.x, ++nt) {
+                const TileCoord t = decode_tile(src, tilePrefix, L, uniTiles, idx);
+                const bool diag = (t.tm == t.tn);
+                const uint32_t buf = nt & 1;
+                // the epilogue must have drained this accumulator buffer (two tiles ago)
+                if (!mbar_wait(&sh.accEmpty[buf], ((nt >> 1) & 1) ^ 1, &sh)) { ok = false; break; }
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t tmemD = tmemBase + buf * kTileN;
+                for (int kb = 0; kb < numSlabs; ++kb, ++it) {
+                    const int s = it % kStages;
+                    if (!mbar_wait(&sh.full[s], (it / kStages) & 1, &sh)) { ok = false; break; }
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const uint32_t aAddr = smem_addr(tiles + (size_t)s * kStageBytes);
                     const uint64_t descA = make_smem_desc(aAddr);
-                    const uint64_t descB = make_smem_desc(aAddr + kOperandBytes);
+                    const uint64_t descB = diag ? descA : make_smem_desc(aAddr + kOperandBytes);
 #pragma unroll
                     for (int k = 0; k < kSlabBytes / 32; ++k)          // one MMA consumes 32 bytes of k per row
                         mma_issue<kInt8>(tmemD, descA + (uint64_t)(2 * k), descB + (uint64_t)(2 * k), idesc, (kb > 0 || k > 0) ? 1u : 0u);
                     mma_commit(&sh.empty[s]);                          // frees the stage when those MMAs retire
                 }
-                mma_commit(&sh.accReady);                              // accumulator complete (or abandoned)
+                mma_commit(&sh.accFull[buf]);                          // accumulator complete (or abandoned)
             }
-        } else {
-            // ---------------- epilogue: TMEM -> registers -> shared (transpose) -> global ----------------
-            const int q = warp & 3;                                    // TMEM lane quarter this warp may read
-            const bool ready = mbar_wait(&sh.accReady, 0, &sh);
+        }
+    } else {
+        // ---------------- epilogue: TMEM -> registers -> shared (transpose) -> global ----------------
+        const int q = warp & 3;                                        // TMEM lane quarter this warp may read
+        const int ew = warp - 2;
+        uint32_t nt = 0;
+        for (int idx = blockIdx.x; idx < totalTiles; idx += gridDim.x, ++nt) {
+            const TileCoord t = decode_tile(src, tilePrefix, L, uniTiles, idx);
+            const ClassDesc c = src.get(t.l);
+            const int rowA = t.tm * kTileM, rowB = t.tn * kTileN;      // class-local
+            const bool diag = (t.tm == t.tn);
+            const uint32_t buf = nt & 1;
+            if (!mbar_wait(&sh.accFull[buf], (nt >> 1) & 1, &sh)) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            if (ready && !*(volatile int32_t *)&sh.abort) {
-                uint32_t *Sl = S + c.sOff;
-                const int ew = warp - 2;
+            if (*(volatile int32_t *)&sh.abort) break;
+            uint32_t *Sl = S + c.sOff;
+            const int cg = (lane & 7) * 4;                             // this lane's 4 columns of a 32-wide block
 #pragma unroll 1
-                for (int cb = 0; cb < kTileN / 32; ++cb) {
-                    uint32_t v[32];
-                    tmem_load_32cols(tmemD + ((uint32_t)(q * 32) << 16) + (uint32_t)(cb * 32), v);
+            for (int cb = 0; cb < kTileN / 32; ++cb) {
+                uint32_t v[32];
+                tmem_load_32cols(tmemBase + buf * kTileN + ((uint32_t)(q * 32) << 16) + (uint32_t)(cb * 32), v);
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) stage32[ew][lane][j] = v[j];     // lane = row inside the quarter
-                    __syncwarp();
-                    // 8 lanes cover the 32 columns of one row with 128-bit stores; 4 rows per pass
-                    const int colBase = rowB + cb * 32 + (lane & 7) * 4;
+                for (int j = 0; j < 32; ++j) stage32[ew][lane][j] = v[j];         // lane = row inside the quarter
+                __syncwarp();
+                // block rows -> S[rowA + ..][rowB + ..]: 8 lanes cover 32 columns with 128-bit stores, 4 rows per pass
+                {
+                    const int col = rowB + cb * 32 + cg;
 #pragma unroll
                     for (int pass = 0; pass < 8; ++pass) {
                         const int r = pass * 4 + (lane >> 3);
                         const int row = rowA + q * 32 + r;
-                        if (row < c.M && colBase < c.ld) {
+                        if (row < c.M && col < c.ld) {
                             uint4 o;
-                            o.x = colBase + 0 < c.M ? stage32[ew][r][(lane & 7) * 4 + 0] : 0u;
-                            o.y = colBase + 1 < c.M ? stage32[ew][r][(lane & 7) * 4 + 1] : 0u;
-                            o.z = colBase + 2 < c.M ? stage32[ew][r][(lane & 7) * 4 + 2] : 0u;
-                            o.w = colBase + 3 < c.M ? stage32[ew][r][(lane & 7) * 4 + 3] : 0u;
-                            *reinterpret_cast<uint4 *>(Sl + (int64_t)row * c.ld + colBase) = o;
+                            o.x = col + 0 < c.M ? stage32[ew][r][cg + 0] : 0u;
+                            o.y = col + 1 < c.M ? stage32[ew][r][cg + 1] : 0u;
+                            o.z = col + 2 < c.M ? stage32[ew][r][cg + 2] : 0u;
+                            o.w = col + 3 < c.M ? stage32[ew][r][cg + 3] : 0u;
+                            *reinterpret_cast<uint4 *>(Sl + (int64_t)row * c.ld + col) = o;
                         }
                     }
-                    __syncwarp();
                 }
+                // the mirrored block -> S[rowB + ..][rowA + ..] (tiles below the diagonal are never computed)
+                if (!diag) {
+                    const int col = rowA + q * 32 + cg;
+#pragma unroll
+                    for (int pass = 0; pass < 8; ++pass) {
+                        const int jj = pass * 4 + (lane >> 3);
+                        const int row = rowB + cb * 32 + jj;
+                        if (row < c.M && col < c.ld) {
+                            uint4 o;
+                            o.x = col + 0 < c.M ? stage32[ew][cg + 0][jj] : 0u;
+                            o.y = col + 1 < c.M ? stage32[ew][cg + 1][jj] : 0u;
+                            o.z = col + 2 < c.M ? stage32[ew][cg + 2][jj] : 0u;
+                            o.w = col + 3 < c.M ? stage32[ew][cg + 3][jj] : 0u;
+                            *reinterpret_cast<uint4 *>(Sl + (int64_t)row * c.ld + col) = o;
+                        }
+                    }
+                }
+                __syncwarp();
             }
+            // hand the accumulator buffer back to the MMA warp
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sh.accEmpty[buf]);
         }
-        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-        __syncthreads();
-        if (warp == 1) {
-            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmemD), "r"(kTmemCols) : "memory");
-        }
-        if (threadIdx.x == 0 && sh.abort && status) atomicOr(status, kDevTimeout);
     }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 1) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmemBase), "r"(kTmemCols) : "memory");
+    }
+    if (threadIdx.x == 0 && sh.abort && status) atomicOr(status, kDevTimeout);
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
@@ -275,7 +347,6 @@ rcd_status launch_similarity_tc(rcd_ctx *ctx, const void *Xs, rcd_feat_dtype dty
     // TMA needs 16-byte row pitch and base; a row shorter than one 128-byte slab goes to the generic kernel
     if (rowBytes % 16 != 0 || rowBytes < kSlabBytes || ((uintptr_t)Xs) % 16 != 0 || ((uintptr_t)S) % 16 != 0) return RCD_OK;
     if (cls.L == 0 || cls.maxM == 0 || Ntot == 0) { *handled = true; return RCD_OK; }
-    if (cls.L > 65535) return RCD_OK;                   // grid.z limit: the generic kernel loops over classes
     EncodeTiledFn encode = encode_tiled_fn();
     if (!encode) return fail(ctx, RCD_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
 
@@ -291,15 +362,18 @@ rcd_status launch_similarity_tc(rcd_ctx *ctx, const void *Xs, rcd_feat_dtype dty
 
     const int numSlabs = (int)((rowBytes + kSlabBytes - 1) / kSlabBytes);
     const size_t smem = (size_t)kStages * kStageBytes + 1024;
-    const int maxLd = pad4(cls.maxM);
-    dim3 grid((maxLd + kTileN - 1) / kTileN, (int)((cls.maxM + kTileM - 1) / kTileM), cls.L);
+    if (cls.upperTiles <= 0 || cls.upperTiles > 0x7fffffffLL) return RCD_OK;
+    const int totalTiles = (int)cls.upperTiles;
+    const int grid = totalTiles < ctx->smCount ? totalTiles : ctx->smCount;
     int32_t *status = const_cast<int32_t *>(ctx->statusDev);
     if (dtype == RCD_FEAT_I8) {
         RCD_CUDA(ctx, cudaFuncSetAttribute(sim_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        sim_tc_kernel<true><<<grid, kTcThreads, smem, st>>>(map, cls.src, cls.L, numSlabs, (uint32_t *)S, status);
+        sim_tc_kernel<true><<<grid, kTcThreads, smem, st>>>(map, cls.src, cls.L, cls.tilePrefixDev, cls.uniTiles, totalTiles,
+                                                           numSlabs, (uint32_t *)S, status);
     } else {
         RCD_CUDA(ctx, cudaFuncSetAttribute(sim_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        sim_tc_kernel<false><<<grid, kTcThreads, smem, st>>>(map, cls.src, cls.L, numSlabs, (uint32_t *)S, status);
+        sim_tc_kernel<false><<<grid, kTcThreads, smem, st>>>(map, cls.src, cls.L, cls.tilePrefixDev, cls.uniTiles, totalTiles,
+                                                            numSlabs, (uint32_t *)S, status);
     }
     ctx->kernelLaunches++;
     ctx->tcLaunches++;
