@@ -175,7 +175,7 @@ def run_ours(args):
     Xh = rcd.features_to_torch(wl.features, pin=True)
     yh = torch.from_numpy(wl.labels).pin_memory()
     Xd, yd = Xh.to(dev), yh.to(dev)
-    ctx = rcd.Context(local, sweep_batch_max=args.sweep_batch, profile=1)
+    ctx = rcd.Context(local, sweep_batch_max=args.sweep_batch, profile=1, greedy_path=args.greedy_path)
 
     def barrier():
         torch.cuda.synchronize()
@@ -279,7 +279,8 @@ def run_ours(args):
                          "l2": "inputs larger than L2 (S is %.0f MB per class, re-read every sweep)" % (4e-6 * M * M),
                          "sweep_batch_max": args.sweep_batch or 8, "sharding": "one dataset per rank, no collective"},
               "gain_evals_per_s": world * wl.L * M * (M + 1) / 2 * args.steps / (ms * 1e-3),
-              "phases_ms": {k: prof[k] for k in ("group_ms", "similarity_ms", "greedy_ms", "total_ms")},
+              "phases_ms": dict({k: prof[k] for k in ("group_ms", "similarity_ms", "greedy_ms", "total_ms")},
+                                sweep_phases_ms=prof["persistent_sweep_ns"] * 1e-6, pick_phases_ms=prof["persistent_pick_ns"] * 1e-6),
               "similarity": similarity,
               "e2e": {"value": e2e_value, "unit": "samples/s", "h2d_bytes_per_step": int(h2d),
                       "d2h_bytes_per_step": int(d2h), "wall_ms_per_step": e2e_wall_ms / args.steps},
@@ -309,6 +310,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="C2", choices=["C1", "C2", "C3", "C4", "C5"])
     ap.add_argument("--sweep-batch", type=int, default=0, help="sweep_batch_max (0 = library default)")
+    ap.add_argument("--greedy-path", type=int, default=0, help="0 = one cooperative launch, 1 = two launches per round")
     ap.add_argument("--ref-picks", type=int, default=150, help="picks per class in the CPU-oracle sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

@@ -59,7 +59,9 @@ typedef struct {
     int32_t sweep_batch_max;   /* blocks whose gains one pass over S may refresh: 1,2,4 or 8; 0 = default (8) */
     int32_t similarity_path;   /* 0 = tensor-core kernel when the shape allows, 2 = always the generic kernel */
     int32_t profile;           /* 0 off; 1 time the phases of rcd_partition; 2 also time every sweep launch */
-    int32_t reserved[13];      /* must be 0 */
+    int32_t greedy_path;       /* 0 = whole greedy loop in one cooperative launch when the device allows;
+                                  1 = two launches per greedy step (always used with profile 2) */
+    int32_t reserved[12];      /* must be 0 */
 } rcd_config;
 
 /* Timings and counters of the last rcd_partition / rcd_partition_host on a context (profile >= 1). */
@@ -75,7 +77,9 @@ typedef struct {
     int64_t kernel_launches;   /* kernels this library launched during the call */
     int64_t steps;             /* greedy steps executed (= largest class size) */
     int64_t similarity_tc_launches; /* similarity launches of the last call that ran on the tensor cores */
-    int64_t reserved[5];
+    int64_t persistent_sweep_ns;    /* one-launch greedy loop: time in sweep phases (incl. their barrier) */
+    int64_t persistent_pick_ns;     /* one-launch greedy loop: time in pick phases (incl. their barrier) */
+    int64_t reserved[3];
 } rcd_profile;
 
 typedef struct rcd_ctx rcd_ctx;

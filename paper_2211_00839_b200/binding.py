@@ -41,14 +41,15 @@ class RcdError(RuntimeError):
 
 class RcdConfig(C.Structure):
     _fields_ = [("sweep_batch_max", C.c_int32), ("similarity_path", C.c_int32), ("profile", C.c_int32),
-                ("reserved", C.c_int32 * 13)]
+                ("greedy_path", C.c_int32), ("reserved", C.c_int32 * 12)]
 
 
 class RcdProfile(C.Structure):
     _fields_ = [("total_ms", C.c_double), ("group_ms", C.c_double), ("similarity_ms", C.c_double),
                 ("greedy_ms", C.c_double), ("sweep_ms", C.c_double), ("sweep_launches", C.c_int64),
                 ("sweep_bytes", C.c_int64), ("sweep_elem_ops", C.c_int64), ("kernel_launches", C.c_int64),
-                ("steps", C.c_int64), ("similarity_tc_launches", C.c_int64), ("reserved", C.c_int64 * 5)]
+                ("steps", C.c_int64), ("similarity_tc_launches", C.c_int64), ("persistent_sweep_ns", C.c_int64),
+                ("persistent_pick_ns", C.c_int64), ("reserved", C.c_int64 * 3)]
 
 
 def _load() -> C.CDLL:
@@ -132,7 +133,8 @@ def features_to_torch(features: np.ndarray, device=None, pin: bool = False):
 class Context:
     """Owns one ``rcd_ctx`` on a CUDA device."""
 
-    def __init__(self, device: int = 0, sweep_batch_max: int = 0, similarity_path: int = 0, profile: int = 0):
+    def __init__(self, device: int = 0, sweep_batch_max: int = 0, similarity_path: int = 0, profile: int = 0,
+                 greedy_path: int = 0):
         torch = _torch()
         if not torch.cuda.is_available():
             raise RcdError(4, "no CUDA device: this library has no CPU path")
@@ -142,6 +144,7 @@ class Context:
         cfg.sweep_batch_max = sweep_batch_max
         cfg.similarity_path = similarity_path
         cfg.profile = profile
+        cfg.greedy_path = greedy_path
         self._h = C.c_void_p()
         st = lib.rcd_create(C.byref(self._h), self.device, C.byref(cfg))
         if st != 0:

@@ -76,9 +76,10 @@ size_t layout_workspace(void *base, rcd_feat_dtype dtype, const Sizes &sz, Works
     w.sweepParts = c.take<int32_t>(L * kMaxSweepBatch);
     w.sweepCS = c.take<int32_t>(L);
     w.rowCtr = c.take<int32_t>(L);
-    w.sweepList = c.take<int32_t>(2 * L);
+    w.sweepList = c.take<int32_t>(3 * L);
     w.stepBytes = c.take<unsigned long long>((size_t)sz.maxM + 1);
     w.stepOps = c.take<unsigned long long>((size_t)sz.maxM + 1);
+    w.phaseNs = c.take<unsigned long long>(3);      // two phase clocks + the grid-barrier counter
     w.bytes = align_up(c.off);
     if (ws) *ws = w;
     return w.bytes;
@@ -260,7 +261,8 @@ rcd_status rcd_create(rcd_ctx **out, int cuda_device, const rcd_config *cfg)
             return RCD_ERR_INVALID_ARG;
         if (cfg->similarity_path != 0 && cfg->similarity_path != 2) return RCD_ERR_INVALID_ARG;
         if (cfg->profile < 0 || cfg->profile > 2) return RCD_ERR_INVALID_ARG;
-        for (int i = 0; i < 13; ++i) if (cfg->reserved[i] != 0) return RCD_ERR_INVALID_ARG;
+        if (cfg->greedy_path != 0 && cfg->greedy_path != 1) return RCD_ERR_INVALID_ARG;
+        for (int i = 0; i < 12; ++i) if (cfg->reserved[i] != 0) return RCD_ERR_INVALID_ARG;
     }
     int count = 0;
     if (cudaGetDeviceCount(&count) != cudaSuccess || cuda_device < 0 || cuda_device >= count) {
@@ -276,6 +278,7 @@ rcd_status rcd_create(rcd_ctx **out, int cuda_device, const rcd_config *cfg)
     ctx->device = cuda_device;
     ctx->smCount = prop.multiProcessorCount;
     ctx->maxSmemOptin = (int)prop.sharedMemPerBlockOptin;
+    ctx->cooperative = prop.cooperativeLaunch != 0;
     if (cfg) ctx->cfg = *cfg;
     ctx->hostStageInts = 1 << 20;
     if (cudaMallocHost((void **)&ctx->hostStage, (ctx->hostStageInts + 16) * sizeof(int32_t)) != cudaSuccess) {
@@ -331,6 +334,12 @@ rcd_status rcd_get_profile(rcd_ctx *ctx, rcd_profile *out)
     RCD_CUDA(ctx, cudaEventElapsedTime(&ms, ctx->evPhase[0], ctx->evPhase[1])); out->group_ms = ms;
     RCD_CUDA(ctx, cudaEventElapsedTime(&ms, ctx->evPhase[1], ctx->evPhase[2])); out->similarity_ms = ms;
     RCD_CUDA(ctx, cudaEventElapsedTime(&ms, ctx->evPhase[2], ctx->evPhase[3])); out->greedy_ms = ms;
+    if (ctx->phaseNsDev) {
+        unsigned long long ns[2] = {0, 0};
+        RCD_CUDA(ctx, cudaMemcpy(ns, ctx->phaseNsDev, sizeof ns, cudaMemcpyDeviceToHost));
+        out->persistent_sweep_ns = (int64_t)ns[0];
+        out->persistent_pick_ns = (int64_t)ns[1];
+    }
     if (ctx->stepBytesDev && ctx->steps > 0) {
         std::vector<unsigned long long> bytes((size_t)ctx->steps + 1), ops((size_t)ctx->steps + 1);
         RCD_CUDA(ctx, cudaMemcpy(bytes.data(), ctx->stepBytesDev, bytes.size() * sizeof(unsigned long long), cudaMemcpyDeviceToHost));
@@ -417,6 +426,7 @@ rcd_status rcd_partition(rcd_ctx *ctx, const void *features_dev, rcd_feat_dtype 
     ctx->phaseValid = false;
     ctx->stepBytesDev = nullptr;
     ctx->stepOpsDev = nullptr;
+    ctx->phaseNsDev = nullptr;
     ctx->sweepEventsUsed = 0;
     const bool prof = ctx->cfg.profile >= 1;
     if (prof) RCD_CUDA(ctx, cudaEventRecord(ctx->evPhase[0], st));

@@ -59,6 +59,8 @@ struct GreedyParams {
     int32_t *nSweep;
     unsigned long long *stepBytes;
     unsigned long long *stepOps;
+    unsigned long long *phaseNs;    // [2] time block 0 spent in sweep phases / pick phases (persistent kernel)
+    unsigned *barrier;              // arrival counter of the persistent kernel's grid barrier
     int32_t *status;
     const int32_t *perm;
     int32_t *assignment;
@@ -74,36 +76,45 @@ struct GreedyParams {
 __host__ __device__ inline int rows_per_group(int P) { return P == 8 ? 4 : 8; }
 
 // ---------------------------------------------------------------------------------------------
-// Choice of the next block and of the blocks the next sweep refreshes.  Called by every thread of
-// the class's CTA after a __syncthreads(); the block values and flags are staged in shared memory
-// once, then warp 0 decides.
+// Choice of the next block and of the blocks the next sweep refreshes.  The class's block values
+// and flags live in shared memory while its CTA works on it (plan_load), so a chain of picks
+// re-reads nothing from global memory; plan_decide is run by warp 0.
 constexpr int kMaxBlocks = 1024;
 template <typename FV>
 struct PlanShared {
-    FV f[kMaxBlocks];
+    FV f[kMaxBlocks];              // tracked f of every block
+    int32_t room[kMaxBlocks];      // quota - count
     uint8_t open[kMaxBlocks];      // bit 0: block is not full, bit 1: its stored gains are out of date
+    int32_t nextJ;                 // plan_decide's answer: block of the next pick (-1: none)
+    int32_t needSweep;             //                       1 = that pick must wait for a sweep
 };
 
 template <typename SV>
-__device__ void plan_next(const GreedyParams<SV> &prm, int l, int nextStep, PlanShared<typename Arith<SV>::FV> &sh)
+__device__ __forceinline__ void plan_load(const GreedyParams<SV> &prm, int l, PlanShared<typename Arith<SV>::FV> &sh)
+{
+    const int W = prm.W;
+    for (int p = threadIdx.x; p < W; p += blockDim.x) {
+        const int64_t at = (int64_t)l * W + p;
+        const int room = prm.quota[at] - prm.cnt[at];
+        sh.f[p] = prm.fval[at];
+        sh.room[p] = room;
+        sh.open[p] = (uint8_t)((room > 0 ? 1 : 0) | (prm.valid[at] ? 0 : 2));
+    }
+}
+
+// Warp 0 only.  nR = samples of the class still unassigned.
+template <typename SV>
+__device__ void plan_decide(const GreedyParams<SV> &prm, int l, const ClassDesc &c, int nR, int nextStep,
+                            PlanShared<typename Arith<SV>::FV> &sh)
 {
     using FV = typename Arith<SV>::FV;
     const int lane = threadIdx.x & 31;
     const int W = prm.W;
-    const int nR = prm.nR[l];
     uint8_t *valid = prm.valid + (int64_t)l * W;
     if (nR == 0) {
-        if (threadIdx.x == 0) { prm.jstar[l] = -1; prm.sweepN[l] = 0; }
+        if (lane == 0) { prm.jstar[l] = -1; prm.sweepN[l] = 0; sh.nextJ = -1; sh.needSweep = 0; }
         return;
     }
-    for (int p = threadIdx.x; p < W; p += blockDim.x) {
-        const int64_t at = (int64_t)l * W + p;
-        sh.f[p] = prm.fval[at];
-        sh.open[p] = (uint8_t)((prm.cnt[at] < prm.quota[at] ? 1 : 0) | (valid[p] ? 0 : 2));
-    }
-    __syncthreads();
-    if ((threadIdx.x >> 5) != 0) return;
-    const ClassDesc c = prm.desc[l];
 
     // j* = argmin over non-full blocks of f, ties -> lowest index
     FV bestF = 0;
@@ -124,12 +135,15 @@ __device__ void plan_next(const GreedyParams<SV> &prm, int l, int nextStep, Plan
         if (oP != INT_MAX && (bestP == INT_MAX || oF < bestF || (oF == bestF && oP < bestP))) { bestF = oF; bestP = oP; }
     }
     if (bestP == INT_MAX) {
-        if (lane == 0) { prm.jstar[l] = -1; prm.sweepN[l] = 0; atomicOr(prm.status, kDevNoCandidate); }
+        if (lane == 0) {
+            prm.jstar[l] = -1; prm.sweepN[l] = 0; sh.nextJ = -1; sh.needSweep = 0;
+            atomicOr(prm.status, kDevNoCandidate);
+        }
         return;
     }
     const int jstar = bestP;
     if (!(sh.open[jstar] & 2)) {
-        if (lane == 0) { prm.jstar[l] = jstar; prm.sweepN[l] = 0; }
+        if (lane == 0) { prm.jstar[l] = jstar; prm.sweepN[l] = 0; sh.nextJ = jstar; sh.needSweep = 0; }
         return;
     }
     // how many blocks one pass can refresh: bounded by the configuration, by the shared memory
@@ -172,11 +186,13 @@ __device__ void plan_next(const GreedyParams<SV> &prm, int l, int nextStep, Plan
     int CS = 1;
     while (CS < 16 && 2 * CS <= chunks && 2 * CS * together * nGroups <= prm.sweepWarps) CS *= 2;
     if (lane == 0) {
+        sh.nextJ = jstar;
+        sh.needSweep = 1;
         prm.jstar[l] = jstar;
         prm.sweepN[l] = P;
         prm.sweepCS[l] = CS;
         prm.rowCtr[l] = 0;
-        int par = nextStep & 1;
+        int par = nextStep % 3;
         int slot = atomicAdd(&prm.nSweep[par], 1);
         prm.sweepList[(int64_t)par * prm.L + slot] = l;
         atomicAdd(&prm.stepBytes[nextStep], (unsigned long long)((int64_t)nR * c.ld + (int64_t)n * c.ld) * sizeof(SV));
@@ -204,9 +220,14 @@ __global__ void __launch_bounds__(kSelectThreads, 4) init_kernel(GreedyParams<SV
         prm.fval[(int64_t)l * W + p] = (FV)0;
         prm.valid[(int64_t)l * W + p] = 0;
     }
-    if (threadIdx.x == 0) prm.nR[l] = c.M;
+    if (threadIdx.x == 0) {
+        prm.nR[l] = c.M;
+        if (c.M > 0) atomicAdd(&prm.nSweep[3], 1);         // classes still to finish
+    }
     __syncthreads();
-    plan_next(prm, l, 0, shPlan);
+    plan_load(prm, l, shPlan);
+    __syncthreads();
+    if (threadIdx.x < 32) plan_decide(prm, l, c, c.M, 0, shPlan);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -450,21 +471,21 @@ __device__ __forceinline__ void sweep_class(const GreedyParams<SV> &prm, int l, 
     }
 }
 
+// The sweep of greedy step `step`, run by every CTA of the launch (kSweepThreads threads each).
 template <typename SV>
-__global__ void __launch_bounds__(kSweepThreads, 1) sweep_kernel(GreedyParams<SV> prm, int step)
+__device__ __forceinline__ void sweep_step(const GreedyParams<SV> &prm, int step, int4 *shCover)
 {
     using GV = typename Arith<SV>::GV;
-    extern __shared__ int4 shCover[];
     __shared__ long long shF[kMaxSweepBatch];
     __shared__ int32_t shParts[kMaxSweepBatch];
     __shared__ int shTicket[kSweepThreads / 32];
     __shared__ GV shPart[kSweepThreads];
     __shared__ int shGo;
-    cudaGridDependencySynchronize();              // the previous launch (select / init) has finished
-    cudaTriggerProgrammaticLaunchCompletion();
-    const int par = step & 1;
+    // three lists in rotation: this step reads list step%3, its picks fill (step+1)%3, and the one
+    // after that is cleared here, a full step (and at least one barrier / launch boundary) before use
+    const int par = step % 3;
     const int nS = prm.nSweep[par];
-    if (blockIdx.x == 0 && threadIdx.x == 0) prm.nSweep[par ^ 1] = 0;   // list the coming select fills
+    if (blockIdx.x == 0 && threadIdx.x == 0) prm.nSweep[(step + 2) % 3] = 0;
     if (nS == 0) return;
     const int start = (int)(((int64_t)blockIdx.x * nS) / gridDim.x);
     for (int k = 0; k < nS; ++k) {
@@ -504,9 +525,24 @@ __global__ void __launch_bounds__(kSweepThreads, 1) sweep_kernel(GreedyParams<SV
     }
 }
 
-// ---------------------------------------------------------------------------------------------
 template <typename SV>
-__global__ void __launch_bounds__(kSelectThreads, 2) select_kernel(GreedyParams<SV> prm, int step)
+__global__ void __launch_bounds__(kSweepThreads, 1) sweep_kernel(GreedyParams<SV> prm, int step)
+{
+    extern __shared__ int4 shCover[];
+    cudaGridDependencySynchronize();              // the previous launch (select / init) has finished
+    cudaTriggerProgrammaticLaunchCompletion();
+    sweep_step(prm, step, shCover);
+}
+
+// ---------------------------------------------------------------------------------------------
+// The picks of class l in round `round`, by one CTA of kSelectThreads threads: pick after pick
+// (GreedyStep's argmax over the stored gains of the chosen block, then the bookkeeping of
+// Algorithm 1's "A := A u {v*}, R := R \ {v*}" and the choice of the next block) until the next
+// block's stored gains are out of date -- then a sweep is scheduled for round + 1 -- or the class
+// is finished.  Inside the chain nothing waits on the coverage update: a pick only needs stored
+// gains, so row v* is folded into the coverage vector while the next block is being chosen.
+template <typename SV>
+__device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, int round)
 {
     using GV = typename Arith<SV>::GV;
     using FV = typename Arith<SV>::FV;
@@ -514,77 +550,86 @@ __global__ void __launch_bounds__(kSelectThreads, 2) select_kernel(GreedyParams<
     __shared__ GV shG[kSelectThreads / 32];
     __shared__ int shV[kSelectThreads / 32];
     __shared__ int shPick;
-    cudaGridDependencySynchronize();              // the sweep of this step has finished
-    cudaTriggerProgrammaticLaunchCompletion();
-    const int l = blockIdx.x;
-    const int nR = prm.nR[l];
+    int nR = prm.nR[l];
     if (nR == 0) return;
-    const int j = prm.jstar[l];
+    int j = prm.jstar[l];
     if (j < 0) return;
     const ClassDesc c = prm.desc[l];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int ld4 = c.ld >> 2;
     int32_t *cand = prm.cand + c.row0;
     int32_t *pos = prm.pos + c.row0;
-    const GV *G = prm.gains + c.vOff + (int64_t)j * c.ld;
-    const int lastV = cand[nR - 1];               // needed by the removal below; fetched early
-
-    // v* = argmax over the unassigned samples, ties -> lowest class-local index (GreedyStep).
-    // Walks all samples with independent, coalesced loads (pos[v] < 0 marks an assigned sample).
-    GV bestG = 0;
-    int bestV = INT_MAX;
-#pragma unroll 4
-    for (int v = threadIdx.x; v < c.M; v += kSelectThreads) {
-        const GV g = G[v];
-        const int ps = pos[v];
-        if (ps >= 0 && (bestV == INT_MAX || g > bestG)) { bestG = g; bestV = v; }
-    }
-    for (int off = 16; off > 0; off >>= 1) {
-        GV oG = __shfl_xor_sync(0xffffffffu, bestG, off);
-        int oV = __shfl_xor_sync(0xffffffffu, bestV, off);
-        if (oV != INT_MAX && (bestV == INT_MAX || oG > bestG || (oG == bestG && oV < bestV))) { bestG = oG; bestV = oV; }
-    }
-    if (lane == 0) { shG[warp] = bestG; shV[warp] = bestV; }
+    plan_load(prm, l, shPlan);
     __syncthreads();
-    if (warp == 0) {
-        bestG = lane < kSelectThreads / 32 ? shG[lane] : (GV)0;
-        bestV = lane < kSelectThreads / 32 ? shV[lane] : INT_MAX;
+
+    for (;;) {
+        const GV *G = prm.gains + c.vOff + (int64_t)j * c.ld;
+        // v* = argmax over the unassigned samples, ties -> lowest class-local index.  Walks all
+        // samples with independent, coalesced loads (pos[v] < 0 marks an assigned sample).
+        GV bestG = 0;
+        int bestV = INT_MAX;
+#pragma unroll 4
+        for (int v = threadIdx.x; v < c.M; v += kSelectThreads) {
+            const GV g = G[v];
+            const int ps = pos[v];
+            if (ps >= 0 && (bestV == INT_MAX || g > bestG)) { bestG = g; bestV = v; }
+        }
         for (int off = 16; off > 0; off >>= 1) {
             GV oG = __shfl_xor_sync(0xffffffffu, bestG, off);
             int oV = __shfl_xor_sync(0xffffffffu, bestV, off);
             if (oV != INT_MAX && (bestV == INT_MAX || oG > bestG || (oG == bestG && oV < bestV))) { bestG = oG; bestV = oV; }
         }
-        if (lane == 0) {
-            shPick = bestV;
-            shG[0] = bestG;
+        if (lane == 0) { shG[warp] = bestG; shV[warp] = bestV; }
+        __syncthreads();
+        if (warp == 0) {
+            bestG = lane < kSelectThreads / 32 ? shG[lane] : (GV)0;
+            bestV = lane < kSelectThreads / 32 ? shV[lane] : INT_MAX;
+            for (int off = 16; off > 0; off >>= 1) {
+                GV oG = __shfl_xor_sync(0xffffffffu, bestG, off);
+                int oV = __shfl_xor_sync(0xffffffffu, bestV, off);
+                if (oV != INT_MAX && (bestV == INT_MAX || oG > bestG || (oG == bestG && oV < bestV))) { bestG = oG; bestV = oV; }
+            }
+            if (lane == 0) {
+                shPick = bestV;
+                // block j has received a sample: value, room, and its stored gains are now out of date
+                if (bestV != INT_MAX) {
+                    shPlan.f[j] += (FV)bestG;
+                    const int room = shPlan.room[j] - 1;
+                    shPlan.room[j] = room;
+                    shPlan.open[j] = (uint8_t)((room > 0 ? 1 : 0) | 2);
+                    prm.valid[(int64_t)l * prm.W + j] = 0;     // (plan_decide, same lane, may set it again)
+                }
+            }
+            __syncwarp();
         }
-    }
-    __syncthreads();
-    const int vstar = shPick;
-    const GV gstar = shG[0];
-    if (vstar == INT_MAX || vstar < 0 || vstar >= c.M) {
-        if (threadIdx.x == 0) atomicOr(prm.status, kDevBadState);
-        return;
-    }
-    // bookkeeping by the last warp while the others fold row v* into the coverage vector
-    if (threadIdx.x == kSelectThreads - 32) {
-        const int64_t at = (int64_t)l * prm.W + j;
-        prm.fval[at] += (FV)gstar;
-        prm.cnt[at] += 1;
-        prm.valid[at] = 0;
-        const int global = prm.perm[c.row0 + vstar];
-        prm.assignment[global] = j;
-        if (prm.order) prm.order[c.row0 + (c.M - nR)] = global;
-        const int k = pos[vstar];
-        cand[k] = lastV;
-        pos[lastV] = k;
-        pos[vstar] = -1;
-        prm.nR[l] = nR - 1;
-    }
-    // cover_j <- max(cover_j, S[v*][.])
-    {
-        const int ld4 = c.ld >> 2;
-        int4 *cov = reinterpret_cast<int4 *>(prm.cover + c.vOff + (int64_t)j * c.ld);
+        __syncthreads();
+        const int vstar = shPick;
+        if (vstar == INT_MAX || vstar < 0 || vstar >= c.M) {
+            if (threadIdx.x == 0) atomicOr(prm.status, kDevBadState);
+            return;
+        }
+        // warp 0: next block (shared memory only).  last warp: global bookkeeping of this pick.
+        // everybody else meanwhile starts fetching row v* and the coverage vector.
         const int4 *row = reinterpret_cast<const int4 *>(prm.S + c.sOff + (int64_t)vstar * c.ld);
+        int4 *cov = reinterpret_cast<int4 *>(prm.cover + c.vOff + (int64_t)j * c.ld);
+        if (warp == 0) {
+            plan_decide(prm, l, c, nR - 1, round + 1, shPlan);
+        } else if (threadIdx.x == kSelectThreads - 32) {
+            const int64_t at = (int64_t)l * prm.W + j;
+            prm.fval[at] = shPlan.f[j];
+            prm.cnt[at] += 1;
+            const int global = prm.perm[c.row0 + vstar];
+            prm.assignment[global] = j;
+            if (prm.order) prm.order[c.row0 + (c.M - nR)] = global;
+            const int k = pos[vstar];
+            const int lastV = cand[nR - 1];
+            cand[k] = lastV;
+            pos[lastV] = k;
+            pos[vstar] = -1;
+            prm.nR[l] = nR - 1;
+            if (nR == 1) atomicSub(&prm.nSweep[3], 1);        // one class fewer to finish
+        }
+        // cover_j <- max(cover_j, S[v*][.])
 #pragma unroll 2
         for (int i = threadIdx.x; i < ld4; i += kSelectThreads) {
             int4 a = cov[i], b = row[i];
@@ -598,9 +643,93 @@ __global__ void __launch_bounds__(kSelectThreads, 2) select_kernel(GreedyParams<
             }
             cov[i] = a;
         }
+        __syncthreads();
+        nR -= 1;
+        j = shPlan.nextJ;
+        if (nR == 0 || j < 0 || shPlan.needSweep) return;
+    }
+}
+
+// Picks of round `round`: every class advances until it needs a sweep (or is finished).
+template <typename SV>
+__global__ void __launch_bounds__(kSelectThreads, 2) chain_kernel(GreedyParams<SV> prm, int round)
+{
+    cudaGridDependencySynchronize();              // the sweep of this round has finished
+    cudaTriggerProgrammaticLaunchCompletion();
+    pick_chain(prm, blockIdx.x, round);
+}
+
+// ---------------------------------------------------------------------------------------------
+// The whole greedy loop in one cooperative launch.  A round = one sweep phase (every class that
+// asked for a sweep, all CTAs) and one pick phase (class l by CTA l mod gridDim.x: picks until the
+// class needs its next sweep), separated by grid barriers.  Control flow is uniform across the
+// grid: the number of unfinished classes is read after a barrier and not touched before the next.
+// Barrier over all CTAs of a cooperative launch (all co-resident): one arrival counter that only
+// grows, so round k waits for k * gridDim.x arrivals.  The wait is bounded; when it runs out (or
+// another CTA has already reported that) the timeout bit is set in the status word and the caller
+// leaves its loop.  Thread 0's fences order this CTA's writes before its arrival and make the other
+// CTAs' writes visible after the wait (the fence drops stale L1 lines of this SM).
+constexpr unsigned kBarrierSpinLimit = 1u << 26;
+__device__ __forceinline__ bool grid_barrier(unsigned *counter, unsigned expected, int32_t *status)
+{
+    __shared__ int shOk;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        atomicAdd(counter, 1u);
+        int ok = 1;
+        unsigned spins = 0;
+        while (*(volatile unsigned *)counter < expected) {
+            if ((++spins & 1023u) == 0 && ((*(volatile int32_t *)status & kDevTimeout) || spins >= kBarrierSpinLimit)) {
+                atomicOr(status, kDevTimeout);
+                ok = 0;
+                break;
+            }
+        }
+        __threadfence();
+        shOk = ok;
     }
     __syncthreads();
-    plan_next(prm, l, step + 1, shPlan);
+    return shOk != 0;
+}
+
+__device__ __forceinline__ unsigned long long global_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+
+// (The loop keeps next to nothing in registers across the two phases -- the phase clocks of CTA 0
+// sit in shared memory, the barrier's target is recomputed from the round number -- so that the
+// sweep's inner loop gets the whole register budget.)
+template <typename SV>
+__global__ void __launch_bounds__(kSweepThreads, 1) greedy_persistent_kernel(GreedyParams<SV> prm, int maxRounds)
+{
+    extern __shared__ int4 shCover[];
+    __shared__ unsigned long long shClock[3];      // last stamp, sweep-phase ns, pick-phase ns (CTA 0, thread 0)
+    if (blockIdx.x == 0 && threadIdx.x == 0) { shClock[0] = global_ns(); shClock[1] = 0; shClock[2] = 0; }
+    for (int r = 0; r < maxRounds; ++r) {
+        if (*(volatile int32_t *)&prm.nSweep[3] == 0) break;     // every class is finished
+        sweep_step(prm, r, shCover);
+        if (!grid_barrier(prm.barrier, (unsigned)(2 * r + 1) * gridDim.x, prm.status)) break;   // gains of round r are in place
+        if (blockIdx.x == 0 && threadIdx.x == 0) {
+            const unsigned long long t1 = global_ns();
+            shClock[1] += t1 - shClock[0];
+            shClock[0] = t1;
+        }
+        for (int l = blockIdx.x; l < prm.L; l += gridDim.x) {
+            pick_chain(prm, l, r);
+            __syncthreads();
+        }
+        if (!grid_barrier(prm.barrier, (unsigned)(2 * r + 2) * gridDim.x, prm.status)) break;   // picks of round r, sweep list of round r+1
+        if (blockIdx.x == 0 && threadIdx.x == 0) {
+            const unsigned long long t1 = global_ns();
+            shClock[2] += t1 - shClock[0];
+            shClock[0] = t1;
+        }
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0) { prm.phaseNs[0] = shClock[1]; prm.phaseNs[1] = shClock[2]; }
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -650,6 +779,8 @@ static rcd_status run_greedy(rcd_ctx *ctx, const Sizes &sz, const Workspace &ws,
     prm.nSweep = ws.nSweep;
     prm.stepBytes = ws.stepBytes;
     prm.stepOps = ws.stepOps;
+    prm.phaseNs = ws.phaseNs;
+    prm.barrier = (unsigned *)(ws.phaseNs + 2);
     prm.status = ws.status;
     prm.perm = ws.perm;
     prm.assignment = assignment;
@@ -664,7 +795,7 @@ static rcd_status run_greedy(rcd_ctx *ctx, const Sizes &sz, const Workspace &ws,
 
     int maxLd = 0;
     for (const auto &c : descHost) if (c.ld > maxLd) maxLd = c.ld;
-    const int64_t smemCap = (int64_t)ctx->maxSmemOptin - 2048;     // static shared + margin
+    const int64_t smemCap = (int64_t)ctx->maxSmemOptin - 20 * 1024;  // static shared of the kernels + margin
     int64_t smem = (int64_t)batch * maxLd * (int64_t)sizeof(SV);
     if (smem > smemCap) smem = smemCap;
     if ((int64_t)maxLd * (int64_t)sizeof(SV) > smem)
@@ -683,7 +814,9 @@ static rcd_status run_greedy(rcd_ctx *ctx, const Sizes &sz, const Workspace &ws,
     }
     RCD_CUDA(ctx, cudaFuncSetAttribute(sweep_kernel<SV>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
 
-    RCD_CUDA(ctx, cudaMemsetAsync(ws.nSweep, 0, 2 * sizeof(int32_t), st));
+    RCD_CUDA(ctx, cudaMemsetAsync(ws.nSweep, 0, 4 * sizeof(int32_t), st));
+    RCD_CUDA(ctx, cudaMemsetAsync(ws.phaseNs, 0, 3 * sizeof(unsigned long long), st));
+    ctx->phaseNsDev = ws.phaseNs;
     RCD_CUDA(ctx, cudaMemsetAsync(ws.stepBytes, 0, (size_t)(sz.maxM + 1) * sizeof(unsigned long long), st));
     RCD_CUDA(ctx, cudaMemsetAsync(ws.stepOps, 0, (size_t)(sz.maxM + 1) * sizeof(unsigned long long), st));
     init_kernel<SV><<<sz.L, kSelectThreads, 0, st>>>(prm);
@@ -691,20 +824,37 @@ static rcd_status run_greedy(rcd_ctx *ctx, const Sizes &sz, const Workspace &ws,
     RCD_CUDA(ctx, cudaGetLastError());
 
     const bool perSweep = ctx->cfg.profile >= 2;
-    if (perSweep) {
-        while ((int64_t)ctx->evSweep.size() < 2 * sz.maxM) {
-            cudaEvent_t e;
-            RCD_CUDA(ctx, cudaEventCreate(&e));
-            ctx->evSweep.push_back(e);
-        }
-    }
     ctx->sweepEventsUsed = 0;
-    for (int64_t t = 0; t < sz.maxM; ++t) {
-        if (perSweep) RCD_CUDA(ctx, cudaEventRecord(ctx->evSweep[2 * t], st));
-        RCD_CUDA(ctx, launch_pdl(sweep_kernel<SV>, dim3(ctx->smCount), dim3(kSweepThreads), (size_t)smem, st, prm, (int)t));
-        if (perSweep) RCD_CUDA(ctx, cudaEventRecord(ctx->evSweep[2 * t + 1], st));
-        RCD_CUDA(ctx, launch_pdl(select_kernel<SV>, dim3(sz.L), dim3(kSelectThreads), 0, st, prm, (int)t));
-        ctx->kernelLaunches += 2;
+    // One cooperative launch for the whole loop when the device can hold one sweep CTA per SM at once;
+    // per-sweep event timing (profile 2) needs the sweeps as separate launches.
+    bool persistent = ctx->cfg.greedy_path != 1 && !perSweep && ctx->cooperative;
+    if (persistent) {
+        RCD_CUDA(ctx, cudaFuncSetAttribute(greedy_persistent_kernel<SV>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        int perSm = 0;
+        RCD_CUDA(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&perSm, greedy_persistent_kernel<SV>, kSweepThreads, (size_t)smem));
+        if (perSm < 1) persistent = false;
+    }
+    if (persistent) {
+        int steps = (int)sz.maxM;
+        void *args[] = {(void *)&prm, (void *)&steps};
+        RCD_CUDA(ctx, cudaLaunchCooperativeKernel((const void *)greedy_persistent_kernel<SV>, dim3(ctx->smCount), dim3(kSweepThreads),
+                                                  args, (size_t)smem, st));
+        ctx->kernelLaunches += 1;
+    } else {
+        if (perSweep) {
+            while ((int64_t)ctx->evSweep.size() < 2 * sz.maxM) {
+                cudaEvent_t e;
+                RCD_CUDA(ctx, cudaEventCreate(&e));
+                ctx->evSweep.push_back(e);
+            }
+        }
+        for (int64_t t = 0; t < sz.maxM; ++t) {
+            if (perSweep) RCD_CUDA(ctx, cudaEventRecord(ctx->evSweep[2 * t], st));
+            RCD_CUDA(ctx, launch_pdl(sweep_kernel<SV>, dim3(ctx->smCount), dim3(kSweepThreads), (size_t)smem, st, prm, (int)t));
+            if (perSweep) RCD_CUDA(ctx, cudaEventRecord(ctx->evSweep[2 * t + 1], st));
+            RCD_CUDA(ctx, launch_pdl(chain_kernel<SV>, dim3(sz.L), dim3(kSelectThreads), 0, st, prm, (int)t));
+            ctx->kernelLaunches += 2;
+        }
     }
     if (perSweep) ctx->sweepEventsUsed = 2 * sz.maxM;
     RCD_CUDA(ctx, cudaGetLastError());

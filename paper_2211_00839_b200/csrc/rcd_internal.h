@@ -86,10 +86,11 @@ struct Workspace {
     int32_t *sweepParts;    // [L][kMaxSweepBatch]
     int32_t *sweepCS;       // [L] warps per row group in the next sweep
     int32_t *rowCtr;        // [L] ticket counter over row groups of the running sweep
-    int32_t *sweepList;     // [2][L] classes that sweep in the next step (double-buffered by step parity)
-    int32_t *nSweep;        // [2]
+    int32_t *sweepList;     // [3][L] classes that sweep in a step (three lists in rotation)
+    int32_t *nSweep;        // [3] (+1 pad)
     unsigned long long *stepBytes;   // [steps+1] bytes the sweep of step t has to read
     unsigned long long *stepOps;     // [steps+1] element x block pairs of that sweep
+    unsigned long long *phaseNs;     // [2] sweep-phase / pick-phase nanoseconds of the persistent kernel
     int32_t *status;        // [1]
     size_t bytes;           // total bytes laid out
 };
@@ -118,6 +119,7 @@ struct rcd_ctx {
     int device = 0;
     int smCount = 0;
     int maxSmemOptin = 0;
+    bool cooperative = false;           // device supports cooperative launches
     rcd_config cfg{};
     std::string err;
     int32_t *hostStage = nullptr;       // pinned, counts / status read-back
@@ -133,6 +135,7 @@ struct rcd_ctx {
     int64_t steps = 0;
     const unsigned long long *stepBytesDev = nullptr;
     const unsigned long long *stepOpsDev = nullptr;
+    const unsigned long long *phaseNsDev = nullptr;
     const int32_t *statusDev = nullptr;
 };
 

@@ -98,11 +98,12 @@ def check_exact(rcd, orc, wl, variant="incremental", **cfg):
     return a, o, v, ref
 
 
+@pytest.mark.parametrize("path", [0, 1])        # one cooperative launch / two launches per step
 @pytest.mark.parametrize("batch", [1, 2, 4, 8])
-def test_partition_c1_exact(rcd, orc, batch):
+def test_partition_c1_exact(rcd, orc, batch, path):
     from paper_2211_00839_b200.workloads import make_workload
     wl = make_workload("C1")
-    a, o, v, ref = check_exact(rcd, orc, wl, variant="plain", sweep_batch_max=batch)
+    a, o, v, ref = check_exact(rcd, orc, wl, variant="plain", sweep_batch_max=batch, greedy_path=path)
     for l in range(wl.L):
         ids = np.nonzero(wl.labels == l)[0]
         assert np.bincount(a[ids], minlength=wl.W).tolist() == [25, 25, 50, 100]
@@ -127,8 +128,8 @@ def test_partition_int8_ragged_classes(rcd, orc, seed):
     caps = np.array([1, 2.5, 1, 4, 0.5, 3, 1, 1, 2], dtype=np.float64)
     wl = Workload("ragged", "int8", np.ascontiguousarray(feats[perm]), np.ascontiguousarray(labels[perm]), caps,
                   len(sizes), len(caps))
-    for batch in (8, 1):
-        check_exact(rcd, orc, wl, sweep_batch_max=batch)
+    for batch, path in ((8, 0), (1, 0), (8, 1)):
+        check_exact(rcd, orc, wl, sweep_batch_max=batch, greedy_path=path)
 
 
 def test_partition_int8_ties_and_duplicates(rcd, orc):
@@ -204,11 +205,11 @@ def test_partition_c3_reduced_float(rcd, orc):
     check_float(rcd, orc, wl)
 
 
-@pytest.mark.parametrize("batch", [1, 8])
-def test_partition_c4_reduced_float(rcd, orc, batch):
+@pytest.mark.parametrize("batch,path", [(1, 0), (8, 0), (8, 1)])
+def test_partition_c4_reduced_float(rcd, orc, batch, path):
     from paper_2211_00839_b200.workloads import make_workload
     wl = make_workload("C4", L=5, M=500, d=256)
-    check_float(rcd, orc, wl, sweep_batch_max=batch)
+    check_float(rcd, orc, wl, sweep_batch_max=batch, greedy_path=path)
 
 
 # ----------------------------------------------------------------------------- objective
