@@ -177,11 +177,12 @@ __device__ void plan_decide(const GreedyParams<SV> &prm, int l, const ClassDesc 
         __syncwarp();
     }
     if (lane == 0) for (int k = n; k < P; ++k) parts[k] = jstar;
-    // warps per row group: enough that the row groups of the classes expected to sweep together
-    // (about L / P of them) cover every warp of the launch, at least one 128-column chunk per warp
+    // warps per row group: enough that the row groups of the classes that sweep together (every
+    // unfinished class, once per round) cover every warp of the launch, at least one 128-column chunk per warp
     const int R = rows_per_group(P);
     const int64_t nGroups = (nR + R - 1) / R;
-    const int64_t together = prm.L / P > 1 ? prm.L / P : 1;
+    const int rem = *(volatile int32_t *)&prm.nSweep[3];              // unfinished classes: they all sweep in the same round
+    const int64_t together = rem > 1 ? rem : 1;
     const int chunks = (c.ld + 127) / 128;
     int CS = 1;
     while (CS < 16 && 2 * CS <= chunks && 2 * CS * together * nGroups <= prm.sweepWarps) CS *= 2;
@@ -487,21 +488,35 @@ __device__ __forceinline__ void sweep_step(const GreedyParams<SV> &prm, int step
     const int nS = prm.nSweep[par];
     if (blockIdx.x == 0 && threadIdx.x == 0) prm.nSweep[(step + 2) % 3] = 0;
     if (nS == 0) return;
+    // Every CTA has a home position in the list (CTAs spread evenly over the sweeping classes) and
+    // serves, again and again, the nearest class at or after it that still has row groups to hand
+    // out.  One parallel look at all ticket counters finds that class; a class whose tickets have
+    // run out stays that way for the rest of the round, so the loop ends.
     const int start = (int)(((int64_t)blockIdx.x * nS) / gridDim.x);
-    for (int k = 0; k < nS; ++k) {
-        int s = start + k;
+    for (;;) {
+        if (threadIdx.x == 0) shGo = INT_MAX;
+        __syncthreads();
+        for (int s = threadIdx.x; s < nS; s += blockDim.x) {
+            const int ls = prm.sweepList[(int64_t)par * prm.L + s];
+            const int Rs = rows_per_group(prm.sweepN[ls]);
+            const int groups = (prm.nR[ls] + Rs - 1) / Rs;
+            if (*(volatile int32_t *)&prm.rowCtr[ls] < groups) {
+                int dist = s - start;
+                if (dist < 0) dist += nS;
+                atomicMin(&shGo, dist);
+            }
+        }
+        __syncthreads();
+        const int go = shGo;
+        if (go == INT_MAX) break;
+        int s = start + go;
         if (s >= nS) s -= nS;
         const int l = prm.sweepList[(int64_t)par * prm.L + s];
         const ClassDesc c = prm.desc[l];
         const int nR = prm.nR[l];
         const int P = prm.sweepN[l];
         const int CS = prm.sweepCS[l];
-        const int R = rows_per_group(P);
-        const int nGroups = (nR + R - 1) / R;
-        if (threadIdx.x == 0) shGo = (*(volatile int32_t *)&prm.rowCtr[l] < nGroups) ? 1 : 0;
-        __syncthreads();
-        const int go = shGo;
-        if (go) {
+        {
             const int ld4 = c.ld >> 2;
             const int32_t *parts = prm.sweepParts + (int64_t)l * kMaxSweepBatch;
             const int4 *cov = reinterpret_cast<const int4 *>(prm.cover + c.vOff);
@@ -568,11 +583,25 @@ __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, i
         // samples with independent, coalesced loads (pos[v] < 0 marks an assigned sample).
         GV bestG = 0;
         int bestV = INT_MAX;
-#pragma unroll 4
-        for (int v = threadIdx.x; v < c.M; v += kSelectThreads) {
-            const GV g = G[v];
-            const int ps = pos[v];
-            if (ps >= 0 && (bestV == INT_MAX || g > bestG)) { bestG = g; bestV = v; }
+        // batches of kArgmaxBatch samples per thread: all loads of a batch are issued before the
+        // first comparison, so a class of up to kArgmaxBatch * kSelectThreads samples costs one
+        // memory round trip
+        constexpr int kArgmaxBatch = 12;
+        for (int v0 = threadIdx.x; v0 < c.M; v0 += kArgmaxBatch * kSelectThreads) {
+            GV g[kArgmaxBatch];
+            int ps[kArgmaxBatch];
+#pragma unroll
+            for (int i = 0; i < kArgmaxBatch; ++i) {
+                const int v = v0 + i * kSelectThreads;
+                ps[i] = -1;
+                g[i] = 0;
+                if (v < c.M) { g[i] = G[v]; ps[i] = pos[v]; }
+            }
+#pragma unroll
+            for (int i = 0; i < kArgmaxBatch; ++i) {
+                const int v = v0 + i * kSelectThreads;
+                if (ps[i] >= 0 && (bestV == INT_MAX || g[i] > bestG)) { bestG = g[i]; bestV = v; }
+            }
         }
         for (int off = 16; off > 0; off >>= 1) {
             GV oG = __shfl_xor_sync(0xffffffffu, bestG, off);
