@@ -249,7 +249,10 @@ def run_ours(args):
     achieved = prof["sweep_bytes"] / loop_s / 1e9 if loop_s > 0 else 0.0
     roofline = {"bound": "hbm", "kernel": "greedy_persistent_kernel", "achieved": achieved, "peak": peaks["hbm_gbs"],
                 "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "peak_source": peaks["source"],
-                "traffic": None, "launch_ms": prof["greedy_ms"], "bytes_per_launch": prof["sweep_bytes"],
+                # dram__bytes_read.sum + dram__bytes_write.sum of one launch on the default C2 workload
+                # (ncu capture summarised in profiles/greedy_persistent_kernel_C2.md)
+                "traffic": 491.18e9 if (args.config == "C2" and args.sweep_batch in (0, 8) and args.greedy_path == 0) else None,
+                "launch_ms": prof["greedy_ms"], "bytes_per_launch": prof["sweep_bytes"],
                 "rounds_with_sweeps": int(prof["sweep_launches"])}
     # the same bytes against the time the kernel spends in its sweep phases (its own clock, CTA 0)
     if prof["persistent_sweep_ns"] > 0:

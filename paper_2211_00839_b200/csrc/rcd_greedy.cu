@@ -1,4 +1,4 @@
-// The greedy loop of Algorithm 1 with the facility-location objective, all classes in lockstep.
+// The greedy loop of Algorithm 1 with the facility-location objective, for all classes together.
 //
 // Per class the device keeps, for every block p: a coverage vector cover_p[i] =
 // max(0, max_{v' in A_p} S[i][v']), the tracked value f_p = sum_i cover_p[i], the count and the
@@ -7,15 +7,20 @@
 // receives a sample, so a pass over S is only needed when the chosen block's row is out of date,
 // and that pass refreshes up to `sweep_batch_max` out-of-date blocks at once.
 //
-// One greedy step t = two launches:
-//   sweep_kernel   persistent CTAs (one per SM) serve every class that scheduled a sweep; teams
-//                  of 1-16 warps pull groups of rows, each warp streams its 128-column chunks of
-//                  those rows with 128-bit loads against the coverage vectors staged in shared
-//                  memory, reduces with warp shuffles, and the team writes G.
-//   select_kernel  one CTA per class: argmax of G_{j*} over the unassigned samples (warp-shuffle
-//                  reduction, lowest index on ties), coverage / value / count update, removal of
-//                  v* from the candidate list, choice of the next block j* (least f among the
-//                  non-full blocks, lowest index on ties) and scheduling of the next sweep.
+// The loop advances in rounds.  A round is
+//   a sweep phase  every class that asked for a sweep gets one.  Persistent CTAs (one per SM)
+//                  serve the classes; teams of 1-16 warps pull groups of rows, each warp streams
+//                  its 128-column chunks of those rows with 128-bit loads against the coverage
+//                  vectors staged in shared memory, reduces with warp shuffles, the team writes G;
+//   a pick phase   one CTA per class makes pick after pick (argmax of G_{j*} over the unassigned
+//                  samples with a warp-shuffle reduction and lowest-index ties, coverage / value /
+//                  count update, removal of v* from the candidate list, choice of the next block
+//                  j* = least f among the non-full blocks) until the next block's gains are out of
+//                  date, and then asks for the class's next sweep.
+// Classes are independent, so each class makes exactly the picks Algorithm 1 prescribes whatever
+// the interleaving.  The whole loop is one cooperative launch (greedy_persistent_kernel, phases
+// separated by a bounded grid barrier); sweep_kernel / chain_kernel are the same two phases as
+// separate launches, used when every sweep is to be timed on its own.
 #include "rcd_internal.h"
 
 #include <limits.h>
