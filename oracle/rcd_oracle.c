@@ -73,6 +73,48 @@ void rcd_oracle_similarity_bf16(const uint16_t *Xbits, int64_t M, int64_t d, dou
     free(X);
 }
 
+/* Gaussian-kernel similarity (Section 4, item 2: "a Gaussian kernel with L2 distance",
+ * bandwidth sigma = sum_{v,v'} ||v - v'||_2 / n^2).  The paper gives neither the exponent
+ * nor what n counts; the reading taken here: n = |V_l| (the class), the sum runs over all
+ * ordered pairs (the zero diagonal included), and
+ *     sim(v, v') = exp(-||v - v'||^2 / (2 sigma^2)).
+ * A class whose points all coincide has sigma = 0; every similarity is then 1.
+ * X holds the features already widened to double; S and *sigma_out are outputs.           */
+static void gaussian_from_doubles(const double *X, int64_t M, int64_t d, double *S, double *sigma_out)
+{
+    double total = 0.0;
+    for (int64_t a = 0; a < M; ++a)
+        for (int64_t b = 0; b < M; ++b) {
+            double sq = 0.0;
+            for (int64_t k = 0; k < d; ++k) {
+                double diff = X[a * d + k] - X[b * d + k];
+                sq += diff * diff;
+            }
+            S[a * M + b] = sq;                  /* squared distance for now */
+            total += sqrt(sq);
+        }
+    double sigma = M > 0 ? total / ((double)M * (double)M) : 0.0;
+    for (int64_t i = 0; i < M * M; ++i)
+        S[i] = sigma > 0.0 ? exp(-S[i] / (2.0 * sigma * sigma)) : 1.0;
+    if (sigma_out) *sigma_out = sigma;
+}
+
+void rcd_oracle_gaussian_i8(const int8_t *X, int64_t M, int64_t d, double *S, double *sigma_out)
+{
+    double *Xd = (double *)malloc((size_t)(M * d + 1) * sizeof(double));
+    for (int64_t i = 0; i < M * d; ++i) Xd[i] = (double)X[i];
+    gaussian_from_doubles(Xd, M, d, S, sigma_out);
+    free(Xd);
+}
+
+void rcd_oracle_gaussian_bf16(const uint16_t *Xbits, int64_t M, int64_t d, double *S, double *sigma_out)
+{
+    double *Xd = (double *)malloc((size_t)(M * d + 1) * sizeof(double));
+    for (int64_t i = 0; i < M * d; ++i) Xd[i] = bf16_to_double(Xbits[i]);
+    gaussian_from_doubles(Xd, M, d, S, sigma_out);
+    free(Xd);
+}
+
 /* ------------------------------------------------------------------------- */
 /* Quotas (Algorithm 1, "Constraint C_{l,j} = |V_l| r_j / sum_j r_j").
  * Largest-remainder rule: floor every share, then hand the left-over units one

@@ -46,6 +46,8 @@ def _load():
     lib.rcd_oracle_similarity_i8.argtypes = [P, i64, i64, P]
     lib.rcd_oracle_similarity_bf16.argtypes = [P, i64, i64, P]
     lib.rcd_oracle_quotas.argtypes = [i64, P, i32, P]
+    lib.rcd_oracle_gaussian_i8.argtypes = [P, i64, i64, P, P]
+    lib.rcd_oracle_gaussian_bf16.argtypes = [P, i64, i64, P, P]
     for suf, ret in (("i64", i64), ("f64", dbl)):
         f = getattr(lib, "rcd_oracle_f_" + suf)
         f.argtypes = [P, i64, P, i64]
@@ -92,6 +94,31 @@ def similarity(X: np.ndarray) -> np.ndarray:
     else:
         raise TypeError("features must be int8 or uint16 (bf16 bits)")
     return S
+
+
+def similarity_gaussian(X: np.ndarray):
+    """Gaussian-kernel similarity of one class and its bandwidth: (S float64 [M, M], sigma)."""
+    lib = _load()
+    X = np.ascontiguousarray(X)
+    M, d = X.shape
+    S = np.empty((M, M), dtype=np.float64)
+    sigma = C.c_double(0.0)
+    if X.dtype == np.int8:
+        lib.rcd_oracle_gaussian_i8(_ptr(X), M, d, _ptr(S), C.byref(sigma))
+    elif X.dtype == np.uint16:
+        lib.rcd_oracle_gaussian_bf16(_ptr(X), M, d, _ptr(S), C.byref(sigma))
+    else:
+        raise TypeError("features must be int8 or uint16 (bf16 bits)")
+    return S, float(sigma.value)
+
+
+def class_similarity(X: np.ndarray, kind: str = "dot") -> np.ndarray:
+    """S of one class for the chosen similarity ("dot": dot product / cosine; "gaussian")."""
+    if kind == "dot":
+        return similarity(X)
+    if kind == "gaussian":
+        return similarity_gaussian(X)[0]
+    raise ValueError(kind)
 
 
 def quotas(M: int, capacities: Sequence[float]) -> np.ndarray:
@@ -181,7 +208,8 @@ class PartitionResult:
 
 def partition(features: np.ndarray, labels: np.ndarray, capacities: Sequence[float], L: int,
               variant: str = "incremental", threads: int = 1,
-              classes: Optional[Sequence[int]] = None, max_picks: int = -1) -> PartitionResult:
+              classes: Optional[Sequence[int]] = None, max_picks: int = -1,
+              similarity_kind: str = "dot") -> PartitionResult:
     """Algorithm 1 over the whole dataset: classes handled one after another
     (or one per thread: they are independent), blocks joined at the end.
 
@@ -190,7 +218,7 @@ def partition(features: np.ndarray, labels: np.ndarray, capacities: Sequence[flo
     features = np.ascontiguousarray(features)
     N = features.shape[0]
     W = len(capacities)
-    vdt = np.int64 if features.dtype == np.int8 else np.float64
+    vdt = np.int64 if (features.dtype == np.int8 and similarity_kind == "dot") else np.float64
     groups = split_by_label(labels, L)
     res = PartitionResult(N, L, W, vdt)
     res.class_offsets[1:] = np.cumsum([len(g) for g in groups])
@@ -202,7 +230,7 @@ def partition(features: np.ndarray, labels: np.ndarray, capacities: Sequence[flo
         q = quotas(M, capacities)
         if M == 0:
             return l, q, None
-        S = similarity(features[ids])
+        S = class_similarity(features[ids], similarity_kind)
         return l, q, partition_class(S, q, variant, max_picks)
 
     if threads > 1:
@@ -224,16 +252,17 @@ def partition(features: np.ndarray, labels: np.ndarray, capacities: Sequence[flo
     return res
 
 
-def objective(features: np.ndarray, labels: np.ndarray, assignment: np.ndarray, W: int, L: int) -> np.ndarray:
+def objective(features: np.ndarray, labels: np.ndarray, assignment: np.ndarray, W: int, L: int,
+              similarity_kind: str = "dot") -> np.ndarray:
     """f(A_j^l) for all (l, j), recomputed from the plain definition given an assignment."""
     features = np.ascontiguousarray(features)
-    vdt = np.int64 if features.dtype == np.int8 else np.float64
+    vdt = np.int64 if (features.dtype == np.int8 and similarity_kind == "dot") else np.float64
     out = np.zeros((L, W), dtype=vdt)
     groups = split_by_label(labels, L)
     for l, ids in enumerate(groups):
         if len(ids) == 0:
             continue
-        S = similarity(features[ids])
+        S = class_similarity(features[ids], similarity_kind)
         a = np.asarray(assignment)[ids]
         for j in range(W):
             out[l, j] = f_plain(S, np.nonzero(a == j)[0])

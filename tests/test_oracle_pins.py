@@ -365,3 +365,79 @@ def test_replay_accepts_own_trace_and_flags_planted_mistakes():
     oj4[t] = (oj4[t] + 1) % 3
     bad, stats, _ = orc.replay_class(S, q, oj4, ov, 0.0)
     assert bad != -1
+
+
+# ----------------------------------------------------------------------------- Gaussian-kernel similarity (Section 4 item 2)
+
+def test_gaussian_two_points_closed_form():
+    # two points at distance delta: sigma = (0 + delta + delta + 0) / 4 = delta / 2, so the off-diagonal
+    # similarity is exp(-delta^2 / (2 delta^2 / 4)) = exp(-2) whatever delta is
+    for delta in (1, 7, 100):
+        X = np.array([[0, 0, 0], [delta, 0, 0]], dtype=np.int8)
+        S, sigma = orc.similarity_gaussian(X)
+        assert sigma == pytest.approx(delta / 2.0, rel=1e-15)
+        assert S[0, 0] == 1.0 and S[1, 1] == 1.0
+        assert S[0, 1] == pytest.approx(math.exp(-2.0), rel=1e-14) and S[1, 0] == S[0, 1]
+
+
+def test_gaussian_equidistant_points_closed_form():
+    # M scaled one-hot vectors are pairwise at distance c*sqrt(2): sigma = delta (M-1)/M and every
+    # off-diagonal similarity is exp(-M^2 / (2 (M-1)^2))
+    M, c = 6, 9
+    X = (c * np.eye(M, 8)).astype(np.int8)
+    S, sigma = orc.similarity_gaussian(X)
+    delta = c * math.sqrt(2.0)
+    assert sigma == pytest.approx(delta * (M - 1) / M, rel=1e-14)
+    off = math.exp(-M * M / (2.0 * (M - 1) ** 2))
+    assert np.allclose(S[~np.eye(M, dtype=bool)], off, rtol=1e-13)
+    assert np.array_equal(np.diag(S), np.ones(M))
+
+
+def test_gaussian_matches_library_distances_and_is_scale_invariant():
+    from scipy.spatial.distance import cdist
+    from paper_2211_00839_b200.workloads import fp32_to_bf16_bits, bf16_bits_to_fp32
+    rng = np.random.default_rng(12)
+    X = rng.integers(-40, 41, size=(23, 17)).astype(np.int8)
+    S, sigma = orc.similarity_gaussian(X)
+    D = cdist(X.astype(np.float64), X.astype(np.float64))            # library routine for the distances
+    assert sigma == pytest.approx(D.sum() / 23 ** 2, rel=1e-13)
+    assert np.allclose(S, np.exp(-D ** 2 / (2 * sigma ** 2)), rtol=1e-12)
+    assert np.array_equal(S, S.T) and np.all(S > 0) and np.all(S <= 1)
+    # a larger distance never gives a larger similarity
+    order = np.argsort(D[0])
+    assert np.all(np.diff(S[0][order]) <= 1e-15)
+    # doubling every feature doubles every distance and sigma: the similarities do not move
+    S2, sigma2 = orc.similarity_gaussian((2 * X).astype(np.int8))
+    assert sigma2 == pytest.approx(2 * sigma, rel=1e-14) and np.allclose(S2, S, rtol=1e-13)
+    # translation does not matter either; and the bf16 variant sees the rounded values
+    S3, _ = orc.similarity_gaussian((X + 5).astype(np.int8))
+    assert np.allclose(S3, S, rtol=1e-13)
+    x = rng.standard_normal((9, 12)).astype(np.float32)
+    bits = fp32_to_bf16_bits(x)
+    Sb, sb = orc.similarity_gaussian(bits)
+    Db = cdist(bf16_bits_to_fp32(bits).astype(np.float64), bf16_bits_to_fp32(bits).astype(np.float64))
+    assert sb == pytest.approx(Db.sum() / 81, rel=1e-13)
+    assert np.allclose(Sb, np.exp(-Db ** 2 / (2 * sb ** 2)), rtol=1e-12)
+
+
+def test_gaussian_coincident_points():
+    X = np.full((4, 5), 3, dtype=np.int8)
+    S, sigma = orc.similarity_gaussian(X)
+    assert sigma == 0.0 and np.array_equal(S, np.ones((4, 4)))
+
+
+def test_partition_with_gaussian_similarity_keeps_the_invariants():
+    from paper_2211_00839_b200.workloads import make_workload
+    wl = make_workload("C1", L=2, M=40, d=16)
+    res = orc.partition(wl.features, wl.labels, wl.capacities, wl.L, variant="plain", similarity_kind="gaussian")
+    inc = orc.partition(wl.features, wl.labels, wl.capacities, wl.L, variant="incremental", similarity_kind="gaussian")
+    assert np.array_equal(res.assignment, inc.assignment) and np.array_equal(res.order, inc.order)
+    assert res.part_values.dtype == np.float64
+    for l in range(wl.L):
+        ids = np.nonzero(wl.labels == l)[0]
+        assert np.array_equal(np.bincount(res.assignment[ids], minlength=wl.W), res.quotas[l])
+    again = orc.objective(wl.features, wl.labels, res.assignment, wl.W, wl.L, similarity_kind="gaussian")
+    assert np.allclose(again, res.part_values, rtol=1e-12)
+    # with S in (0, 1] and S[i][i] = 1, a block that holds everything covers every point fully
+    S, _ = orc.similarity_gaussian(wl.features[wl.labels == 0])
+    assert orc.f_plain(S, list(range(S.shape[0]))) == pytest.approx(S.shape[0], rel=1e-15)
