@@ -55,13 +55,23 @@ typedef enum {
  *                 cosine), S accumulated and stored in fp32, gains in fp32, f tracked in fp64.  */
 typedef enum { RCD_FEAT_I8 = 0, RCD_FEAT_BF16 = 1 } rcd_feat_dtype;
 
+/* Similarity sim(v, v') of Section 4 item 2.
+ *   RCD_SIM_DOT       the dot product of the feature vectors (the cosine when rows are normalised);
+ *   RCD_SIM_GAUSSIAN  exp(-||v - v'||^2 / (2 sigma^2)) with sigma = the mean of ||v - v'||_2 over all ordered
+ *                     pairs of the class (the paper's Gaussian kernel; exponent and the range of the mean are
+ *                     readings, the paper gives neither).  S is then fp32 in (0, 1] for either feature type,
+ *                     and everything downstream uses the floating-point arithmetic of RCD_FEAT_BF16
+ *                     (gains fp32, tracked f and all objective outputs double).  */
+typedef enum { RCD_SIM_DOT = 0, RCD_SIM_GAUSSIAN = 1 } rcd_similarity_kind;
+
 typedef struct {
     int32_t sweep_batch_max;   /* blocks whose gains one pass over S may refresh: 1,2,4 or 8; 0 = default (8) */
     int32_t similarity_path;   /* 0 = tensor-core kernel when the shape allows, 2 = always the generic kernel */
     int32_t profile;           /* 0 off; 1 time the phases of rcd_partition; 2 also time every sweep launch */
     int32_t greedy_path;       /* 0 = whole greedy loop in one cooperative launch when the device allows;
                                   1 = two launches per greedy step (always used with profile 2) */
-    int32_t reserved[12];      /* must be 0 */
+    int32_t similarity_kind;   /* rcd_similarity_kind used by rcd_partition / rcd_objective (default RCD_SIM_DOT) */
+    int32_t reserved[11];      /* must be 0 */
 } rcd_config;
 
 /* Timings and counters of the last rcd_partition / rcd_partition_host on a context (profile >= 1). */
@@ -118,6 +128,15 @@ RCD_API rcd_status rcd_quotas(int64_t M, const double *capacities_host, int32_t 
 RCD_API rcd_status rcd_similarity(rcd_ctx *ctx, const void *X_dev, rcd_feat_dtype dtype, int64_t M, int64_t d,
                           int64_t batch, void *S_dev, int64_t ldS, void *cuda_stream);
 
+/* Gaussian-kernel similarity of `batch` equal classes (see rcd_similarity_kind), whatever the context's
+ * similarity_kind.  S_dev is fp32 [batch][M][ldS] (ldS = M rounded up to 4, pad columns 0);
+ * sigma_dev_or_null receives the `batch` bandwidths (fp32).  It first forms the dot products like
+ * rcd_similarity, then transforms them in place; the workspace holds row norms and partial sums. */
+RCD_API rcd_status rcd_similarity_gaussian_workspace_bytes(rcd_ctx *ctx, int64_t M, int64_t batch, size_t *bytes_out);
+RCD_API rcd_status rcd_similarity_gaussian(rcd_ctx *ctx, const void *X_dev, rcd_feat_dtype dtype, int64_t M, int64_t d,
+                                   int64_t batch, void *S_dev, int64_t ldS, float *sigma_dev_or_null,
+                                   void *workspace_dev, size_t workspace_bytes, void *cuda_stream);
+
 /* ---- partition (Algorithm 1 + GreedyStep, facility location) ------------------------------ */
 
 /* Upper bound of the workspace rcd_partition needs for N samples of width d in L classes none
@@ -134,7 +153,7 @@ RCD_API rcd_status rcd_partition_workspace_bytes(rcd_ctx *ctx, rcd_feat_dtype dt
  *   assignment_dev [N]            block of every sample, in [0, W)
  *   order_dev_or_null [N]         class-major (ascending label); inside a class the dataset
  *                                 indices of its samples in the order they were picked
- *   part_values_dev_or_null [L][W] tracked f(A_j^l): int64 (I8) or double (BF16)
+ *   part_values_dev_or_null [L][W] tracked f(A_j^l): int64 (I8 with RCD_SIM_DOT), else double
  * workspace_dev: 256-byte aligned, at least rcd_partition_workspace_bytes.
  * The call blocks once, briefly, on `cuda_stream` to read the L class sizes back (they fix the
  * launch shapes); everything after that is only enqueued.  Per class and per pick it runs:
@@ -169,8 +188,8 @@ RCD_API rcd_status rcd_objective_workspace_bytes(rcd_ctx *ctx, rcd_feat_dtype dt
  * assignment (values in [0, W); a negative entry means "in no block").  Independent of the
  * greedy state: it rebuilds S and takes, per row i and block j, the maximum over the block's
  * members.
- *   part_values_dev [L][W]  int64 (I8) or double (BF16)
- *   total_dev               one int64 or double: the sum over all (l, j)
+ *   part_values_dev [L][W]  int64 (I8 with RCD_SIM_DOT), else double
+ *   total_dev               one value of the same type: the sum over all (l, j)
  * Blocks once on the stream, like rcd_partition, to read the class sizes. */
 RCD_API rcd_status rcd_objective(rcd_ctx *ctx, const void *features_dev, rcd_feat_dtype dtype, int64_t N, int64_t d,
                          const int32_t *labels_dev, int32_t L, const int32_t *assignment_dev, int32_t W,

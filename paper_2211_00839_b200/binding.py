@@ -22,13 +22,16 @@ LIB_PATH = os.path.join(_HERE, "librcd.so")
 
 RCD_FEAT_I8 = 0
 RCD_FEAT_BF16 = 1
+RCD_SIM_DOT = 0
+RCD_SIM_GAUSSIAN = 1
 
 STATUS_NAMES = {0: "RCD_OK", 1: "RCD_ERR_INVALID_ARG", 2: "RCD_ERR_UNSUPPORTED", 3: "RCD_ERR_WORKSPACE_TOO_SMALL",
                 4: "RCD_ERR_CUDA", 5: "RCD_ERR_TIMEOUT", 6: "RCD_ERR_INTERNAL"}
 
 # every symbol include/rcd.h declares
 EXPORTS = ["rcd_create", "rcd_destroy", "rcd_last_error", "rcd_version", "rcd_sync_status", "rcd_get_profile",
-           "rcd_quotas", "rcd_similarity", "rcd_partition_workspace_bytes", "rcd_partition",
+           "rcd_quotas", "rcd_similarity", "rcd_similarity_gaussian_workspace_bytes", "rcd_similarity_gaussian",
+           "rcd_partition_workspace_bytes", "rcd_partition",
            "rcd_partition_host_workspace_bytes", "rcd_partition_host", "rcd_objective_workspace_bytes",
            "rcd_objective", "rcd_objective_class_static"]
 
@@ -41,7 +44,7 @@ class RcdError(RuntimeError):
 
 class RcdConfig(C.Structure):
     _fields_ = [("sweep_batch_max", C.c_int32), ("similarity_path", C.c_int32), ("profile", C.c_int32),
-                ("greedy_path", C.c_int32), ("reserved", C.c_int32 * 12)]
+                ("greedy_path", C.c_int32), ("similarity_kind", C.c_int32), ("reserved", C.c_int32 * 11)]
 
 
 class RcdProfile(C.Structure):
@@ -69,6 +72,8 @@ def _load() -> C.CDLL:
     lib.rcd_get_profile.argtypes = [vp, C.POINTER(RcdProfile)]
     lib.rcd_quotas.argtypes = [i64, vp, i32, vp]
     lib.rcd_similarity.argtypes = [vp, vp, C.c_int, i64, i64, i64, vp, i64, vp]
+    lib.rcd_similarity_gaussian_workspace_bytes.argtypes = [vp, i64, i64, C.POINTER(sz)]
+    lib.rcd_similarity_gaussian.argtypes = [vp, vp, C.c_int, i64, i64, i64, vp, i64, vp, vp, sz, vp]
     for name in ("rcd_partition_workspace_bytes", "rcd_partition_host_workspace_bytes",
                  "rcd_objective_workspace_bytes"):
         getattr(lib, name).argtypes = [vp, C.c_int, i64, i64, i32, i64, i32, C.POINTER(sz)]
@@ -134,7 +139,7 @@ class Context:
     """Owns one ``rcd_ctx`` on a CUDA device."""
 
     def __init__(self, device: int = 0, sweep_batch_max: int = 0, similarity_path: int = 0, profile: int = 0,
-                 greedy_path: int = 0):
+                 greedy_path: int = 0, similarity_kind: int = 0):
         torch = _torch()
         if not torch.cuda.is_available():
             raise RcdError(4, "no CUDA device: this library has no CPU path")
@@ -145,6 +150,8 @@ class Context:
         cfg.similarity_path = similarity_path
         cfg.profile = profile
         cfg.greedy_path = greedy_path
+        cfg.similarity_kind = similarity_kind
+        self.similarity_kind = similarity_kind
         self._h = C.c_void_p()
         st = lib.rcd_create(C.byref(self._h), self.device, C.byref(cfg))
         if st != 0:
@@ -208,6 +215,29 @@ class Context:
                                        C.c_void_p(S.data_ptr()), ld, self._stream()))
         return S
 
+    def _value_dtype(self, code: int):
+        torch = _torch()
+        return torch.int64 if (code == RCD_FEAT_I8 and self.similarity_kind == RCD_SIM_DOT) else torch.float64
+
+    def rcd_similarity_gaussian(self, X):
+        """X: [batch, M, d] (or [M, d]) int8 / bfloat16 on the device -> (S [batch, M, ld] float32, sigma [batch] float32)."""
+        torch = _torch()
+        if X.dim() == 2:
+            X = X.unsqueeze(0)
+        X = X.contiguous()
+        batch, M, d = X.shape
+        ld = (M + 3) // 4 * 4
+        code = _dtype_code(X)
+        S = torch.empty((batch, M, ld), dtype=torch.float32, device=X.device)
+        sigma = torch.empty(batch, dtype=torch.float32, device=X.device)
+        need = C.c_size_t()
+        self._check(lib.rcd_similarity_gaussian_workspace_bytes(self._h, M, batch, C.byref(need)))
+        ws = self.workspace(int(need.value))
+        self._check(lib.rcd_similarity_gaussian(self._h, C.c_void_p(X.data_ptr()), code, M, d, batch,
+                                                C.c_void_p(S.data_ptr()), ld, C.c_void_p(sigma.data_ptr()),
+                                                C.c_void_p(ws.data_ptr()), ws.numel(), self._stream()))
+        return S, sigma
+
     def partition_workspace_bytes(self, code: int, N: int, d: int, L: int, M_max: int, W: int, host: bool = False) -> int:
         out = C.c_size_t()
         fn = lib.rcd_partition_host_workspace_bytes if host else lib.rcd_partition_workspace_bytes
@@ -235,8 +265,7 @@ class Context:
         order = torch.empty(N, dtype=torch.int32, device=features.device) if want_order else None
         values = None
         if want_values:
-            values = torch.empty((L, W), dtype=torch.int64 if code == RCD_FEAT_I8 else torch.float64,
-                                 device=features.device)
+            values = torch.empty((L, W), dtype=self._value_dtype(code), device=features.device)
         self._check(lib.rcd_partition(self._h, C.c_void_p(features.data_ptr()), code, N, d,
                                       C.c_void_p(labels.data_ptr()), L, caps.ctypes.data_as(C.c_void_p), W,
                                       C.c_void_p(assignment.data_ptr()),
@@ -265,7 +294,7 @@ class Context:
         if out is None:
             assignment = torch.empty(N, dtype=torch.int32).pin_memory()
             order = torch.empty(N, dtype=torch.int32).pin_memory()
-            values = torch.empty((L, W), dtype=torch.int64 if code == RCD_FEAT_I8 else torch.float64).pin_memory()
+            values = torch.empty((L, W), dtype=self._value_dtype(code)).pin_memory()
         else:
             assignment, order, values = out
         with torch.cuda.device(self.torch_device):
@@ -289,7 +318,7 @@ class Context:
         out = C.c_size_t()
         self._check(lib.rcd_objective_workspace_bytes(self._h, code, N, d, L, M_max, W, C.byref(out)))
         ws = self.workspace(int(out.value))
-        vdt = torch.int64 if code == RCD_FEAT_I8 else torch.float64
+        vdt = self._value_dtype(code)
         values = torch.empty((L, W), dtype=vdt, device=features.device)
         total = torch.empty(1, dtype=vdt, device=features.device)
         self._check(lib.rcd_objective(self._h, C.c_void_p(features.data_ptr()), code, N, d,

@@ -49,7 +49,7 @@ size_t layout_workspace(void *base, rcd_feat_dtype dtype, const Sizes &sz, Works
     const size_t L = (size_t)std::max<int32_t>(sz.L, 1), W = (size_t)std::max<int32_t>(sz.W, 1);
     const size_t N = (size_t)std::max<int64_t>(sz.N, 1);
     const size_t sElem = 4;                                     // int32 / fp32
-    const size_t gElem = dtype == RCD_FEAT_I8 ? 8 : 4;          // int64 / fp32
+    const size_t gElem = sz.floatArith ? 4 : 8;                 // fp32 / int64
     Workspace w{};
     // the head does not depend on the class sizes: it is used before they are known
     w.status = c.take<int32_t>(4);
@@ -62,6 +62,10 @@ size_t layout_workspace(void *base, rcd_feat_dtype dtype, const Sizes &sz, Works
     w.perm = c.take<int32_t>(N);
     w.Xs = c.take<unsigned char>(N * (size_t)sz.d * feat_bytes(dtype));
     w.S = c.take<unsigned char>((size_t)std::max<int64_t>(sz.sElems, 1) * sElem);
+    w.gaussNorms = c.take<int32_t>(N);
+    w.gaussPartial = c.take<double>(L * (size_t)((sz.maxM + 63) / 64 + 1));
+    w.gaussSigma = c.take<float>(L);
+    w.gaussScale = c.take<float>(L);
     w.cover = c.take<unsigned char>((size_t)std::max<int64_t>(sz.vElems, 1) * sElem);
     w.gains = c.take<unsigned char>((size_t)std::max<int64_t>(sz.vElems, 1) * gElem);
     w.fval = c.take<unsigned char>(L * W * 8);
@@ -88,9 +92,15 @@ size_t layout_workspace(void *base, rcd_feat_dtype dtype, const Sizes &sz, Works
 static int32_t chunks_for(int64_t N) { return (int32_t)((N + kGroupChunk - 1) / kGroupChunk); }
 
 // Sizes for the promise "no class larger than Mmax".
-static Sizes bound_sizes(int64_t N, int64_t d, int32_t L, int64_t Mmax, int32_t W)
+static bool float_arith(const rcd_ctx *ctx, rcd_feat_dtype dtype)
+{
+    return dtype == RCD_FEAT_BF16 || ctx->cfg.similarity_kind == RCD_SIM_GAUSSIAN;
+}
+
+static Sizes bound_sizes(const rcd_ctx *ctx, rcd_feat_dtype dtype, int64_t N, int64_t d, int32_t L, int64_t Mmax, int32_t W)
 {
     Sizes sz{};
+    sz.floatArith = float_arith(ctx, dtype);
     sz.N = N; sz.d = d; sz.L = L; sz.W = W;
     if (Mmax > N) Mmax = N;
     sz.maxM = Mmax;
@@ -170,6 +180,7 @@ static rcd_status prepare(rcd_ctx *ctx, const void *features, rcd_feat_dtype dty
     // head of the workspace: status, counts
     Sizes head{};
     head.N = N; head.d = d; head.L = L; head.W = W; head.nChunks = chunks_for(N);
+    head.floatArith = float_arith(ctx, dtype);
     Workspace hw{};
     Sizes tiny = head;
     layout_workspace(workspace, dtype, tiny, &hw);
@@ -237,6 +248,11 @@ static rcd_status prepare(rcd_ctx *ctx, const void *features, rcd_feat_dtype dty
     }
     rs = launch_similarity(ctx, P.ws.Xs, dtype, N, d, cls, P.ws.S, st);
     if (rs != RCD_OK) return rs;
+    if (ctx->cfg.similarity_kind == RCD_SIM_GAUSSIAN) {
+        rs = launch_gaussian(ctx, P.ws.Xs, dtype, N, d, cls, P.ws.S, P.ws.gaussNorms, P.ws.gaussPartial, P.ws.gaussSigma,
+                             P.ws.gaussScale, st);
+        if (rs != RCD_OK) return rs;
+    }
     if (ctx->cfg.profile >= 1) RCD_CUDA(ctx, cudaEventRecord(ctx->evPhase[2], st));
     return RCD_OK;
 }
@@ -262,7 +278,8 @@ rcd_status rcd_create(rcd_ctx **out, int cuda_device, const rcd_config *cfg)
         if (cfg->similarity_path != 0 && cfg->similarity_path != 2) return RCD_ERR_INVALID_ARG;
         if (cfg->profile < 0 || cfg->profile > 2) return RCD_ERR_INVALID_ARG;
         if (cfg->greedy_path != 0 && cfg->greedy_path != 1) return RCD_ERR_INVALID_ARG;
-        for (int i = 0; i < 12; ++i) if (cfg->reserved[i] != 0) return RCD_ERR_INVALID_ARG;
+        if (cfg->similarity_kind != RCD_SIM_DOT && cfg->similarity_kind != RCD_SIM_GAUSSIAN) return RCD_ERR_INVALID_ARG;
+        for (int i = 0; i < 11; ++i) if (cfg->reserved[i] != 0) return RCD_ERR_INVALID_ARG;
     }
     int count = 0;
     if (cudaGetDeviceCount(&count) != cudaSuccess || cuda_device < 0 || cuda_device >= count) {
@@ -396,13 +413,52 @@ rcd_status rcd_similarity(rcd_ctx *ctx, const void *X_dev, rcd_feat_dtype dtype,
     return launch_similarity(ctx, X_dev, dtype, M * batch, d, cls, S_dev, st);
 }
 
+rcd_status rcd_similarity_gaussian_workspace_bytes(rcd_ctx *ctx, int64_t M, int64_t batch, size_t *bytes_out)
+{
+    if (!ctx) return RCD_ERR_INVALID_ARG;
+    if (!bytes_out || M < 0 || batch < 0 || M * batch > 0x7fffffffLL || batch > 0x7fffffffLL)
+        return fail(ctx, RCD_ERR_INVALID_ARG, "bad M, batch or null output");
+    *bytes_out = gaussian_scratch_bytes(M * batch, (int32_t)batch, M) + kAlign;
+    return RCD_OK;
+}
+
+rcd_status rcd_similarity_gaussian(rcd_ctx *ctx, const void *X_dev, rcd_feat_dtype dtype, int64_t M, int64_t d, int64_t batch,
+                                   void *S_dev, int64_t ldS, float *sigma_dev_or_null, void *workspace_dev,
+                                   size_t workspace_bytes, void *cuda_stream)
+{
+    rcd_status rs = rcd_similarity(ctx, X_dev, dtype, M, d, batch, S_dev, ldS, cuda_stream);
+    if (rs != RCD_OK || M == 0 || batch == 0) return rs;
+    if (batch > 65535) return fail(ctx, RCD_ERR_UNSUPPORTED, "Gaussian similarity: more than 65535 classes");
+    if (!workspace_dev || ((uintptr_t)workspace_dev) % kAlign) return fail(ctx, RCD_ERR_INVALID_ARG, "workspace null or not 256-byte aligned");
+    if (workspace_bytes < gaussian_scratch_bytes(M * batch, (int32_t)batch, M))
+        return fail(ctx, RCD_ERR_WORKSPACE_TOO_SMALL, "workspace has %zu bytes, need %zu", workspace_bytes,
+                    gaussian_scratch_bytes(M * batch, (int32_t)batch, M));
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    unsigned char *w = (unsigned char *)workspace_dev;
+    void *norms = w;                                  w += align_up((size_t)(M * batch) * 4);
+    double *partial = (double *)w;                    w += align_up((size_t)batch * (size_t)((M + 63) / 64) * 8);
+    float *sigma = (float *)w;                        w += align_up((size_t)batch * 4);
+    float *scale = (float *)w;
+    SimClasses cls{};
+    cls.src.table = nullptr;
+    cls.src.uniM = (int32_t)M;
+    cls.src.uniLd = (int32_t)ldS;
+    cls.L = (int32_t)batch;
+    cls.maxM = M;
+    rs = launch_gaussian(ctx, X_dev, dtype, M * batch, d, cls, S_dev, norms, partial, sigma, scale, st);
+    if (rs != RCD_OK) return rs;
+    if (sigma_dev_or_null)
+        RCD_CUDA(ctx, cudaMemcpyAsync(sigma_dev_or_null, sigma, (size_t)batch * sizeof(float), cudaMemcpyDeviceToDevice, st));
+    return RCD_OK;
+}
+
 rcd_status rcd_partition_workspace_bytes(rcd_ctx *ctx, rcd_feat_dtype dtype, int64_t N, int64_t d, int32_t L,
                                          int64_t M_max, int32_t W, size_t *bytes_out)
 {
     rcd_status rs = check_common(ctx, dtype, N, d, L, W);
     if (rs != RCD_OK) return rs;
     if (!bytes_out || M_max < 0) return fail(ctx, RCD_ERR_INVALID_ARG, "bad M_max or null output");
-    Sizes sz = bound_sizes(N, d, L, M_max, W);
+    Sizes sz = bound_sizes(ctx, dtype, N, d, L, M_max, W);
     *bytes_out = layout_workspace(nullptr, dtype, sz, nullptr);
     return RCD_OK;
 }
@@ -439,7 +495,7 @@ rcd_status rcd_partition(rcd_ctx *ctx, const void *features_dev, rcd_feat_dtype 
     for (int32_t l = 0; l < L; ++l) quotas_host(P.desc[(size_t)l].M, capacities_host, W, quota.data() + (size_t)l * W);
     RCD_CUDA(ctx, cudaMemcpyAsync(P.ws.quota, quota.data(), quota.size() * sizeof(int32_t), cudaMemcpyHostToDevice, st));
 
-    rs = launch_greedy(ctx, dtype, P.sz, P.ws, P.desc, assignment_dev, order_dev_or_null, st);
+    rs = launch_greedy(ctx, P.sz.floatArith ? RCD_FEAT_BF16 : RCD_FEAT_I8, P.sz, P.ws, P.desc, assignment_dev, order_dev_or_null, st);
     if (rs != RCD_OK) return rs;
     if (prof) RCD_CUDA(ctx, cudaEventRecord(ctx->evPhase[3], st));
     if (part_values_dev_or_null) {
@@ -469,7 +525,7 @@ rcd_status rcd_partition_host_workspace_bytes(rcd_ctx *ctx, rcd_feat_dtype dtype
     rcd_status rs = check_common(ctx, dtype, N, d, L, W);
     if (rs != RCD_OK) return rs;
     if (!bytes_out || M_max < 0) return fail(ctx, RCD_ERR_INVALID_ARG, "bad M_max or null output");
-    Sizes sz = bound_sizes(N, d, L, M_max, W);
+    Sizes sz = bound_sizes(ctx, dtype, N, d, L, M_max, W);
     *bytes_out = layout_workspace(nullptr, dtype, sz, nullptr) + host_tail_bytes(dtype, N, d, L, W) + kAlign;
     return RCD_OK;
 }
@@ -529,7 +585,7 @@ rcd_status rcd_objective_workspace_bytes(rcd_ctx *ctx, rcd_feat_dtype dtype, int
     rcd_status rs = check_common(ctx, dtype, N, d, L, W);
     if (rs != RCD_OK) return rs;
     if (!bytes_out || M_max < 0) return fail(ctx, RCD_ERR_INVALID_ARG, "bad M_max or null output");
-    Sizes sz = bound_sizes(N, d, L, M_max, W);
+    Sizes sz = bound_sizes(ctx, dtype, N, d, L, M_max, W);
     *bytes_out = layout_workspace(nullptr, dtype, sz, nullptr) + objective_scratch_bytes(L, std::min(M_max, N), W);
     return RCD_OK;
 }
@@ -556,7 +612,7 @@ rcd_status rcd_objective(rcd_ctx *ctx, const void *features_dev, rcd_feat_dtype 
     if (P.ws.bytes + scratchB > workspace_bytes)
         return fail(ctx, RCD_ERR_WORKSPACE_TOO_SMALL, "workspace has %zu bytes, objective needs %zu", workspace_bytes, P.ws.bytes + scratchB);
     void *scratch = (unsigned char *)workspace_dev + P.ws.bytes;
-    return launch_objective(ctx, dtype, P.sz, P.ws.desc, P.desc, P.ws.S, P.ws.perm, assignment_dev, part_values_dev,
+    return launch_objective(ctx, P.sz.floatArith ? RCD_FEAT_BF16 : RCD_FEAT_I8, P.sz, P.ws.desc, P.desc, P.ws.S, P.ws.perm, assignment_dev, part_values_dev,
                             total_dev, scratch, st);
 }
 

@@ -72,6 +72,10 @@ struct Workspace {
     ClassDesc *desc;        // [L]
     int32_t *tilePrefix;    // [L+1] first upper-triangle tile of every class (tensor-core similarity)
     void *S;                // similarity matrices
+    void *gaussNorms;       // [N] squared norms of the class-sorted rows (int32 / float)
+    double *gaussPartial;   // [L][ceil(maxM/64)] per-row-block sums of pairwise distances
+    float *gaussSigma;      // [L] bandwidth of every class
+    float *gaussScale;      // [L] 1 / (2 sigma^2)
     void *cover;            // [sum W*ld] coverage vectors (int32 / float)
     void *gains;            // [sum W*ld] stored gains (int64 / float)
     void *fval;             // [L][W] tracked f (int64 / double)
@@ -102,6 +106,7 @@ struct Sizes {
     int64_t vElems;         // sum W * ld_l
     int64_t maxM;
     int32_t nChunks;
+    bool floatArith;        // fp32 S / fp32 gains / double f (bf16 features, or the Gaussian kernel)
 };
 
 constexpr int kGroupChunk = 1024;           // samples per chunk of the stable class split
@@ -163,6 +168,11 @@ rcd_status launch_gather_rows(rcd_ctx *ctx, const void *X, const int32_t *perm, 
 // similarity: S_l = Xs_l Xs_l^T for every class described by desc
 rcd_status launch_similarity(rcd_ctx *ctx, const void *Xs, rcd_feat_dtype dtype, int64_t Ntot, int64_t d,
                              const SimClasses &cls, void *S, cudaStream_t st);
+
+// Gaussian-kernel similarity: transforms the dot products in S in place
+rcd_status launch_gaussian(rcd_ctx *ctx, const void *Xs, rcd_feat_dtype dtype, int64_t N, int64_t d, const SimClasses &cls,
+                           void *S, void *norms, double *partial, float *sigma, float *scale, cudaStream_t st);
+size_t gaussian_scratch_bytes(int64_t N, int32_t L, int64_t maxM);
 
 // greedy loop
 rcd_status launch_greedy(rcd_ctx *ctx, rcd_feat_dtype dtype, const Sizes &sz, const Workspace &ws,
