@@ -52,15 +52,19 @@ def _load():
         f = getattr(lib, "rcd_oracle_f_" + suf)
         f.argtypes = [P, i64, P, i64]
         f.restype = ret
+        fc = getattr(lib, "rcd_oracle_f_cut_" + suf)
+        fc.argtypes = [P, i64, P, i64]
+        fc.restype = ret
         for name in ("rcd_oracle_partition_plain_", "rcd_oracle_partition_incremental_"):
             g = getattr(lib, name + suf)
-            g.argtypes = [P, i64, i32, P, P, P, P, P, i64]
+            g.argtypes = [P, i64, i32, P, P, P, P, P, i64, C.c_int]
             g.restype = i64
-        r = getattr(lib, "rcd_oracle_replay_" + suf)
-        r.argtypes = [P, i64, i32, P, P, P, i64, dbl, P, P]
-        r.restype = i64
+        for name in ("rcd_oracle_replay_", "rcd_oracle_replay_cut_"):
+            r = getattr(lib, name + suf)
+            r.argtypes = [P, i64, i32, P, P, P, i64, dbl, P, P]
+            r.restype = i64
         q = getattr(lib, "rcd_oracle_gains_" + suf)
-        q.argtypes = [P, i64, P, i64, P]
+        q.argtypes = [P, i64, P, i64, P, C.c_int]
         q.restype = None
     _lib = lib
     return lib
@@ -130,25 +134,30 @@ def quotas(M: int, capacities: Sequence[float]) -> np.ndarray:
     return out
 
 
-def f_plain(S: np.ndarray, members: Sequence[int]):
-    """f(A) from the plain facility-location definition."""
+OBJECTIVES = {"facility": 0, "cut": 1}
+
+
+def f_plain(S: np.ndarray, members: Sequence[int], objective: str = "facility"):
+    """f(A) from the plain definition: facility location, or graph cut (Section 4 item 2)."""
     lib = _load()
     S = np.ascontiguousarray(S)
     m = np.ascontiguousarray(members, dtype=np.int32)
-    return getattr(lib, "rcd_oracle_f_" + _suffix(S))(_ptr(S), S.shape[0], _ptr(m), len(m))
+    name = "rcd_oracle_f_cut_" if OBJECTIVES[objective] == 1 else "rcd_oracle_f_"
+    return getattr(lib, name + _suffix(S))(_ptr(S), S.shape[0], _ptr(m), len(m))
 
 
-def gains_plain(S: np.ndarray, members: Sequence[int]) -> np.ndarray:
+def gains_plain(S: np.ndarray, members: Sequence[int], objective: str = "facility") -> np.ndarray:
     """f(A u {v}) - f(A) for every v, from the plain definition."""
     lib = _load()
     S = np.ascontiguousarray(S)
     m = np.ascontiguousarray(members, dtype=np.int32)
     out = np.empty(S.shape[0], dtype=S.dtype)
-    getattr(lib, "rcd_oracle_gains_" + _suffix(S))(_ptr(S), S.shape[0], _ptr(m), len(m), _ptr(out))
+    getattr(lib, "rcd_oracle_gains_" + _suffix(S))(_ptr(S), S.shape[0], _ptr(m), len(m), _ptr(out), OBJECTIVES[objective])
     return out
 
 
-def partition_class(S: np.ndarray, C_quota: Sequence[int], variant: str = "plain", max_picks: int = -1):
+def partition_class(S: np.ndarray, C_quota: Sequence[int], variant: str = "plain", max_picks: int = -1,
+                    objective: str = "facility"):
     """Algorithm 1 on one class.  Returns (assign[M], order_j[T], order_v[T], fvals[W]).
 
     ``max_picks >= 0`` stops the loop after that many picks (bounded timing sample)."""
@@ -163,12 +172,12 @@ def partition_class(S: np.ndarray, C_quota: Sequence[int], variant: str = "plain
     fv = np.empty(W, dtype=S.dtype)
     name = {"plain": "rcd_oracle_partition_plain_", "incremental": "rcd_oracle_partition_incremental_"}[variant]
     T = getattr(lib, name + _suffix(S))(_ptr(S), M, W, _ptr(q), _ptr(assign), _ptr(oj), _ptr(ov), _ptr(fv),
-                                         int(max_picks))
+                                         int(max_picks), OBJECTIVES[objective])
     return assign, oj[:T].copy(), ov[:T].copy(), fv
 
 
 def replay_class(S: np.ndarray, C_quota: Sequence[int], order_j: Sequence[int], order_v: Sequence[int],
-                 rel_tol: float):
+                 rel_tol: float, objective: str = "facility"):
     """Teacher-forced check of a pick sequence.  Returns (first_bad_step or -1, stats[4], fvals[W])."""
     lib = _load()
     S = np.ascontiguousarray(S)
@@ -177,7 +186,8 @@ def replay_class(S: np.ndarray, C_quota: Sequence[int], order_j: Sequence[int], 
     ov = np.ascontiguousarray(order_v, dtype=np.int32)
     stats = np.zeros(4, dtype=np.float64)
     fv = np.empty(len(q), dtype=S.dtype)
-    bad = getattr(lib, "rcd_oracle_replay_" + _suffix(S))(_ptr(S), S.shape[0], len(q), _ptr(q), _ptr(oj), _ptr(ov),
+    rname = "rcd_oracle_replay_cut_" if OBJECTIVES[objective] == 1 else "rcd_oracle_replay_"
+    bad = getattr(lib, rname + _suffix(S))(_ptr(S), S.shape[0], len(q), _ptr(q), _ptr(oj), _ptr(ov),
                                                          len(oj), float(rel_tol), _ptr(stats), _ptr(fv))
     return int(bad), stats, fv
 
@@ -209,7 +219,7 @@ class PartitionResult:
 def partition(features: np.ndarray, labels: np.ndarray, capacities: Sequence[float], L: int,
               variant: str = "incremental", threads: int = 1,
               classes: Optional[Sequence[int]] = None, max_picks: int = -1,
-              similarity_kind: str = "dot") -> PartitionResult:
+              similarity_kind: str = "dot", objective: str = "facility") -> PartitionResult:
     """Algorithm 1 over the whole dataset: classes handled one after another
     (or one per thread: they are independent), blocks joined at the end.
 
@@ -231,7 +241,7 @@ def partition(features: np.ndarray, labels: np.ndarray, capacities: Sequence[flo
         if M == 0:
             return l, q, None
         S = class_similarity(features[ids], similarity_kind)
-        return l, q, partition_class(S, q, variant, max_picks)
+        return l, q, partition_class(S, q, variant, max_picks, objective)
 
     if threads > 1:
         with ThreadPoolExecutor(max_workers=threads) as ex:
@@ -253,7 +263,7 @@ def partition(features: np.ndarray, labels: np.ndarray, capacities: Sequence[flo
 
 
 def objective(features: np.ndarray, labels: np.ndarray, assignment: np.ndarray, W: int, L: int,
-              similarity_kind: str = "dot") -> np.ndarray:
+              similarity_kind: str = "dot", objective: str = "facility") -> np.ndarray:
     """f(A_j^l) for all (l, j), recomputed from the plain definition given an assignment."""
     features = np.ascontiguousarray(features)
     vdt = np.int64 if (features.dtype == np.int8 and similarity_kind == "dot") else np.float64
@@ -265,5 +275,5 @@ def objective(features: np.ndarray, labels: np.ndarray, assignment: np.ndarray, 
         S = class_similarity(features[ids], similarity_kind)
         a = np.asarray(assignment)[ids]
         for j in range(W):
-            out[l, j] = f_plain(S, np.nonzero(a == j)[0])
+            out[l, j] = f_plain(S, np.nonzero(a == j)[0], objective)
     return out

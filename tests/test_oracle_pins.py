@@ -146,7 +146,7 @@ def test_hand_worked_traces(variant, as_float):
     cases = json.load(open(os.path.join(GOLDEN, "hand_traces.json")))["cases"]
     for c in cases:
         S = np.array(c["S"], dtype=np.float64 if as_float else np.int64)
-        assign, oj, ov, fv = orc.partition_class(S, c["quotas"], variant)
+        assign, oj, ov, fv = orc.partition_class(S, c["quotas"], variant, objective=c.get("objective", "facility"))
         assert oj.tolist() == c["order_j"], c["name"]
         assert ov.tolist() == c["order_v"], c["name"]
         assert assign.tolist() == c["assign"], c["name"]
@@ -441,3 +441,79 @@ def test_partition_with_gaussian_similarity_keeps_the_invariants():
     # with S in (0, 1] and S[i][i] = 1, a block that holds everything covers every point fully
     S, _ = orc.similarity_gaussian(wl.features[wl.labels == 0])
     assert orc.f_plain(S, list(range(S.shape[0]))) == pytest.approx(S.shape[0], rel=1e-15)
+
+
+# ----------------------------------------------------------------------------- graph-cut objective (Section 4 item 2)
+
+def brute_cut(S, A):
+    A = sorted(A)
+    out = [v for v in range(S.shape[0]) if v not in A]
+    if not A or not out:
+        return S.dtype.type(0)
+    return S[np.ix_(out, A)].sum()
+
+
+def test_graph_cut_closed_forms():
+    M = 7
+    S = np.ones((M, M), dtype=np.int64)
+    for n in range(M + 1):
+        assert orc.f_plain(S, list(range(n)), "cut") == (M - n) * n          # |V \ A| * |A| unit edges
+    assert orc.f_plain((5 * np.eye(M)).astype(np.int64), [1, 3], "cut") == 0   # no edges between distinct samples
+    # rows are the outside samples, columns the members: a non-symmetric S exposes a transposed operand
+    S = np.array([[0, 1], [5, 0]], dtype=np.int64)
+    assert orc.f_plain(S, [0], "cut") == 5 and orc.f_plain(S, [1], "cut") == 1
+    # not monotone: the full set cuts nothing
+    rng = np.random.default_rng(21)
+    S = rand_sym_int(rng, 9, 0, 30)
+    assert orc.f_plain(S, list(range(9)), "cut") == 0 and orc.f_plain(S, [], "cut") == 0
+    for A in ([2], [0, 5, 7], [1, 2, 3, 4, 8]):
+        assert orc.f_plain(S, A, "cut") == brute_cut(S, A)
+        g = orc.gains_plain(S, A, "cut")
+        for v in range(9):
+            if v not in A:
+                assert g[v] == brute_cut(S, A + [v]) - brute_cut(S, A)
+
+
+@pytest.mark.parametrize("seed", range(5))
+def test_graph_cut_every_pick_enumerated_and_variants_agree(seed):
+    rng = np.random.default_rng(500 + seed)
+    M = int(rng.integers(5, 12))
+    W = int(rng.integers(1, 4))
+    S = rand_sym_int(rng, M, -10, 40)
+    q = orc.quotas(M, rng.uniform(0.5, 3.0, size=W)).tolist()
+    plain = orc.partition_class(S, q, "plain", objective="cut")
+    inc = orc.partition_class(S, q, "incremental", objective="cut")
+    for x, y in zip(plain, inc):
+        assert np.array_equal(x, y)
+    assign, oj, ov, fv = plain
+    A = [set() for _ in range(W)]
+    J, R, t = set(range(W)), set(range(M)), 0
+    while R and J:
+        fJ = {j: brute_cut(S, A[j]) for j in J}
+        jstar = min(J, key=lambda j: (fJ[j], j))
+        if len(A[jstar]) + 1 <= q[jstar]:
+            vals = {v: brute_cut(S, A[jstar] | {v}) for v in R}
+            vstar = min(R, key=lambda v: (-vals[v], v))
+            assert (oj[t], ov[t]) == (jstar, vstar)
+            A[jstar].add(vstar); R.remove(vstar); t += 1
+        else:
+            J.remove(jstar)
+    assert t == len(oj)
+    for j in range(W):
+        assert fv[j] == brute_cut(S, A[j])
+    bad, stats, fv2 = orc.replay_class(S, q, oj, ov, 0.0, objective="cut")
+    assert bad == -1 and stats.tolist() == [0, 0, 0, 0] and np.array_equal(fv2, fv)
+
+
+def test_graph_cut_incremental_close_to_plain_in_double_and_invariants():
+    from paper_2211_00839_b200.workloads import make_workload
+    wl = make_workload("C4", L=2, M=40, d=32, seed=77)
+    res = orc.partition(wl.features, wl.labels, wl.capacities[:4], wl.L, variant="plain", objective="cut")
+    inc = orc.partition(wl.features, wl.labels, wl.capacities[:4], wl.L, variant="incremental", objective="cut")
+    assert np.array_equal(res.assignment, inc.assignment) and np.array_equal(res.order, inc.order)
+    assert np.allclose(res.part_values, inc.part_values, rtol=1e-12)
+    for l in range(wl.L):
+        ids = np.nonzero(wl.labels == l)[0]
+        assert np.array_equal(np.bincount(res.assignment[ids], minlength=4), res.quotas[l])
+    again = orc.objective(wl.features, wl.labels, res.assignment, 4, wl.L, objective="cut")
+    assert np.allclose(again, res.part_values, rtol=1e-12)
