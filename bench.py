@@ -176,7 +176,8 @@ def run_ours(args):
     yh = torch.from_numpy(wl.labels).pin_memory()
     Xd, yd = Xh.to(dev), yh.to(dev)
     kind = rcd.RCD_SIM_GAUSSIAN if args.similarity == "gaussian" else rcd.RCD_SIM_DOT
-    ctx = rcd.Context(local, sweep_batch_max=args.sweep_batch, profile=1, greedy_path=args.greedy_path, similarity_kind=kind)
+    ctx = rcd.Context(local, sweep_batch_max=args.sweep_batch, profile=1, greedy_path=args.greedy_path, similarity_kind=kind,
+                      objective=rcd.RCD_OBJ_GRAPH_CUT if args.objective == "cut" else rcd.RCD_OBJ_FACILITY)
 
     def barrier():
         torch.cuda.synchronize()
@@ -248,11 +249,11 @@ def run_ours(args):
     peaks = load_peaks()
     loop_s = prof["greedy_ms"] * 1e-3
     achieved = prof["sweep_bytes"] / loop_s / 1e9 if loop_s > 0 else 0.0
-    roofline = {"bound": "hbm", "kernel": "greedy_persistent_kernel", "achieved": achieved, "peak": peaks["hbm_gbs"],
+    roofline = {"bound": "hbm", "kernel": "greedy_persistent_kernel" if args.objective == "facility" else "cut_chain_kernel", "achieved": achieved, "peak": peaks["hbm_gbs"],
                 "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "peak_source": peaks["source"],
                 # dram__bytes_read.sum + dram__bytes_write.sum of one launch on the default C2 workload
                 # (ncu capture summarised in profiles/greedy_persistent_kernel_C2.md)
-                "traffic": 491.18e9 if (args.config == "C2" and args.sweep_batch in (0, 8) and args.greedy_path == 0 and args.similarity == "dot") else None,
+                "traffic": 491.18e9 if (args.config == "C2" and args.sweep_batch in (0, 8) and args.greedy_path == 0 and args.similarity == "dot" and args.objective == "facility") else None,
                 "launch_ms": prof["greedy_ms"], "bytes_per_launch": prof["sweep_bytes"],
                 "rounds_with_sweeps": int(prof["sweep_launches"])}
     # the same bytes against the time the kernel spends in its sweep phases (its own clock, CTA 0)
@@ -262,7 +263,8 @@ def run_ours(args):
                                     "pick_phases_ms": prof["persistent_pick_ns"] * 1e-6,
                                     "elem_block_ops_per_s": prof["sweep_elem_ops"] / (prof["persistent_sweep_ns"] * 1e-9)}
     # and with every round's sweep as a launch of its own (sweep_kernel), one CUDA-event pair each
-    ctx2 = rcd.Context(local, sweep_batch_max=args.sweep_batch, profile=2, similarity_kind=kind)
+    ctx2 = rcd.Context(local, sweep_batch_max=args.sweep_batch, profile=2, similarity_kind=kind,
+                       objective=rcd.RCD_OBJ_GRAPH_CUT if args.objective == "cut" else rcd.RCD_OBJ_FACILITY)
     ctx2.rcd_partition(Xd, yd, wl.capacities, wl.L, M_max=M)
     ctx2.sync_status()
     p2 = ctx2.profile()
@@ -289,10 +291,11 @@ def run_ours(args):
     result = {"metric": "samples partitioned/sec", "value": value, "unit": "samples/s", "n_gpus": world,
               "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps,
               "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-              "dtype": "int64" if (wl.dtype == "int8" and args.similarity == "dot") else "f32", "data": "synthetic",
+              "dtype": "int64" if (wl.dtype == "int8" and args.similarity == "dot") else ("f32" if args.objective == "facility" else "f64"),
+              "data": "synthetic",
               "config": {"workload": workload_name(args.config, wl),
                          "l2": "inputs larger than L2 (S is %.0f MB per class, re-read every sweep)" % (4e-6 * M * M),
-                         "sweep_batch_max": args.sweep_batch or 8, "similarity": args.similarity, "sharding": "one dataset per rank, no collective"},
+                         "sweep_batch_max": args.sweep_batch or 8, "similarity": args.similarity, "objective": args.objective, "sharding": "one dataset per rank, no collective"},
               "gain_evals_per_s": world * wl.L * M * (M + 1) / 2 * args.steps / (ms * 1e-3),
               "phases_ms": dict({k: prof[k] for k in ("group_ms", "similarity_ms", "greedy_ms", "total_ms")},
                                 sweep_phases_ms=prof["persistent_sweep_ns"] * 1e-6, pick_phases_ms=prof["persistent_pick_ns"] * 1e-6),
@@ -326,6 +329,7 @@ def main():
     ap.add_argument("--config", default="C2", choices=["C1", "C2", "C3", "C4", "C5"])
     ap.add_argument("--sweep-batch", type=int, default=0, help="sweep_batch_max (0 = library default)")
     ap.add_argument("--similarity", default="dot", choices=["dot", "gaussian"], help="similarity of Section 4 item 2")
+    ap.add_argument("--objective", default="facility", choices=["facility", "cut"], help="submodular function of Section 4 item 2")
     ap.add_argument("--greedy-path", type=int, default=0, help="0 = one cooperative launch, 1 = two launches per round")
     ap.add_argument("--ref-picks", type=int, default=150, help="picks per class in the CPU-oracle sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")

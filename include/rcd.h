@@ -64,6 +64,14 @@ typedef enum { RCD_FEAT_I8 = 0, RCD_FEAT_BF16 = 1 } rcd_feat_dtype;
  *                     (gains fp32, tracked f and all objective outputs double).  */
 typedef enum { RCD_SIM_DOT = 0, RCD_SIM_GAUSSIAN = 1 } rcd_similarity_kind;
 
+/* Submodular function f used by GreedyStep and by the argmin over blocks (Section 4 item 2).
+ *   RCD_OBJ_FACILITY   facility location, f(A) = sum_{v in V_l} max_{v' in A} sim(v, v') (clamped at 0);
+ *   RCD_OBJ_GRAPH_CUT  graph cut, f(A) = sum_{v in V_l \\ A} sum_{v' in A} sim(v, v').  Needs no pass over S per
+ *                      pick (the gain of u is a column sum minus twice its tie to the block); values are
+ *                      int64 for int8 features with RCD_SIM_DOT, double otherwise.  Not monotone: gains
+ *                      can be negative; Algorithm 1 runs unchanged. */
+typedef enum { RCD_OBJ_FACILITY = 0, RCD_OBJ_GRAPH_CUT = 1 } rcd_objective_kind;
+
 typedef struct {
     int32_t sweep_batch_max;   /* blocks whose gains one pass over S may refresh: 1,2,4 or 8; 0 = default (8) */
     int32_t similarity_path;   /* 0 = tensor-core kernel when the shape allows, 2 = always the generic kernel */
@@ -71,7 +79,8 @@ typedef struct {
     int32_t greedy_path;       /* 0 = whole greedy loop in one cooperative launch when the device allows;
                                   1 = two launches per greedy step (always used with profile 2) */
     int32_t similarity_kind;   /* rcd_similarity_kind used by rcd_partition / rcd_objective (default RCD_SIM_DOT) */
-    int32_t reserved[11];      /* must be 0 */
+    int32_t objective;         /* rcd_objective_kind used by rcd_partition / rcd_objective (default facility location) */
+    int32_t reserved[10];      /* must be 0 */
 } rcd_config;
 
 /* Timings and counters of the last rcd_partition / rcd_partition_host on a context (profile >= 1). */

@@ -24,6 +24,8 @@ RCD_FEAT_I8 = 0
 RCD_FEAT_BF16 = 1
 RCD_SIM_DOT = 0
 RCD_SIM_GAUSSIAN = 1
+RCD_OBJ_FACILITY = 0
+RCD_OBJ_GRAPH_CUT = 1
 
 STATUS_NAMES = {0: "RCD_OK", 1: "RCD_ERR_INVALID_ARG", 2: "RCD_ERR_UNSUPPORTED", 3: "RCD_ERR_WORKSPACE_TOO_SMALL",
                 4: "RCD_ERR_CUDA", 5: "RCD_ERR_TIMEOUT", 6: "RCD_ERR_INTERNAL"}
@@ -44,7 +46,7 @@ class RcdError(RuntimeError):
 
 class RcdConfig(C.Structure):
     _fields_ = [("sweep_batch_max", C.c_int32), ("similarity_path", C.c_int32), ("profile", C.c_int32),
-                ("greedy_path", C.c_int32), ("similarity_kind", C.c_int32), ("reserved", C.c_int32 * 11)]
+                ("greedy_path", C.c_int32), ("similarity_kind", C.c_int32), ("objective", C.c_int32), ("reserved", C.c_int32 * 10)]
 
 
 class RcdProfile(C.Structure):
@@ -139,7 +141,7 @@ class Context:
     """Owns one ``rcd_ctx`` on a CUDA device."""
 
     def __init__(self, device: int = 0, sweep_batch_max: int = 0, similarity_path: int = 0, profile: int = 0,
-                 greedy_path: int = 0, similarity_kind: int = 0):
+                 greedy_path: int = 0, similarity_kind: int = 0, objective: int = 0):
         torch = _torch()
         if not torch.cuda.is_available():
             raise RcdError(4, "no CUDA device: this library has no CPU path")
@@ -151,6 +153,7 @@ class Context:
         cfg.profile = profile
         cfg.greedy_path = greedy_path
         cfg.similarity_kind = similarity_kind
+        cfg.objective = objective
         self.similarity_kind = similarity_kind
         self._h = C.c_void_p()
         st = lib.rcd_create(C.byref(self._h), self.device, C.byref(cfg))

@@ -49,7 +49,7 @@ size_t layout_workspace(void *base, rcd_feat_dtype dtype, const Sizes &sz, Works
     const size_t L = (size_t)std::max<int32_t>(sz.L, 1), W = (size_t)std::max<int32_t>(sz.W, 1);
     const size_t N = (size_t)std::max<int64_t>(sz.N, 1);
     const size_t sElem = 4;                                     // int32 / fp32
-    const size_t gElem = sz.floatArith ? 4 : 8;                 // fp32 / int64
+    const size_t gElem = (sz.floatArith && !sz.graphCut) ? 4 : 8;   // fp32 gains / int64 gains, or 8-byte ties
     Workspace w{};
     // the head does not depend on the class sizes: it is used before they are known
     w.status = c.take<int32_t>(4);
@@ -66,6 +66,7 @@ size_t layout_workspace(void *base, rcd_feat_dtype dtype, const Sizes &sz, Works
     w.gaussPartial = c.take<double>(L * (size_t)((sz.maxM + 63) / 64 + 1));
     w.gaussSigma = c.take<float>(L);
     w.gaussScale = c.take<float>(L);
+    w.cutBase = c.take<unsigned char>(sz.graphCut ? N * 8 : 8);
     w.cover = c.take<unsigned char>((size_t)std::max<int64_t>(sz.vElems, 1) * sElem);
     w.gains = c.take<unsigned char>((size_t)std::max<int64_t>(sz.vElems, 1) * gElem);
     w.fval = c.take<unsigned char>(L * W * 8);
@@ -101,6 +102,7 @@ static Sizes bound_sizes(const rcd_ctx *ctx, rcd_feat_dtype dtype, int64_t N, in
 {
     Sizes sz{};
     sz.floatArith = float_arith(ctx, dtype);
+    sz.graphCut = ctx->cfg.objective == RCD_OBJ_GRAPH_CUT;
     sz.N = N; sz.d = d; sz.L = L; sz.W = W;
     if (Mmax > N) Mmax = N;
     sz.maxM = Mmax;
@@ -181,6 +183,7 @@ static rcd_status prepare(rcd_ctx *ctx, const void *features, rcd_feat_dtype dty
     Sizes head{};
     head.N = N; head.d = d; head.L = L; head.W = W; head.nChunks = chunks_for(N);
     head.floatArith = float_arith(ctx, dtype);
+    head.graphCut = ctx->cfg.objective == RCD_OBJ_GRAPH_CUT;
     Workspace hw{};
     Sizes tiny = head;
     layout_workspace(workspace, dtype, tiny, &hw);
@@ -279,7 +282,8 @@ rcd_status rcd_create(rcd_ctx **out, int cuda_device, const rcd_config *cfg)
         if (cfg->profile < 0 || cfg->profile > 2) return RCD_ERR_INVALID_ARG;
         if (cfg->greedy_path != 0 && cfg->greedy_path != 1) return RCD_ERR_INVALID_ARG;
         if (cfg->similarity_kind != RCD_SIM_DOT && cfg->similarity_kind != RCD_SIM_GAUSSIAN) return RCD_ERR_INVALID_ARG;
-        for (int i = 0; i < 11; ++i) if (cfg->reserved[i] != 0) return RCD_ERR_INVALID_ARG;
+        if (cfg->objective != RCD_OBJ_FACILITY && cfg->objective != RCD_OBJ_GRAPH_CUT) return RCD_ERR_INVALID_ARG;
+        for (int i = 0; i < 10; ++i) if (cfg->reserved[i] != 0) return RCD_ERR_INVALID_ARG;
     }
     int count = 0;
     if (cudaGetDeviceCount(&count) != cudaSuccess || cuda_device < 0 || cuda_device >= count) {
@@ -495,7 +499,8 @@ rcd_status rcd_partition(rcd_ctx *ctx, const void *features_dev, rcd_feat_dtype 
     for (int32_t l = 0; l < L; ++l) quotas_host(P.desc[(size_t)l].M, capacities_host, W, quota.data() + (size_t)l * W);
     RCD_CUDA(ctx, cudaMemcpyAsync(P.ws.quota, quota.data(), quota.size() * sizeof(int32_t), cudaMemcpyHostToDevice, st));
 
-    rs = launch_greedy(ctx, P.sz.floatArith ? RCD_FEAT_BF16 : RCD_FEAT_I8, P.sz, P.ws, P.desc, assignment_dev, order_dev_or_null, st);
+    if (P.sz.graphCut) rs = launch_cut(ctx, P.sz, P.ws, assignment_dev, order_dev_or_null, st);
+    else rs = launch_greedy(ctx, P.sz.floatArith ? RCD_FEAT_BF16 : RCD_FEAT_I8, P.sz, P.ws, P.desc, assignment_dev, order_dev_or_null, st);
     if (rs != RCD_OK) return rs;
     if (prof) RCD_CUDA(ctx, cudaEventRecord(ctx->evPhase[3], st));
     if (part_values_dev_or_null) {
@@ -612,6 +617,8 @@ rcd_status rcd_objective(rcd_ctx *ctx, const void *features_dev, rcd_feat_dtype 
     if (P.ws.bytes + scratchB > workspace_bytes)
         return fail(ctx, RCD_ERR_WORKSPACE_TOO_SMALL, "workspace has %zu bytes, objective needs %zu", workspace_bytes, P.ws.bytes + scratchB);
     void *scratch = (unsigned char *)workspace_dev + P.ws.bytes;
+    if (P.sz.graphCut)
+        return launch_cut_objective(ctx, P.sz, P.ws.desc, P.ws.S, P.ws.perm, assignment_dev, part_values_dev, total_dev, scratch, st);
     return launch_objective(ctx, P.sz.floatArith ? RCD_FEAT_BF16 : RCD_FEAT_I8, P.sz, P.ws.desc, P.desc, P.ws.S, P.ws.perm, assignment_dev, part_values_dev,
                             total_dev, scratch, st);
 }

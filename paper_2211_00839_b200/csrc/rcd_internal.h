@@ -76,6 +76,7 @@ struct Workspace {
     double *gaussPartial;   // [L][ceil(maxM/64)] per-row-block sums of pairwise distances
     float *gaussSigma;      // [L] bandwidth of every class
     float *gaussScale;      // [L] 1 / (2 sigma^2)
+    void *cutBase;          // [N] graph cut: column sum minus diagonal of every sample (int64 / double)
     void *cover;            // [sum W*ld] coverage vectors (int32 / float)
     void *gains;            // [sum W*ld] stored gains (int64 / float)
     void *fval;             // [L][W] tracked f (int64 / double)
@@ -107,6 +108,7 @@ struct Sizes {
     int64_t maxM;
     int32_t nChunks;
     bool floatArith;        // fp32 S / fp32 gains / double f (bf16 features, or the Gaussian kernel)
+    bool graphCut;          // graph-cut objective: the gains array holds 8-byte ties
 };
 
 constexpr int kGroupChunk = 1024;           // samples per chunk of the stable class split
@@ -178,6 +180,11 @@ size_t gaussian_scratch_bytes(int64_t N, int32_t L, int64_t maxM);
 rcd_status launch_greedy(rcd_ctx *ctx, rcd_feat_dtype dtype, const Sizes &sz, const Workspace &ws,
                          const std::vector<ClassDesc> &descHost, int32_t *assignment, int32_t *order,
                          cudaStream_t st);
+
+// graph-cut objective: the whole greedy loop, and f from an assignment
+rcd_status launch_cut(rcd_ctx *ctx, const Sizes &sz, const Workspace &ws, int32_t *assignment, int32_t *order, cudaStream_t st);
+rcd_status launch_cut_objective(rcd_ctx *ctx, const Sizes &sz, const ClassDesc *descDev, const void *S, const int32_t *perm,
+                                const int32_t *assignment, void *partValues, void *total, void *scratch, cudaStream_t st);
 
 // objective from an assignment
 rcd_status launch_objective(rcd_ctx *ctx, rcd_feat_dtype dtype, const Sizes &sz, const ClassDesc *descDev,
