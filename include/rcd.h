@@ -116,6 +116,11 @@ RCD_API const char *rcd_version(void);
 
 /* Waits for `cuda_stream` and returns the device-side status of the last call on the context. */
 RCD_API rcd_status rcd_sync_status(rcd_ctx *ctx, void *cuda_stream);
+/* Self-test of the bounded waits the kernels use (grid barrier of the greedy loop, mbarrier waits of the
+ * tensor-core kernel): enqueues a one-CTA kernel that arrives at a barrier expecting two arrivals.  The wait
+ * gives up after a few thousand polls and records the timeout in the context's status word, so the next
+ * rcd_sync_status returns RCD_ERR_TIMEOUT and the context stays usable.  Nothing faults or hangs. */
+RCD_API rcd_status rcd_selftest_bounded_wait(rcd_ctx *ctx, void *cuda_stream);
 /* Waits for the events of the last profiled call and fills `out`. */
 RCD_API rcd_status rcd_get_profile(rcd_ctx *ctx, rcd_profile *out);
 

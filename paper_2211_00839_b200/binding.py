@@ -31,7 +31,7 @@ STATUS_NAMES = {0: "RCD_OK", 1: "RCD_ERR_INVALID_ARG", 2: "RCD_ERR_UNSUPPORTED",
                 4: "RCD_ERR_CUDA", 5: "RCD_ERR_TIMEOUT", 6: "RCD_ERR_INTERNAL"}
 
 # every symbol include/rcd.h declares
-EXPORTS = ["rcd_create", "rcd_destroy", "rcd_last_error", "rcd_version", "rcd_sync_status", "rcd_get_profile",
+EXPORTS = ["rcd_create", "rcd_destroy", "rcd_last_error", "rcd_version", "rcd_sync_status", "rcd_selftest_bounded_wait", "rcd_get_profile",
            "rcd_quotas", "rcd_similarity", "rcd_similarity_gaussian_workspace_bytes", "rcd_similarity_gaussian",
            "rcd_partition_workspace_bytes", "rcd_partition",
            "rcd_partition_host_workspace_bytes", "rcd_partition_host", "rcd_objective_workspace_bytes",
@@ -71,6 +71,7 @@ def _load() -> C.CDLL:
     lib.rcd_version.argtypes = []
     lib.rcd_version.restype = C.c_char_p
     lib.rcd_sync_status.argtypes = [vp, vp]
+    lib.rcd_selftest_bounded_wait.argtypes = [vp, vp]
     lib.rcd_get_profile.argtypes = [vp, C.POINTER(RcdProfile)]
     lib.rcd_quotas.argtypes = [i64, vp, i32, vp]
     lib.rcd_similarity.argtypes = [vp, vp, C.c_int, i64, i64, i64, vp, i64, vp]
@@ -193,6 +194,10 @@ class Context:
             self._ws = None
             self._ws = torch.empty(int(nbytes), dtype=torch.uint8, device=self.torch_device)
         return self._ws
+
+    def selftest_bounded_wait(self):
+        """Enqueue the wait that can never be satisfied; the following sync_status() raises RCD_ERR_TIMEOUT."""
+        self._check(lib.rcd_selftest_bounded_wait(self._h, self._stream()))
 
     def sync_status(self):
         self._check(lib.rcd_sync_status(self._h, self._stream()))

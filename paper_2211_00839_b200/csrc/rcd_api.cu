@@ -341,6 +341,16 @@ rcd_status rcd_sync_status(rcd_ctx *ctx, void *cuda_stream)
     return fail(ctx, RCD_ERR_INTERNAL, "device status %d: greedy state inconsistent", word);
 }
 
+rcd_status rcd_selftest_bounded_wait(rcd_ctx *ctx, void *cuda_stream)
+{
+    if (!ctx) return RCD_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    RCD_CUDA(ctx, cudaSetDevice(ctx->device));
+    RCD_CUDA(ctx, cudaMemsetAsync(ctx->statusOwn, 0, 64, st));
+    ctx->statusDev = ctx->statusOwn;
+    return launch_bounded_wait_selftest(ctx, (unsigned *)(ctx->statusOwn + 8), ctx->statusOwn, st);
+}
+
 rcd_status rcd_get_profile(rcd_ctx *ctx, rcd_profile *out)
 {
     if (!ctx || !out) return RCD_ERR_INVALID_ARG;

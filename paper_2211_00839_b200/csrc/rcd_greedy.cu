@@ -555,6 +555,36 @@ __global__ void __launch_bounds__(kSweepThreads, 1) sweep_kernel(GreedyParams<SV
 }
 
 // ---------------------------------------------------------------------------------------------
+// Element-wise maximum of two 16-byte pieces (int32 or fp32 lanes).
+template <typename SV>
+__device__ __forceinline__ int4 max_int4(int4 a, int4 b)
+{
+    if constexpr (Arith<SV>::kInt) {
+        a.x = max(a.x, b.x); a.y = max(a.y, b.y); a.z = max(a.z, b.z); a.w = max(a.w, b.w);
+    } else {
+        a.x = __float_as_int(fmaxf(__int_as_float(a.x), __int_as_float(b.x)));
+        a.y = __float_as_int(fmaxf(__int_as_float(a.y), __int_as_float(b.y)));
+        a.z = __float_as_int(fmaxf(__int_as_float(a.z), __int_as_float(b.z)));
+        a.w = __float_as_int(fmaxf(__int_as_float(a.w), __int_as_float(b.w)));
+    }
+    return a;
+}
+
+// 16 bytes global -> shared without passing through registers (completion: cp.async.wait_group).
+__device__ __forceinline__ void async_copy16(int4 *smemDst, const int4 *src)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" :: "r"((uint32_t)__cvta_generic_to_shared(smemDst)), "l"(src) : "memory");
+}
+
+// Finishes a coverage update whose operands were copied to shared memory earlier (row v* in
+// scratch[0, ld4), the old coverage in scratch[ld4, 2 ld4)): dst[i] = max of the two.
+template <typename SV>
+__device__ __forceinline__ void fold_pending(int4 *dst, const int4 *scratch, int ld4)
+{
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    for (int i = threadIdx.x; i < ld4; i += kSelectThreads) dst[i] = max_int4<SV>(scratch[ld4 + i], scratch[i]);
+}
+
 // The picks of class l in round `round`, by one CTA of kSelectThreads threads: pick after pick
 // (GreedyStep's argmax over the stored gains of the chosen block, then the bookkeeping of
 // Algorithm 1's "A := A u {v*}, R := R \ {v*}" and the choice of the next block) until the next
@@ -562,7 +592,7 @@ __global__ void __launch_bounds__(kSweepThreads, 1) sweep_kernel(GreedyParams<SV
 // is finished.  Inside the chain nothing waits on the coverage update: a pick only needs stored
 // gains, so row v* is folded into the coverage vector while the next block is being chosen.
 template <typename SV>
-__device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, int round)
+__device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, int round, int4 *scratch, int scratchBytes)
 {
     using GV = typename Arith<SV>::GV;
     using FV = typename Arith<SV>::FV;
@@ -581,6 +611,12 @@ __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, i
     int32_t *pos = prm.pos + c.row0;
     plan_load(prm, l, shPlan);
     __syncthreads();
+    // Folding row v* into the coverage vector is off the critical path (a pick reads stored gains,
+    // never the coverage).  When the caller lends enough shared memory, row v* and the coverage
+    // vector are fetched with asynchronous copies once v* is known, and the max/store happens one
+    // pick later, after the next argmax; each thread consumes exactly the pieces it copied.
+    const bool defer = scratch != nullptr && (int64_t)2 * c.ld * (int64_t)sizeof(SV) <= scratchBytes;
+    int4 *pendDst = nullptr;
 
     for (;;) {
         const GV *G = prm.gains + c.vOff + (int64_t)j * c.ld;
@@ -607,6 +643,10 @@ __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, i
                 const int v = v0 + i * kSelectThreads;
                 if (ps[i] >= 0 && (bestV == INT_MAX || g[i] > bestG)) { bestG = g[i]; bestV = v; }
             }
+        }
+        if (pendDst) {                                  // finish the previous pick's coverage update
+            fold_pending<SV>(pendDst, scratch, ld4);
+            pendDst = nullptr;
         }
         for (int off = 16; off > 0; off >>= 1) {
             GV oG = __shfl_xor_sync(0xffffffffu, bestG, off);
@@ -640,7 +680,7 @@ __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, i
         const int vstar = shPick;
         if (vstar == INT_MAX || vstar < 0 || vstar >= c.M) {
             if (threadIdx.x == 0) atomicOr(prm.status, kDevBadState);
-            return;
+            break;
         }
         // warp 0: next block (shared memory only).  last warp: global bookkeeping of this pick.
         // everybody else meanwhile starts fetching row v* and the coverage vector.
@@ -664,24 +704,23 @@ __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, i
             if (nR == 1) atomicSub(&prm.nSweep[3], 1);        // one class fewer to finish
         }
         // cover_j <- max(cover_j, S[v*][.])
-#pragma unroll 2
-        for (int i = threadIdx.x; i < ld4; i += kSelectThreads) {
-            int4 a = cov[i], b = row[i];
-            if constexpr (Arith<SV>::kInt) {
-                a.x = max(a.x, b.x); a.y = max(a.y, b.y); a.z = max(a.z, b.z); a.w = max(a.w, b.w);
-            } else {
-                a.x = __float_as_int(fmaxf(__int_as_float(a.x), __int_as_float(b.x)));
-                a.y = __float_as_int(fmaxf(__int_as_float(a.y), __int_as_float(b.y)));
-                a.z = __float_as_int(fmaxf(__int_as_float(a.z), __int_as_float(b.z)));
-                a.w = __float_as_int(fmaxf(__int_as_float(a.w), __int_as_float(b.w)));
+        if (defer) {
+            for (int i = threadIdx.x; i < ld4; i += kSelectThreads) {
+                async_copy16(scratch + i, row + i);
+                async_copy16(scratch + ld4 + i, cov + i);
             }
-            cov[i] = a;
+            asm volatile("cp.async.commit_group;" ::: "memory");
+            pendDst = cov;
+        } else {
+#pragma unroll 2
+            for (int i = threadIdx.x; i < ld4; i += kSelectThreads) cov[i] = max_int4<SV>(cov[i], row[i]);
         }
         __syncthreads();
         nR -= 1;
         j = shPlan.nextJ;
-        if (nR == 0 || j < 0 || shPlan.needSweep) return;
+        if (nR == 0 || j < 0 || shPlan.needSweep) break;
     }
+    if (pendDst) fold_pending<SV>(pendDst, scratch, ld4);
 }
 
 // Picks of round `round`: every class advances until it needs a sweep (or is finished).
@@ -690,7 +729,7 @@ __global__ void __launch_bounds__(kSelectThreads, 2) chain_kernel(GreedyParams<S
 {
     cudaGridDependencySynchronize();              // the sweep of this round has finished
     cudaTriggerProgrammaticLaunchCompletion();
-    pick_chain(prm, blockIdx.x, round);
+    pick_chain(prm, blockIdx.x, round, nullptr, 0);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -703,8 +742,9 @@ __global__ void __launch_bounds__(kSelectThreads, 2) chain_kernel(GreedyParams<S
 // another CTA has already reported that) the timeout bit is set in the status word and the caller
 // leaves its loop.  Thread 0's fences order this CTA's writes before its arrival and make the other
 // CTAs' writes visible after the wait (the fence drops stale L1 lines of this SM).
-constexpr unsigned kBarrierSpinLimit = 1u << 26;
-__device__ __forceinline__ bool grid_barrier(unsigned *counter, unsigned expected, int32_t *status)
+constexpr unsigned kBarrierSpinLimit = 1u << 21;       // polls of about a microsecond each: a second or two
+__device__ __forceinline__ bool grid_barrier(unsigned *counter, unsigned expected, int32_t *status,
+                                             unsigned spinLimit = kBarrierSpinLimit)
 {
     __shared__ int shOk;
     __syncthreads();
@@ -714,7 +754,7 @@ __device__ __forceinline__ bool grid_barrier(unsigned *counter, unsigned expecte
         int ok = 1;
         unsigned spins = 0;
         while (*(volatile unsigned *)counter < expected) {
-            if ((++spins & 1023u) == 0 && ((*(volatile int32_t *)status & kDevTimeout) || spins >= kBarrierSpinLimit)) {
+            if ((++spins & 1023u) == 0 && ((*(volatile int32_t *)status & kDevTimeout) || spins >= spinLimit)) {
                 atomicOr(status, kDevTimeout);
                 ok = 0;
                 break;
@@ -753,7 +793,7 @@ __global__ void __launch_bounds__(kSweepThreads, 1) greedy_persistent_kernel(Gre
             shClock[0] = t1;
         }
         for (int l = blockIdx.x; l < prm.L; l += gridDim.x) {
-            pick_chain(prm, l, r);
+            pick_chain(prm, l, r, shCover, prm.smemBytes);       // the sweep's shared memory is idle in this phase
             __syncthreads();
         }
         if (!grid_barrier(prm.barrier, (unsigned)(2 * r + 2) * gridDim.x, prm.status)) break;   // picks of round r, sweep list of round r+1
@@ -895,6 +935,22 @@ static rcd_status run_greedy(rcd_ctx *ctx, const Sizes &sz, const Workspace &ws,
     ctx->steps = sz.maxM;
     ctx->stepBytesDev = ws.stepBytes;
     ctx->stepOpsDev = ws.stepOps;
+    return RCD_OK;
+}
+
+// One CTA arrives at a barrier that expects two: the bounded wait must run out, set the timeout
+// bit and return (used by rcd_selftest_bounded_wait to show that a wait which can never be
+// satisfied ends as an error status, not as a hang).
+__global__ void bounded_wait_selftest_kernel(unsigned *counter, int32_t *status)
+{
+    grid_barrier(counter, 2u, status, 1u << 12);
+}
+
+rcd_status launch_bounded_wait_selftest(rcd_ctx *ctx, unsigned *counter, int32_t *status, cudaStream_t st)
+{
+    bounded_wait_selftest_kernel<<<1, 64, 0, st>>>(counter, status);
+    ctx->kernelLaunches++;
+    RCD_CUDA(ctx, cudaGetLastError());
     return RCD_OK;
 }
 

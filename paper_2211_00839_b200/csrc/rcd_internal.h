@@ -181,6 +181,8 @@ rcd_status launch_greedy(rcd_ctx *ctx, rcd_feat_dtype dtype, const Sizes &sz, co
                          const std::vector<ClassDesc> &descHost, int32_t *assignment, int32_t *order,
                          cudaStream_t st);
 
+rcd_status launch_bounded_wait_selftest(rcd_ctx *ctx, unsigned *counter, int32_t *status, cudaStream_t st);
+
 // graph-cut objective: the whole greedy loop, and f from an assignment
 rcd_status launch_cut(rcd_ctx *ctx, const Sizes &sz, const Workspace &ws, int32_t *assignment, int32_t *order, cudaStream_t st);
 rcd_status launch_cut_objective(rcd_ctx *ctx, const Sizes &sz, const ClassDesc *descDev, const void *S, const int32_t *perm,

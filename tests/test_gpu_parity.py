@@ -295,3 +295,20 @@ def test_empty_input(rcd):
         a, o, v = ctx.rcd_partition(X, y, [1.0, 2.0], 3)
         ctx.sync_status()
         assert a.numel() == 0 and v.shape == (3, 2) and int(v.abs().sum()) == 0
+
+
+def test_bounded_wait_times_out_as_a_status_not_a_hang(rcd):
+    """A device-side wait that nothing can satisfy ends after its poll limit and surfaces as
+    RCD_ERR_TIMEOUT; the context and the GPU stay usable."""
+    import torch
+    from paper_2211_00839_b200.workloads import make_workload
+    wl = make_workload("C1")
+    with rcd.Context(0) as ctx:
+        ctx.selftest_bounded_wait()
+        with pytest.raises(rcd.RcdError) as e:
+            ctx.sync_status()
+        assert e.value.status == 5          # RCD_ERR_TIMEOUT
+        X, y = to_device(rcd, wl)
+        a, o, v = ctx.rcd_partition(X, y, wl.capacities, wl.L)
+        ctx.sync_status()                   # clean again
+        assert int(a.min()) >= 0
