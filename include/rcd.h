@@ -80,7 +80,9 @@ typedef struct {
                                   1 = two launches per greedy step (always used with profile 2) */
     int32_t similarity_kind;   /* rcd_similarity_kind used by rcd_partition / rcd_objective (default RCD_SIM_DOT) */
     int32_t objective;         /* rcd_objective_kind used by rcd_partition / rcd_objective (default facility location) */
-    int32_t reserved[10];      /* must be 0 */
+    int32_t sweep_mode;        /* 0 = threshold passes once the blocks have a few members (up to 64 blocks per pass);
+                                  1 = dense passes only (sweep_batch_max blocks per pass) */
+    int32_t reserved[9];       /* must be 0 */
 } rcd_config;
 
 /* Timings and counters of the last rcd_partition / rcd_partition_host on a context (profile >= 1). */
@@ -98,7 +100,9 @@ typedef struct {
     int64_t similarity_tc_launches; /* similarity launches of the last call that ran on the tensor cores */
     int64_t persistent_sweep_ns;    /* one-launch greedy loop: time in sweep phases (incl. their barrier) */
     int64_t persistent_pick_ns;     /* one-launch greedy loop: time in pick phases (incl. their barrier) */
-    int64_t reserved[3];
+    int64_t threshold_hits;         /* threshold passes: elements of S above the threshold ... */
+    int64_t threshold_elems;        /* ... out of this many elements compared */
+    int64_t threshold_max_blocks;   /* most blocks one threshold pass refreshed */
 } rcd_profile;
 
 typedef struct rcd_ctx rcd_ctx;

@@ -46,7 +46,7 @@ class RcdError(RuntimeError):
 
 class RcdConfig(C.Structure):
     _fields_ = [("sweep_batch_max", C.c_int32), ("similarity_path", C.c_int32), ("profile", C.c_int32),
-                ("greedy_path", C.c_int32), ("similarity_kind", C.c_int32), ("objective", C.c_int32), ("reserved", C.c_int32 * 10)]
+                ("greedy_path", C.c_int32), ("similarity_kind", C.c_int32), ("objective", C.c_int32), ("sweep_mode", C.c_int32), ("reserved", C.c_int32 * 9)]
 
 
 class RcdProfile(C.Structure):
@@ -54,7 +54,8 @@ class RcdProfile(C.Structure):
                 ("greedy_ms", C.c_double), ("sweep_ms", C.c_double), ("sweep_launches", C.c_int64),
                 ("sweep_bytes", C.c_int64), ("sweep_elem_ops", C.c_int64), ("kernel_launches", C.c_int64),
                 ("steps", C.c_int64), ("similarity_tc_launches", C.c_int64), ("persistent_sweep_ns", C.c_int64),
-                ("persistent_pick_ns", C.c_int64), ("reserved", C.c_int64 * 3)]
+                ("persistent_pick_ns", C.c_int64), ("threshold_hits", C.c_int64),
+                ("threshold_elems", C.c_int64), ("threshold_max_blocks", C.c_int64)]
 
 
 def _load() -> C.CDLL:
@@ -142,7 +143,7 @@ class Context:
     """Owns one ``rcd_ctx`` on a CUDA device."""
 
     def __init__(self, device: int = 0, sweep_batch_max: int = 0, similarity_path: int = 0, profile: int = 0,
-                 greedy_path: int = 0, similarity_kind: int = 0, objective: int = 0):
+                 greedy_path: int = 0, similarity_kind: int = 0, objective: int = 0, sweep_mode: int = 0):
         torch = _torch()
         if not torch.cuda.is_available():
             raise RcdError(4, "no CUDA device: this library has no CPU path")
@@ -155,6 +156,7 @@ class Context:
         cfg.greedy_path = greedy_path
         cfg.similarity_kind = similarity_kind
         cfg.objective = objective
+        cfg.sweep_mode = sweep_mode
         self.similarity_kind = similarity_kind
         self._h = C.c_void_p()
         st = lib.rcd_create(C.byref(self._h), self.device, C.byref(cfg))

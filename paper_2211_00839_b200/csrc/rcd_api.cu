@@ -78,13 +78,18 @@ size_t layout_workspace(void *base, rcd_feat_dtype dtype, const Sizes &sz, Works
     w.nR = c.take<int32_t>(L);
     w.jstar = c.take<int32_t>(L);
     w.sweepN = c.take<int32_t>(L);
-    w.sweepParts = c.take<int32_t>(L * kMaxSweepBatch);
+    w.sweepParts = c.take<int32_t>(L * kSparseMax);
+    w.sweepMode = c.take<int32_t>(L);
+    w.thr = c.take<unsigned char>((size_t)std::max<int64_t>(sz.vElems / (int64_t)W, 1) * sElem + 64);
+    w.hitCount = c.take<unsigned long long>(L);
+    w.sparseElems = c.take<unsigned long long>(L);
+    w.sparseFrom = c.take<int32_t>(L);
     w.sweepCS = c.take<int32_t>(L);
     w.rowCtr = c.take<int32_t>(L);
     w.sweepList = c.take<int32_t>(3 * L);
     w.stepBytes = c.take<unsigned long long>((size_t)sz.maxM + 1);
     w.stepOps = c.take<unsigned long long>((size_t)sz.maxM + 1);
-    w.phaseNs = c.take<unsigned long long>(3);      // two phase clocks + the grid-barrier counter
+    w.phaseNs = c.take<unsigned long long>(6);      // two phase clocks, the grid-barrier counter, threshold-pass hits / elements
     w.bytes = align_up(c.off);
     if (ws) *ws = w;
     return w.bytes;
@@ -283,7 +288,8 @@ rcd_status rcd_create(rcd_ctx **out, int cuda_device, const rcd_config *cfg)
         if (cfg->greedy_path != 0 && cfg->greedy_path != 1) return RCD_ERR_INVALID_ARG;
         if (cfg->similarity_kind != RCD_SIM_DOT && cfg->similarity_kind != RCD_SIM_GAUSSIAN) return RCD_ERR_INVALID_ARG;
         if (cfg->objective != RCD_OBJ_FACILITY && cfg->objective != RCD_OBJ_GRAPH_CUT) return RCD_ERR_INVALID_ARG;
-        for (int i = 0; i < 10; ++i) if (cfg->reserved[i] != 0) return RCD_ERR_INVALID_ARG;
+        if (cfg->sweep_mode != 0 && cfg->sweep_mode != 1) return RCD_ERR_INVALID_ARG;
+        for (int i = 0; i < 9; ++i) if (cfg->reserved[i] != 0) return RCD_ERR_INVALID_ARG;
     }
     int count = 0;
     if (cudaGetDeviceCount(&count) != cudaSuccess || cuda_device < 0 || cuda_device >= count) {
@@ -366,10 +372,13 @@ rcd_status rcd_get_profile(rcd_ctx *ctx, rcd_profile *out)
     RCD_CUDA(ctx, cudaEventElapsedTime(&ms, ctx->evPhase[1], ctx->evPhase[2])); out->similarity_ms = ms;
     RCD_CUDA(ctx, cudaEventElapsedTime(&ms, ctx->evPhase[2], ctx->evPhase[3])); out->greedy_ms = ms;
     if (ctx->phaseNsDev) {
-        unsigned long long ns[2] = {0, 0};
+        unsigned long long ns[6] = {0, 0, 0, 0, 0, 0};
         RCD_CUDA(ctx, cudaMemcpy(ns, ctx->phaseNsDev, sizeof ns, cudaMemcpyDeviceToHost));
         out->persistent_sweep_ns = (int64_t)ns[0];
         out->persistent_pick_ns = (int64_t)ns[1];
+        out->threshold_hits = (int64_t)ns[3];
+        out->threshold_elems = (int64_t)ns[4];
+        out->threshold_max_blocks = (int64_t)ns[5];
     }
     if (ctx->stepBytesDev && ctx->steps > 0) {
         std::vector<unsigned long long> bytes((size_t)ctx->steps + 1), ops((size_t)ctx->steps + 1);

@@ -48,8 +48,11 @@ __global__ void __launch_bounds__(kCutThreads, 2) cut_chain_kernel(CutParams<SV>
     __shared__ int shPick, shBlock;
     const int l = blockIdx.x;
     const ClassDesc c = prm.desc[l];
-    if (c.M == 0) return;
     const int W = prm.W;
+    if (c.M == 0) {                                           // empty class: every block has value 0
+        for (int p = threadIdx.x; p < W; p += kCutThreads) prm.fval[(int64_t)l * W + p] = 0;
+        return;
+    }
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const SV *Sl = prm.S + c.sOff;
     FV *base = prm.base + c.row0;

@@ -57,14 +57,20 @@ struct GreedyParams {
     int32_t *nR;
     int32_t *jstar;
     int32_t *sweepN;
-    int32_t *sweepParts;
+    int32_t *sweepParts;    // [L][kSparseMax] blocks the class's next sweep refreshes
+    int32_t *sweepMode;     // [L] 0 = dense pass (coverage vectors in shared memory), 1 = threshold pass
+    SV *thr;                // per class [ld]: min over the listed blocks of their coverage (threshold pass)
+    unsigned long long *hitCount;   // [L] elements above the threshold in the class's last threshold pass
+    unsigned long long *sparseElems; // [L] elements that pass compared (0: the last pass was dense)
+    int32_t *sparseFrom;    // [L] members every out-of-date block must have before the next threshold pass is tried
     int32_t *sweepCS;       // warps that share one row group in the next sweep (1, 2, 4, 8 or 16)
     int32_t *rowCtr;
     int32_t *sweepList;
     int32_t *nSweep;
     unsigned long long *stepBytes;
     unsigned long long *stepOps;
-    unsigned long long *phaseNs;    // [2] time block 0 spent in sweep phases / pick phases (persistent kernel)
+    unsigned long long *phaseNs;    // [0..1] time block 0 spent in sweep / pick phases (persistent kernel), [2] grid-barrier
+                                    // counter, [3..5] threshold passes: elements above the threshold / elements compared / most blocks in one pass
     unsigned *barrier;              // arrival counter of the persistent kernel's grid barrier
     int32_t *status;
     const int32_t *perm;
@@ -76,6 +82,7 @@ struct GreedyParams {
     int32_t segIters;       // int path: chunk iterations a 32-bit partial sum can take without overflow
     int32_t sweepWarps;     // warps of one sweep launch (CTAs x 16)
     uint32_t one;           // the value 1, opaque to the compiler (see accumulate_chunk)
+    int32_t sparseMinMembers;   // threshold passes start once every out-of-date block has this many members (<0: never)
 };
 
 __host__ __device__ inline int rows_per_group(int P) { return P == 8 ? 4 : 8; }
@@ -92,6 +99,8 @@ struct PlanShared {
     uint8_t open[kMaxBlocks];      // bit 0: block is not full, bit 1: its stored gains are out of date
     int32_t nextJ;                 // plan_decide's answer: block of the next pick (-1: none)
     int32_t needSweep;             //                       1 = that pick must wait for a sweep
+    int32_t sweepBlocks;           //                       blocks in the scheduled sweep's list
+    int32_t sweepSparse;           //                       1 = the scheduled sweep is a threshold pass
 };
 
 template <typename SV>
@@ -108,6 +117,13 @@ __device__ __forceinline__ void plan_load(const GreedyParams<SV> &prm, int l, Pl
 }
 
 // Warp 0 only.  nR = samples of the class still unassigned.
+constexpr int kSparseQueue = 256;                                  // threshold pass: queue entries per warp
+constexpr int kSparseRows = 2;                                     // threshold pass: rows per warp and ticket
+constexpr int kSparseStages = 8;                                   // threshold pass: ring of chunks of S per warp
+constexpr int kSparseRingBytes = kSparseStages * kSparseRows * 512;   // rows x 32 lanes x 16 bytes per stage
+constexpr int kSparseWarpBytes = kSparseRingBytes + kSparseQueue * 8; // ring + queue
+constexpr int kSparseQueueBytes = kSparseWarpBytes * (kSweepThreads / 32);
+
 template <typename SV>
 __device__ void plan_decide(const GreedyParams<SV> &prm, int l, const ClassDesc &c, int nR, int nextStep,
                             PlanShared<typename Arith<SV>::FV> &sh)
@@ -125,18 +141,23 @@ __device__ void plan_decide(const GreedyParams<SV> &prm, int l, const ClassDesc 
     FV bestF = 0;
     int bestP = INT_MAX;
     int nStale = 0;
+    int fewest = INT_MAX;                          // members of the emptiest out-of-date non-full block
     for (int p = lane; p < W; p += 32) {
         const uint8_t o = sh.open[p];
         if (o & 1) {
             const FV fp = sh.f[p];
             if (bestP == INT_MAX || fp < bestF) { bestF = fp; bestP = p; }
-            if (o & 2) ++nStale;
+            if (o & 2) {
+                ++nStale;
+                fewest = min(fewest, prm.quota[(int64_t)l * W + p] - sh.room[p]);
+            }
         }
     }
     for (int off = 16; off > 0; off >>= 1) {
         FV oF = __shfl_xor_sync(0xffffffffu, bestF, off);
         int oP = __shfl_xor_sync(0xffffffffu, bestP, off);
         nStale += __shfl_xor_sync(0xffffffffu, nStale, off);
+        fewest = min(fewest, __shfl_xor_sync(0xffffffffu, fewest, off));
         if (oP != INT_MAX && (bestP == INT_MAX || oF < bestF || (oF == bestF && oP < bestP))) { bestF = oF; bestP = oP; }
     }
     if (bestP == INT_MAX) {
@@ -155,12 +176,39 @@ __device__ void plan_decide(const GreedyParams<SV> &prm, int l, const ClassDesc 
     // that holds their coverage vectors and by the number of out-of-date blocks
     int cap = prm.batchMax;
     while (cap > 1 && (int64_t)cap * c.ld * (int64_t)sizeof(SV) > prm.smemBytes) cap >>= 1;
-    // n blocks are refreshed; the kernel is instantiated for lists of 1, 2, 4, 8, so the list is
+    // Threshold pass: once every out-of-date block has a few members, almost no S[v][i] exceeds the
+    // blocks' coverage, so the pass only compares S with one threshold vector and touches the
+    // blocks' coverage per exceeding element: it can refresh up to kSparseMax blocks at once.
+    // A threshold pass is tried when every out-of-date block has sparseFrom[l] members; if more than
+    // 1 element in 32 turned out to be above the threshold, the next try waits until the blocks
+    // have twice the members they had.  Near the end of a class (few rows left) the dense pass,
+    // which can split the columns of a row over several warps, keeps more warps busy.
+    int from = 0;
+    if (lane == 0) {
+        from = prm.sparseFrom[l];
+        const unsigned long long elems = prm.sparseElems[l];
+        if (elems) {
+            const unsigned long long hits = prm.hitCount[l];
+            atomicAdd(&prm.phaseNs[3], hits);
+            atomicAdd(&prm.phaseNs[4], elems);
+            if (hits * 32ull > elems) { from = 2 * fewest; prm.sparseFrom[l] = from; }
+            prm.hitCount[l] = 0;
+            prm.sparseElems[l] = 0;
+        }
+    }
+    from = __shfl_sync(0xffffffffu, from, 0);
+    const int64_t together0 = max(*(volatile int32_t *)&prm.nSweep[3], 1);
+    const bool sparse = prm.sparseMinMembers >= 0 && prm.batchMax > 1 && nStale > 1 && fewest >= from &&
+                        (int64_t)c.ld * (int64_t)sizeof(SV) + kSparseQueueBytes <= prm.smemBytes &&
+                        together0 * ((nR + kSparseRows - 1) / kSparseRows) * 4 >= prm.sweepWarps;
+    if (sparse) cap = kSparseMax;
+    // n blocks are refreshed; the dense pass is instantiated for lists of 1, 2, 4, 8, so its list is
     // padded with copies of j* up to the next power of two (same bytes read, identical values written)
     const int n = nStale < cap ? nStale : cap;
     int P = 1;
     while (P < n) P *= 2;
-    int32_t *parts = prm.sweepParts + (int64_t)l * kMaxSweepBatch;
+    if (sparse) P = n;
+    int32_t *parts = prm.sweepParts + (int64_t)l * kSparseMax;
     if (lane == 0) { parts[0] = jstar; valid[jstar] = 1; sh.open[jstar] = 1; }
     __syncwarp();
     for (int k = 1; k < n; ++k) {
@@ -184,16 +232,23 @@ __device__ void plan_decide(const GreedyParams<SV> &prm, int l, const ClassDesc 
     if (lane == 0) for (int k = n; k < P; ++k) parts[k] = jstar;
     // warps per row group: enough that the row groups of the classes that sweep together (every
     // unfinished class, once per round) cover every warp of the launch, at least one 128-column chunk per warp
-    const int R = rows_per_group(P);
+    const int R = sparse ? kSparseRows : rows_per_group(P);
     const int64_t nGroups = (nR + R - 1) / R;
     const int rem = *(volatile int32_t *)&prm.nSweep[3];              // unfinished classes: they all sweep in the same round
     const int64_t together = rem > 1 ? rem : 1;
     const int chunks = (c.ld + 127) / 128;
     int CS = 1;
-    while (CS < 16 && 2 * CS <= chunks && 2 * CS * together * nGroups <= prm.sweepWarps) CS *= 2;
+    while (!sparse && CS < 16 && 2 * CS <= chunks && 2 * CS * together * nGroups <= prm.sweepWarps) CS *= 2;
     if (lane == 0) {
         sh.nextJ = jstar;
         sh.needSweep = 1;
+        sh.sweepBlocks = P;
+        sh.sweepSparse = sparse ? 1 : 0;
+        prm.sweepMode[l] = sparse ? 1 : 0;
+        if (sparse) {
+            prm.sparseElems[l] = (unsigned long long)nR * (unsigned long long)c.M;
+            atomicMax(&prm.phaseNs[5], (unsigned long long)P);
+        }
         prm.jstar[l] = jstar;
         prm.sweepN[l] = P;
         prm.sweepCS[l] = CS;
@@ -201,8 +256,8 @@ __device__ void plan_decide(const GreedyParams<SV> &prm, int l, const ClassDesc 
         int par = nextStep % 3;
         int slot = atomicAdd(&prm.nSweep[par], 1);
         prm.sweepList[(int64_t)par * prm.L + slot] = l;
-        atomicAdd(&prm.stepBytes[nextStep], (unsigned long long)((int64_t)nR * c.ld + (int64_t)n * c.ld) * sizeof(SV));
-        atomicAdd(&prm.stepOps[nextStep], (unsigned long long)((int64_t)nR * c.M * n));
+        atomicAdd(&prm.stepBytes[nextStep], (unsigned long long)((int64_t)nR * c.ld + (int64_t)(sparse ? 1 : n) * c.ld) * sizeof(SV));
+        atomicAdd(&prm.stepOps[nextStep], (unsigned long long)((int64_t)nR * c.M * (sparse ? 1 : n)));
     }
 }
 
@@ -228,6 +283,9 @@ __global__ void __launch_bounds__(kSelectThreads, 4) init_kernel(GreedyParams<SV
     }
     if (threadIdx.x == 0) {
         prm.nR[l] = c.M;
+        prm.sparseFrom[l] = prm.sparseMinMembers;
+        prm.sparseElems[l] = 0;
+        prm.hitCount[l] = 0;
         if (c.M > 0) atomicAdd(&prm.nSweep[3], 1);         // classes still to finish
     }
     __syncthreads();
@@ -477,13 +535,184 @@ __device__ __forceinline__ void sweep_class(const GreedyParams<SV> &prm, int l, 
     }
 }
 
+// 16 bytes global -> shared without passing through registers (completion: cp.async.wait_group).
+__device__ __forceinline__ void async_copy16(int4 *smemDst, const int4 *src)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" :: "r"((uint32_t)__cvta_generic_to_shared(smemDst)), "l"(src) : "memory");
+}
+
+// Threshold pass over one class.  shThr[i] = min over the P listed blocks of cover_p[i]: an element
+// S[v][i] <= shThr[i] adds nothing to any listed block's gain, and once the blocks have some
+// members that is true of all but a few elements per row.  The warp therefore only compares its R
+// rows against the threshold (one compare per element, whatever P is) and appends the elements
+// above it to a small queue in shared memory.  The queue is drained with the lanes arranged as
+// (queue slot, block): lane (s, p) fetches cover_p[i] for the s-th queued element and adds
+// max(0, S[v][i] - cover_p[i]) to its running sum for that element's row, so 32 / P' elements
+// (P' = P rounded up to a power of two) are in flight at once.  The slots' sums are added at the
+// end of the row group.  With more than 32 blocks every lane serves blocks p and p + 32.
+
+template <typename SV, int A>
+__device__ __noinline__ void sweep_class_sparse(const GreedyParams<SV> &prm, int l, const ClassDesc c, int nR, int P,
+                                                   const int4 *shThr, const int32_t *parts, uint2 *queue)
+{
+    int4 *ring = reinterpret_cast<int4 *>(queue);                    // per warp: ring, queue, sums
+    queue += kSparseRingBytes / 8;
+    using GV = typename Arith<SV>::GV;
+    constexpr int R = kSparseRows;
+    const int lane = threadIdx.x & 31;
+    const unsigned below = (1u << lane) - 1u;
+    const int ld4 = c.ld >> 2;
+    const int nGroups = (nR + R - 1) / R;
+    const SV *Sl = prm.S + c.sOff;
+    const int32_t *cand = prm.cand + c.row0;
+    GV *G = prm.gains + c.vOff;
+    const SV *cover = prm.cover + c.vOff;
+    int Pp = 1;                                                     // lanes per queue slot
+    while (Pp < P && Pp < 32) Pp *= 2;
+    const int slots = 32 / Pp;
+    const int slot = lane / Pp;
+    int myPart[A];
+    const SV *myCov[A];
+#pragma unroll
+    for (int a = 0; a < A; ++a) {
+        const int p = (lane & (Pp - 1)) + 32 * a;
+        myPart[a] = p < P ? parts[p] : -1;
+        myCov[a] = cover + (int64_t)(myPart[a] < 0 ? parts[0] : myPart[a]) * c.ld;
+    }
+    unsigned hits = 0;
+    for (;;) {
+        int g = 0;
+        if (lane == 0) g = atomicAdd(&prm.rowCtr[l], 1);
+        g = __shfl_sync(0xffffffffu, g, 0);
+        if (g >= nGroups) break;
+        const int k0 = g * R;
+        const int4 *rp[R];
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            const int k = k0 + r;
+            rp[r] = reinterpret_cast<const int4 *>(Sl + (int64_t)cand[k < nR ? k : nR - 1] * c.ld);
+        }
+        GV acc[R][A];                                               // running sums of this lane, [row][block of the lane]
+#pragma unroll
+        for (int r = 0; r < R; ++r)
+#pragma unroll
+            for (int a = 0; a < A; ++a) acc[r][a] = 0;
+        int qn = 0;                                                 // queued elements (same in every lane)
+        auto drain = [&]() {
+            __syncwarp();
+            for (int i0 = slot; i0 < qn; i0 += 2 * slots) {
+                uint2 e[2];
+                bool ok[2];
+#pragma unroll
+                for (int u = 0; u < 2; ++u) {
+                    const int i = i0 + u * slots;
+                    ok[u] = i < qn;
+                    e[u] = queue[ok[u] ? i : i0];
+                }
+                GV d[2][A];
+#pragma unroll
+                for (int u = 0; u < 2; ++u) {
+                    const int col = (int)(e[u].x & 0x0fffffffu);
+#pragma unroll
+                    for (int a = 0; a < A; ++a) {
+                        const SV cv = myCov[a][col];
+                        if constexpr (Arith<SV>::kInt) {
+                            const int dd = (int)e[u].y - cv;
+                            d[u][a] = (ok[u] && myPart[a] >= 0 && dd > 0) ? (GV)dd : (GV)0;
+                        } else {
+                            const float dd = __uint_as_float(e[u].y) - cv;
+                            d[u][a] = (ok[u] && myPart[a] >= 0 && dd > 0.f) ? dd : 0.f;
+                        }
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < 2; ++u) {
+                    const int r = (int)(e[u].x >> 28);
+#pragma unroll
+                    for (int rr = 0; rr < R; ++rr)
+#pragma unroll
+                        for (int a = 0; a < A; ++a) acc[rr][a] += (r == rr) ? d[u][a] : (GV)0;
+                }
+            }
+            __syncwarp();
+            qn = 0;
+        };
+        // S streams through a ring in shared memory filled by asynchronous copies, kSparseStages - 1
+        // chunks ahead; every lane reads back only the 16-byte pieces it copied itself, so waiting
+        // for its own copy groups is all the synchronisation the ring needs
+        auto issue = [&](int base, int st) {
+            const int cc = base + lane;
+            if (cc < ld4) {
+#pragma unroll
+                for (int r = 0; r < R; ++r) async_copy16(ring + (st * R + r) * 32 + lane, rp[r] + cc);
+            }
+            asm volatile("cp.async.commit_group;" ::: "memory");
+        };
+#pragma unroll
+        for (int st = 0; st < kSparseStages - 1; ++st) issue(st * 32, st);
+        int stage = 0;
+        for (int base = 0; base < ld4; base += 32) {                // every lane runs every chunk: ballots below
+            const int cc = base + lane;
+            const bool inside = cc < ld4;
+            {
+                int ahead = stage + kSparseStages - 1;
+                if (ahead >= kSparseStages) ahead -= kSparseStages;
+                issue(base + (kSparseStages - 1) * 32, ahead);       // past the row's end: an empty group
+            }
+            asm volatile("cp.async.wait_group %0;" :: "n"(kSparseStages - 1) : "memory");
+            int4 t = make_int4(0, 0, 0, 0);
+            if (inside) t = shThr[cc];
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                int4 s = make_int4(0, 0, 0, 0);
+                unsigned h = 0;
+                if (inside) {
+                    s = ring[(stage * R + r) * 32 + lane];
+                    if constexpr (Arith<SV>::kInt) {
+                        h = (s.x > t.x ? 1u : 0u) | (s.y > t.y ? 2u : 0u) | (s.z > t.z ? 4u : 0u) | (s.w > t.w ? 8u : 0u);
+                    } else {
+                        h = (__int_as_float(s.x) > __int_as_float(t.x) ? 1u : 0u) | (__int_as_float(s.y) > __int_as_float(t.y) ? 2u : 0u) |
+                            (__int_as_float(s.z) > __int_as_float(t.z) ? 4u : 0u) | (__int_as_float(s.w) > __int_as_float(t.w) ? 8u : 0u);
+                    }
+                }
+                if (__any_sync(0xffffffffu, h != 0)) {
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const bool mine = (h >> e) & 1u;
+                        const unsigned m = __ballot_sync(0xffffffffu, mine);
+                        if (mine) {
+                            const int sv = e == 0 ? s.x : (e == 1 ? s.y : (e == 2 ? s.z : s.w));
+                            queue[qn + __popc(m & below)] = make_uint2((unsigned)(cc * 4 + e) | ((unsigned)r << 28), (unsigned)sv);
+                        }
+                        qn += __popc(m);
+                    }
+                    if (qn > kSparseQueue - 128) { hits += qn; drain(); }
+                }
+            }
+            if (++stage == kSparseStages) stage = 0;
+        }
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+        if (qn) { hits += qn; drain(); }
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+#pragma unroll
+            for (int a = 0; a < A; ++a) {
+                GV t = acc[r][a];
+                for (int off = Pp; off < 32; off <<= 1) t += __shfl_xor_sync(0xffffffffu, t, off);
+                if (slot == 0 && k0 + r < nR && myPart[a] >= 0) G[(int64_t)myPart[a] * c.ld + cand[k0 + r]] = t;
+            }
+        }
+    }
+    if (lane == 0 && hits) atomicAdd(&prm.hitCount[l], (unsigned long long)hits);
+}
+
 // The sweep of greedy step `step`, run by every CTA of the launch (kSweepThreads threads each).
 template <typename SV>
 __device__ __forceinline__ void sweep_step(const GreedyParams<SV> &prm, int step, int4 *shCover)
 {
     using GV = typename Arith<SV>::GV;
     __shared__ long long shF[kMaxSweepBatch];
-    __shared__ int32_t shParts[kMaxSweepBatch];
+    __shared__ int32_t shParts[kSparseMax];
     __shared__ int shTicket[kSweepThreads / 32];
     __shared__ GV shPart[kSweepThreads];
     __shared__ int shGo;
@@ -503,7 +732,7 @@ __device__ __forceinline__ void sweep_step(const GreedyParams<SV> &prm, int step
         __syncthreads();
         for (int s = threadIdx.x; s < nS; s += blockDim.x) {
             const int ls = prm.sweepList[(int64_t)par * prm.L + s];
-            const int Rs = rows_per_group(prm.sweepN[ls]);
+            const int Rs = prm.sweepMode[ls] ? kSparseRows : rows_per_group(prm.sweepN[ls]);
             const int groups = (prm.nR[ls] + Rs - 1) / Rs;
             if (*(volatile int32_t *)&prm.rowCtr[ls] < groups) {
                 int dist = s - start;
@@ -521,9 +750,18 @@ __device__ __forceinline__ void sweep_step(const GreedyParams<SV> &prm, int step
         const int nR = prm.nR[l];
         const int P = prm.sweepN[l];
         const int CS = prm.sweepCS[l];
-        {
-            const int ld4 = c.ld >> 2;
-            const int32_t *parts = prm.sweepParts + (int64_t)l * kMaxSweepBatch;
+        const int ld4 = c.ld >> 2;
+        const int32_t *parts = prm.sweepParts + (int64_t)l * kSparseMax;
+        if (prm.sweepMode[l]) {
+            // threshold pass: one vector in shared memory, the blocks' coverage stays in global memory
+            const int4 *thr = reinterpret_cast<const int4 *>(prm.thr + c.vOff / prm.W);
+            for (int i = threadIdx.x; i < ld4; i += blockDim.x) shCover[i] = thr[i];
+            if (threadIdx.x < P) shParts[threadIdx.x] = parts[threadIdx.x];
+            __syncthreads();
+            uint2 *queue = reinterpret_cast<uint2 *>(reinterpret_cast<char *>(shCover + ld4) + (threadIdx.x >> 5) * kSparseWarpBytes);
+            if (P <= 32) sweep_class_sparse<SV, 1>(prm, l, c, nR, P, shCover, shParts, queue);
+            else sweep_class_sparse<SV, 2>(prm, l, c, nR, P, shCover, shParts, queue);
+        } else {
             const int4 *cov = reinterpret_cast<const int4 *>(prm.cover + c.vOff);
             for (int i = threadIdx.x; i < P * ld4; i += blockDim.x) {
                 int p = i / ld4, cc = i - p * ld4;
@@ -546,7 +784,7 @@ __device__ __forceinline__ void sweep_step(const GreedyParams<SV> &prm, int step
 }
 
 template <typename SV>
-__global__ void __launch_bounds__(kSweepThreads, 1) sweep_kernel(GreedyParams<SV> prm, int step)
+__global__ void __launch_bounds__(kSweepThreads, 1) sweep_kernel(const __grid_constant__ GreedyParams<SV> prm, int step)
 {
     extern __shared__ int4 shCover[];
     cudaGridDependencySynchronize();              // the previous launch (select / init) has finished
@@ -570,11 +808,20 @@ __device__ __forceinline__ int4 max_int4(int4 a, int4 b)
     return a;
 }
 
-// 16 bytes global -> shared without passing through registers (completion: cp.async.wait_group).
-__device__ __forceinline__ void async_copy16(int4 *smemDst, const int4 *src)
+template <typename SV>
+__device__ __forceinline__ int4 min_int4(int4 a, int4 b)
 {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" :: "r"((uint32_t)__cvta_generic_to_shared(smemDst)), "l"(src) : "memory");
+    if constexpr (Arith<SV>::kInt) {
+        a.x = min(a.x, b.x); a.y = min(a.y, b.y); a.z = min(a.z, b.z); a.w = min(a.w, b.w);
+    } else {
+        a.x = __float_as_int(fminf(__int_as_float(a.x), __int_as_float(b.x)));
+        a.y = __float_as_int(fminf(__int_as_float(a.y), __int_as_float(b.y)));
+        a.z = __float_as_int(fminf(__int_as_float(a.z), __int_as_float(b.z)));
+        a.w = __float_as_int(fminf(__int_as_float(a.w), __int_as_float(b.w)));
+    }
+    return a;
 }
+
 
 // Finishes a coverage update whose operands were copied to shared memory earlier (row v* in
 // scratch[0, ld4), the old coverage in scratch[ld4, 2 ld4)): dst[i] = max of the two.
@@ -721,6 +968,25 @@ __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, i
         if (nR == 0 || j < 0 || shPlan.needSweep) break;
     }
     if (pendDst) fold_pending<SV>(pendDst, scratch, ld4);
+    if (shPlan.needSweep && shPlan.sweepSparse) {
+        // threshold of the coming pass: element-wise minimum of the listed blocks' coverage vectors
+        // (each thread reads back exactly the pieces of the coverage vectors it wrote itself)
+        const int P = shPlan.sweepBlocks;
+        const int32_t *parts = prm.sweepParts + (int64_t)l * kSparseMax;
+        const int4 *cov = reinterpret_cast<const int4 *>(prm.cover + c.vOff);
+        int4 *thr = reinterpret_cast<int4 *>(prm.thr + c.vOff / prm.W);
+        for (int i = threadIdx.x; i < ld4; i += kSelectThreads) {
+            int4 m = cov[(int64_t)parts[0] * ld4 + i];
+            for (int k0 = 1; k0 < P; k0 += 8) {                     // eight independent loads at a time
+                int4 t[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) t[u] = cov[(int64_t)parts[k0 + u < P ? k0 + u : 0] * ld4 + i];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) m = min_int4<SV>(m, t[u]);
+            }
+            thr[i] = m;
+        }
+    }
 }
 
 // Picks of round `round`: every class advances until it needs a sweep (or is finished).
@@ -778,7 +1044,7 @@ __device__ __forceinline__ unsigned long long global_ns()
 // sit in shared memory, the barrier's target is recomputed from the round number -- so that the
 // sweep's inner loop gets the whole register budget.)
 template <typename SV>
-__global__ void __launch_bounds__(kSweepThreads, 1) greedy_persistent_kernel(GreedyParams<SV> prm, int maxRounds)
+__global__ void __launch_bounds__(kSweepThreads, 1) greedy_persistent_kernel(const __grid_constant__ GreedyParams<SV> prm, int maxRounds)
 {
     extern __shared__ int4 shCover[];
     __shared__ unsigned long long shClock[3];      // last stamp, sweep-phase ns, pick-phase ns (CTA 0, thread 0)
@@ -847,6 +1113,11 @@ static rcd_status run_greedy(rcd_ctx *ctx, const Sizes &sz, const Workspace &ws,
     prm.jstar = ws.jstar;
     prm.sweepN = ws.sweepN;
     prm.sweepParts = ws.sweepParts;
+    prm.sweepMode = ws.sweepMode;
+    prm.thr = (SV *)ws.thr;
+    prm.hitCount = ws.hitCount;
+    prm.sparseElems = ws.sparseElems;
+    prm.sparseFrom = ws.sparseFrom;
     prm.sweepCS = ws.sweepCS;
     prm.rowCtr = ws.rowCtr;
     prm.sweepList = ws.sweepList;
@@ -866,11 +1137,14 @@ static rcd_status run_greedy(rcd_ctx *ctx, const Sizes &sz, const Workspace &ws,
     prm.batchMax = batch;
     prm.sweepWarps = ctx->smCount * (kSweepThreads / 32);
     prm.one = 1u;
+    prm.sparseMinMembers = ctx->cfg.sweep_mode == 1 ? -1 : 8;
 
     int maxLd = 0;
     for (const auto &c : descHost) if (c.ld > maxLd) maxLd = c.ld;
     const int64_t smemCap = (int64_t)ctx->maxSmemOptin - 20 * 1024;  // static shared of the kernels + margin
     int64_t smem = (int64_t)batch * maxLd * (int64_t)sizeof(SV);
+    if (prm.sparseMinMembers >= 0)                                   // threshold pass: one vector + the warps' rings and queues
+        smem = std::max<int64_t>(smem, (int64_t)maxLd * (int64_t)sizeof(SV) + kSparseQueueBytes);
     if (smem > smemCap) smem = smemCap;
     if ((int64_t)maxLd * (int64_t)sizeof(SV) > smem)
         return fail(ctx, RCD_ERR_UNSUPPORTED,
@@ -889,7 +1163,7 @@ static rcd_status run_greedy(rcd_ctx *ctx, const Sizes &sz, const Workspace &ws,
     RCD_CUDA(ctx, cudaFuncSetAttribute(sweep_kernel<SV>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
 
     RCD_CUDA(ctx, cudaMemsetAsync(ws.nSweep, 0, 4 * sizeof(int32_t), st));
-    RCD_CUDA(ctx, cudaMemsetAsync(ws.phaseNs, 0, 3 * sizeof(unsigned long long), st));
+    RCD_CUDA(ctx, cudaMemsetAsync(ws.phaseNs, 0, 6 * sizeof(unsigned long long), st));
     ctx->phaseNsDev = ws.phaseNs;
     RCD_CUDA(ctx, cudaMemsetAsync(ws.stepBytes, 0, (size_t)(sz.maxM + 1) * sizeof(unsigned long long), st));
     RCD_CUDA(ctx, cudaMemsetAsync(ws.stepOps, 0, (size_t)(sz.maxM + 1) * sizeof(unsigned long long), st));

@@ -11,7 +11,8 @@
 
 namespace rcd {
 
-constexpr int kMaxSweepBatch = 8;          // blocks refreshed by one pass over S
+constexpr int kMaxSweepBatch = 8;          // blocks refreshed by one dense pass over S
+constexpr int kSparseMax = 64;             // blocks refreshed by one threshold pass over S
 constexpr int kSweepThreads = 512;         // sweep CTA: 16 warps, one CTA per SM
 constexpr int kSelectThreads = 512;        // pick/update CTA: one per class
 constexpr size_t kAlign = 256;
@@ -88,14 +89,19 @@ struct Workspace {
     int32_t *nR;            // [L] unassigned count
     int32_t *jstar;         // [L] block chosen for the next pick (-1: none)
     int32_t *sweepN;        // [L] blocks to refresh in the next sweep (0: none)
-    int32_t *sweepParts;    // [L][kMaxSweepBatch]
+    int32_t *sweepParts;    // [L][kSparseMax]
+    int32_t *sweepMode;     // [L] dense / threshold pass
+    void *thr;              // [sum ld] threshold vector of every class (int32 / float)
+    unsigned long long *hitCount;   // [L]
+    unsigned long long *sparseElems; // [L]
+    int32_t *sparseFrom;    // [L]
     int32_t *sweepCS;       // [L] warps per row group in the next sweep
     int32_t *rowCtr;        // [L] ticket counter over row groups of the running sweep
     int32_t *sweepList;     // [3][L] classes that sweep in a step (three lists in rotation)
     int32_t *nSweep;        // [3] (+1 pad)
     unsigned long long *stepBytes;   // [steps+1] bytes the sweep of step t has to read
     unsigned long long *stepOps;     // [steps+1] element x block pairs of that sweep
-    unsigned long long *phaseNs;     // [2] sweep-phase / pick-phase nanoseconds of the persistent kernel
+    unsigned long long *phaseNs;     // [6] sweep-/pick-phase ns of the persistent kernel, barrier counter, threshold-pass hits / elements / max blocks
     int32_t *status;        // [1]
     size_t bytes;           // total bytes laid out
 };

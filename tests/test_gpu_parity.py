@@ -212,6 +212,53 @@ def test_partition_c4_reduced_float(rcd, orc, batch, path):
     check_float(rcd, orc, wl, sweep_batch_max=batch, greedy_path=path)
 
 
+# ----------------------------------------------------------------------------- threshold passes
+
+def run_with_profile(rcd, wl, **cfg):
+    with rcd.Context(0, profile=1, **cfg) as ctx:
+        X, y = to_device(rcd, wl)
+        a, o, v = ctx.rcd_partition(X, y, wl.capacities, wl.L)
+        ctx.sync_status()
+        return a.cpu().numpy(), o.cpu().numpy(), v.cpu().numpy(), ctx.profile()
+
+
+@pytest.mark.parametrize("path", [0, 1])
+def test_threshold_passes_int8_exact(rcd, orc, path):
+    """Classes large enough that the sweeps switch to threshold passes: same picks as the oracle, and
+    the same as with dense passes only."""
+    from paper_2211_00839_b200.workloads import make_workload
+    wl = make_workload("C2", L=3, M=1200)
+    ref = orc.partition(wl.features, wl.labels, wl.capacities, wl.L, variant="incremental")
+    a, o, v, prof = run_with_profile(rcd, wl, greedy_path=path)
+    assert prof["threshold_elems"] > 0 and 0 < prof["threshold_hits"] < prof["threshold_elems"] // 32
+    assert np.array_equal(a, ref.assignment) and np.array_equal(o, ref.order) and np.array_equal(v, ref.part_values)
+    a1, o1, v1, prof1 = run_with_profile(rcd, wl, greedy_path=path, sweep_mode=1)
+    assert prof1["threshold_elems"] == 0
+    assert np.array_equal(a1, a) and np.array_equal(o1, o) and np.array_equal(v1, v)
+
+
+def test_threshold_passes_many_blocks_exact(rcd, orc):
+    """W = 64: one threshold pass refreshes more than 32 blocks (two blocks per lane)."""
+    from paper_2211_00839_b200.workloads import make_workload
+    wl = make_workload("C5", L=3, M=1300, d=128)
+    ref = orc.partition(wl.features, wl.labels, wl.capacities, wl.L, variant="incremental")
+    a, o, v, prof = run_with_profile(rcd, wl)
+    assert prof["threshold_elems"] > 0 and prof["threshold_max_blocks"] > 32
+    assert np.array_equal(a, ref.assignment) and np.array_equal(o, ref.order) and np.array_equal(v, ref.part_values)
+
+
+def test_threshold_passes_float(rcd, orc):
+    from paper_2211_00839_b200.workloads import make_workload
+    wl = make_workload("C3", L=2, M=900, d=512)
+    with rcd.Context(0, profile=1) as ctx:
+        X, y = to_device(rcd, wl)
+        ctx.rcd_partition(X, y, wl.capacities, wl.L)
+        ctx.sync_status()
+        assert ctx.profile()["threshold_elems"] > 0
+    check_float(rcd, orc, wl)                       # default configuration: the run above
+    check_float(rcd, orc, wl, sweep_mode=1)
+
+
 # ----------------------------------------------------------------------------- objective
 
 @pytest.mark.parametrize("name,L,M,d", [("C1", 2, 200, 64), ("C5", 3, 300, 128), ("C4", 3, 250, 96)])
