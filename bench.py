@@ -32,6 +32,10 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 
+# DRAM bytes (read + write) of one launch of the dominant kernel under ncu, by (configuration, kernel).
+MEASURED_TRAFFIC = {}
+
+
 def load_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -177,6 +181,7 @@ def run_ours(args):
     Xd, yd = Xh.to(dev), yh.to(dev)
     kind = rcd.RCD_SIM_GAUSSIAN if args.similarity == "gaussian" else rcd.RCD_SIM_DOT
     ctx = rcd.Context(local, sweep_batch_max=args.sweep_batch, profile=1, greedy_path=args.greedy_path, similarity_kind=kind,
+                      async_group=args.async_group,
                       objective=rcd.RCD_OBJ_GRAPH_CUT if args.objective == "cut" else rcd.RCD_OBJ_FACILITY)
 
     def barrier():
@@ -247,13 +252,20 @@ def run_ours(args):
     # plus the coverage vectors of the blocks refreshed (4*ld*(n_R + n) bytes), summed on the device.
     # Duration = CUDA events around the greedy loop on the launching stream (last timed step).
     peaks = load_peaks()
+    default_setup = args.sweep_batch in (0, 8) and args.async_group == 0 and args.similarity == "dot"
     loop_s = prof["greedy_ms"] * 1e-3
     achieved = prof["sweep_bytes"] / loop_s / 1e9 if loop_s > 0 else 0.0
-    roofline = {"bound": "hbm", "kernel": "greedy_persistent_kernel" if args.objective == "facility" else "cut_chain_kernel", "achieved": achieved, "peak": peaks["hbm_gbs"],
+    if args.objective != "facility":
+        kernel_name = "cut_chain_kernel"
+    elif args.greedy_path == 3 or (args.greedy_path == 0 and wl.L * 4 <= torch.cuda.get_device_properties(local).multi_processor_count):
+        kernel_name = "greedy_async_kernel"
+    else:
+        kernel_name = "greedy_persistent_kernel" if args.greedy_path != 1 else "sweep_kernel"
+    roofline = {"bound": "hbm", "kernel": kernel_name, "achieved": achieved, "peak": peaks["hbm_gbs"],
                 "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "peak_source": peaks["source"],
-                # dram__bytes_read.sum + dram__bytes_write.sum of one launch on the default C2 workload
-                # (ncu capture summarised in profiles/greedy_persistent_kernel_C2.md)
-                "traffic": 491.18e9 if (args.config == "C2" and args.sweep_batch in (0, 8) and args.greedy_path == 0 and args.similarity == "dot" and args.objective == "facility") else None,
+                # dram__bytes_read.sum + dram__bytes_write.sum of one launch of that kernel on this workload, from the
+                # ncu capture summarised under profiles/ (None: no capture of the kernel as it stands)
+                "traffic": MEASURED_TRAFFIC.get((args.config, kernel_name)) if default_setup else None,
                 "launch_ms": prof["greedy_ms"], "bytes_per_launch": prof["sweep_bytes"],
                 "rounds_with_sweeps": int(prof["sweep_launches"])}
     # the same bytes against the time the kernel spends in its sweep phases (its own clock, CTA 0)
@@ -330,7 +342,9 @@ def main():
     ap.add_argument("--sweep-batch", type=int, default=0, help="sweep_batch_max (0 = library default)")
     ap.add_argument("--similarity", default="dot", choices=["dot", "gaussian"], help="similarity of Section 4 item 2")
     ap.add_argument("--objective", default="facility", choices=["facility", "cut"], help="submodular function of Section 4 item 2")
-    ap.add_argument("--greedy-path", type=int, default=0, help="0 = one cooperative launch, 1 = two launches per round")
+    ap.add_argument("--greedy-path", type=int, default=0,
+                    help="0 = chosen by the library, 1 = two launches per round, 2 = one launch with rounds, 3 = one launch, asynchronous classes")
+    ap.add_argument("--async-group", type=int, default=0, help="greedy path 3: sweeps served together (0 = library default)")
     ap.add_argument("--ref-picks", type=int, default=150, help="picks per class in the CPU-oracle sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

@@ -76,13 +76,21 @@ typedef struct {
     int32_t sweep_batch_max;   /* blocks whose gains one pass over S may refresh: 1,2,4 or 8; 0 = default (8) */
     int32_t similarity_path;   /* 0 = tensor-core kernel when the shape allows, 2 = always the generic kernel */
     int32_t profile;           /* 0 off; 1 time the phases of rcd_partition; 2 also time every sweep launch */
-    int32_t greedy_path;       /* 0 = whole greedy loop in one cooperative launch when the device allows;
-                                  1 = two launches per greedy step (always used with profile 2) */
+    int32_t greedy_path;       /* form of the greedy loop.  0 = choose: one cooperative launch when the device allows,
+                                  asynchronous classes (3) when there are at most a quarter as many classes as SMs,
+                                  else rounds (2);  1 = two launches per round (always used with profile 2);
+                                  2 = one launch, rounds of a sweep phase and a pick phase separated by grid barriers;
+                                  3 = one launch, every class cycles between sweep and picks on its own: some CTAs
+                                  only make picks, the others only sweep, so picks overlap other classes' sweeps.
+                                  All forms make the same picks. */
     int32_t similarity_kind;   /* rcd_similarity_kind used by rcd_partition / rcd_objective (default RCD_SIM_DOT) */
     int32_t objective;         /* rcd_objective_kind used by rcd_partition / rcd_objective (default facility location) */
     int32_t sweep_mode;        /* 0 = threshold passes once the blocks have a few members (up to 64 blocks per pass);
                                   1 = dense passes only (sweep_batch_max blocks per pass) */
-    int32_t reserved[9];       /* must be 0 */
+    int32_t async_group;       /* greedy_path 3: sweeps published one after another that the sweep CTAs serve together,
+                                  each CTA going to the class nearest its home position; 1 = strictly oldest first;
+                                  0 = default: all classes together */
+    int32_t reserved[8];       /* must be 0 */
 } rcd_config;
 
 /* Timings and counters of the last rcd_partition / rcd_partition_host on a context (profile >= 1). */
@@ -98,8 +106,10 @@ typedef struct {
     int64_t kernel_launches;   /* kernels this library launched during the call */
     int64_t steps;             /* greedy steps executed (= largest class size) */
     int64_t similarity_tc_launches; /* similarity launches of the last call that ran on the tensor cores */
-    int64_t persistent_sweep_ns;    /* one-launch greedy loop: time in sweep phases (incl. their barrier) */
-    int64_t persistent_pick_ns;     /* one-launch greedy loop: time in pick phases (incl. their barrier) */
+    int64_t persistent_sweep_ns;    /* one-launch greedy loop: time in sweep phases (incl. their barrier); asynchronous
+                                       form: time the first sweep CTA spent sweeping (not looking for work) */
+    int64_t persistent_pick_ns;     /* one-launch greedy loop: time in pick phases (incl. their barrier); asynchronous
+                                       form: time the first pick CTA spent making picks (not waiting for sweeps) */
     int64_t threshold_hits;         /* threshold passes: elements of S above the threshold ... */
     int64_t threshold_elems;        /* ... out of this many elements compared */
     int64_t threshold_max_blocks;   /* most blocks one threshold pass refreshed */

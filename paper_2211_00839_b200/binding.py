@@ -46,7 +46,8 @@ class RcdError(RuntimeError):
 
 class RcdConfig(C.Structure):
     _fields_ = [("sweep_batch_max", C.c_int32), ("similarity_path", C.c_int32), ("profile", C.c_int32),
-                ("greedy_path", C.c_int32), ("similarity_kind", C.c_int32), ("objective", C.c_int32), ("sweep_mode", C.c_int32), ("reserved", C.c_int32 * 9)]
+                ("greedy_path", C.c_int32), ("similarity_kind", C.c_int32), ("objective", C.c_int32), ("sweep_mode", C.c_int32), ("async_group", C.c_int32),
+                ("reserved", C.c_int32 * 8)]
 
 
 class RcdProfile(C.Structure):
@@ -143,7 +144,8 @@ class Context:
     """Owns one ``rcd_ctx`` on a CUDA device."""
 
     def __init__(self, device: int = 0, sweep_batch_max: int = 0, similarity_path: int = 0, profile: int = 0,
-                 greedy_path: int = 0, similarity_kind: int = 0, objective: int = 0, sweep_mode: int = 0):
+                 greedy_path: int = 0, similarity_kind: int = 0, objective: int = 0, sweep_mode: int = 0,
+                 async_group: int = 0):
         torch = _torch()
         if not torch.cuda.is_available():
             raise RcdError(4, "no CUDA device: this library has no CPU path")
@@ -157,6 +159,7 @@ class Context:
         cfg.similarity_kind = similarity_kind
         cfg.objective = objective
         cfg.sweep_mode = sweep_mode
+        cfg.async_group = async_group
         self.similarity_kind = similarity_kind
         self._h = C.c_void_p()
         st = lib.rcd_create(C.byref(self._h), self.device, C.byref(cfg))

@@ -87,6 +87,8 @@ size_t layout_workspace(void *base, rcd_feat_dtype dtype, const Sizes &sz, Works
     w.sweepCS = c.take<int32_t>(L);
     w.rowCtr = c.take<int32_t>(L);
     w.sweepList = c.take<int32_t>(3 * L);
+    w.sync = c.take<ClassSync>(L);
+    w.tickets = c.take<int32_t>(N + L);
     w.stepBytes = c.take<unsigned long long>((size_t)sz.maxM + 1);
     w.stepOps = c.take<unsigned long long>((size_t)sz.maxM + 1);
     w.phaseNs = c.take<unsigned long long>(6);      // two phase clocks, the grid-barrier counter, threshold-pass hits / elements
@@ -285,11 +287,12 @@ rcd_status rcd_create(rcd_ctx **out, int cuda_device, const rcd_config *cfg)
             return RCD_ERR_INVALID_ARG;
         if (cfg->similarity_path != 0 && cfg->similarity_path != 2) return RCD_ERR_INVALID_ARG;
         if (cfg->profile < 0 || cfg->profile > 2) return RCD_ERR_INVALID_ARG;
-        if (cfg->greedy_path != 0 && cfg->greedy_path != 1) return RCD_ERR_INVALID_ARG;
+        if (cfg->greedy_path < 0 || cfg->greedy_path > 3) return RCD_ERR_INVALID_ARG;
         if (cfg->similarity_kind != RCD_SIM_DOT && cfg->similarity_kind != RCD_SIM_GAUSSIAN) return RCD_ERR_INVALID_ARG;
         if (cfg->objective != RCD_OBJ_FACILITY && cfg->objective != RCD_OBJ_GRAPH_CUT) return RCD_ERR_INVALID_ARG;
         if (cfg->sweep_mode != 0 && cfg->sweep_mode != 1) return RCD_ERR_INVALID_ARG;
-        for (int i = 0; i < 9; ++i) if (cfg->reserved[i] != 0) return RCD_ERR_INVALID_ARG;
+        if (cfg->async_group < 0 || cfg->async_group > 4096) return RCD_ERR_INVALID_ARG;
+        for (int i = 0; i < 8; ++i) if (cfg->reserved[i] != 0) return RCD_ERR_INVALID_ARG;
     }
     int count = 0;
     if (cudaGetDeviceCount(&count) != cudaSuccess || cuda_device < 0 || cuda_device >= count) {

@@ -83,6 +83,13 @@ struct GreedyParams {
     int32_t sweepWarps;     // warps of one sweep launch (CTAs x 16)
     uint32_t one;           // the value 1, opaque to the compiler (see accumulate_chunk)
     int32_t sparseMinMembers;   // threshold passes start once every out-of-date block has this many members (<0: never)
+    // asynchronous kernel (greedy_async_kernel); asyncMode = 0 everywhere else
+    ClassSync *sync;            // [L] hand-off words
+    int32_t *tickets;           // [N + L] ticket counter of sweep k of class l at tickets[row0_l + l + k]
+    int32_t *pubSeq;            // publication counter (orders the sweeps: oldest first)
+    int32_t asyncMode;
+    int32_t nPick;              // CTAs [0, nPick) make picks, the others sweep
+    int32_t asyncGroup;         // sweeps published one after another that are served together (by CTA home position)
 };
 
 __host__ __device__ inline int rows_per_group(int P) { return P == 8 ? 4 : 8; }
@@ -253,9 +260,13 @@ __device__ void plan_decide(const GreedyParams<SV> &prm, int l, const ClassDesc 
         prm.sweepN[l] = P;
         prm.sweepCS[l] = CS;
         prm.rowCtr[l] = 0;
-        int par = nextStep % 3;
-        int slot = atomicAdd(&prm.nSweep[par], 1);
-        prm.sweepList[(int64_t)par * prm.L + slot] = l;
+        if (prm.asyncMode) {
+            prm.sync[l].nGroups = (int32_t)nGroups;        // published with the epoch by the caller
+        } else {
+            int par = nextStep % 3;
+            int slot = atomicAdd(&prm.nSweep[par], 1);
+            prm.sweepList[(int64_t)par * prm.L + slot] = l;
+        }
         atomicAdd(&prm.stepBytes[nextStep], (unsigned long long)((int64_t)nR * c.ld + (int64_t)(sparse ? 1 : n) * c.ld) * sizeof(SV));
         atomicAdd(&prm.stepOps[nextStep], (unsigned long long)((int64_t)nR * c.M * (sparse ? 1 : n)));
     }
@@ -287,6 +298,12 @@ __global__ void __launch_bounds__(kSelectThreads, 4) init_kernel(GreedyParams<SV
         prm.sparseElems[l] = 0;
         prm.hitCount[l] = 0;
         if (c.M > 0) atomicAdd(&prm.nSweep[3], 1);         // classes still to finish
+        if (prm.asyncMode) {
+            prm.sync[l].epoch = c.M > 0 ? 0 : 1;           // sweep 0 is published by this kernel
+            prm.sync[l].done = 0;
+            prm.sync[l].seq = l;
+            prm.sync[l].nGroups = 0;                       // (plan_decide below sets it)
+        }
     }
     __syncthreads();
     plan_load(prm, l, shPlan);
@@ -389,7 +406,8 @@ __device__ __forceinline__ void accumulate_chunk(uint32_t one, const int4 (&s)[R
 template <typename SV, int P, int R>
 __device__ __forceinline__ void sweep_class(const GreedyParams<SV> &prm, int l, const ClassDesc &c, int nR, int CS,
                                             const int4 *shCover, const long long *shF, const int32_t *parts,
-                                            int *shTicket, typename Arith<SV>::GV *shPart)
+                                            int *shTicket, typename Arith<SV>::GV *shPart,
+                                            int32_t *ticket, int32_t *done, int firstTicket)
 {
     using GV = typename Arith<SV>::GV;
     using AccT = typename std::conditional<Arith<SV>::kInt, uint32_t, float>::type;
@@ -405,14 +423,20 @@ __device__ __forceinline__ void sweep_class(const GreedyParams<SV> &prm, int l, 
     const int32_t *cand = prm.cand + c.row0;
     GV *G = prm.gains + c.vOff;
     GV *myPart = shPart + (team * CS) * 32;       // [CS][32] for this team (teams are CS-aligned)
+    // `ticket` hands out the row groups.  firstTicket >= 0: the CTA has already drawn one ticket per
+    // team (firstTicket + team); `done` (may be null) counts the row groups whose gains are written.
+    bool preDrawn = firstTicket >= 0;
 
     for (;;) {
         int g = 0;
-        if (CS == 1) {
-            if (lane == 0) g = atomicAdd(&prm.rowCtr[l], 1);
+        if (preDrawn) {
+            g = firstTicket + team;
+            preDrawn = false;
+        } else if (CS == 1) {
+            if (lane == 0) g = atomicAdd(ticket, 1);
             g = __shfl_sync(0xffffffffu, g, 0);
         } else {
-            if (wIn == 0 && lane == 0) shTicket[team] = atomicAdd(&prm.rowCtr[l], 1);
+            if (wIn == 0 && lane == 0) shTicket[team] = atomicAdd(ticket, 1);
             team_sync(barId, teamThreads);
             g = shTicket[team];
         }
@@ -423,7 +447,7 @@ __device__ __forceinline__ void sweep_class(const GreedyParams<SV> &prm, int l, 
 #pragma unroll
         for (int r = 0; r < R; ++r) {
             int k = k0 + r;
-            vrow[r] = cand[k < nR ? k : nR - 1];
+            vrow[r] = __ldcg(cand + (k < nR ? k : nR - 1));
             rp[r] = reinterpret_cast<const int4 *>(Sl + (int64_t)vrow[r] * c.ld);
         }
         GV total;
@@ -532,6 +556,10 @@ __device__ __forceinline__ void sweep_class(const GreedyParams<SV> &prm, int l, 
                 G[(int64_t)parts[p] * c.ld + row] = gain;
             }
         }
+        if (done != nullptr && wIn == 0) {
+            __syncwarp();
+            if (lane == 0) { __threadfence(); atomicAdd(done, 1); }
+        }
     }
 }
 
@@ -553,7 +581,8 @@ __device__ __forceinline__ void async_copy16(int4 *smemDst, const int4 *src)
 
 template <typename SV, int A>
 __device__ __noinline__ void sweep_class_sparse(const GreedyParams<SV> &prm, int l, const ClassDesc c, int nR, int P,
-                                                   const int4 *shThr, const int32_t *parts, uint2 *queue)
+                                                   const int4 *shThr, const int32_t *parts, uint2 *queue,
+                                                   int32_t *ticket, int32_t *done, int firstTicket)
 {
     int4 *ring = reinterpret_cast<int4 *>(queue);                    // per warp: ring, queue, sums
     queue += kSparseRingBytes / 8;
@@ -580,17 +609,23 @@ __device__ __noinline__ void sweep_class_sparse(const GreedyParams<SV> &prm, int
         myCov[a] = cover + (int64_t)(myPart[a] < 0 ? parts[0] : myPart[a]) * c.ld;
     }
     unsigned hits = 0;
+    bool preDrawn = firstTicket >= 0;                               // one ticket per warp drawn by the CTA
     for (;;) {
         int g = 0;
-        if (lane == 0) g = atomicAdd(&prm.rowCtr[l], 1);
-        g = __shfl_sync(0xffffffffu, g, 0);
+        if (preDrawn) {
+            g = firstTicket + (threadIdx.x >> 5);
+            preDrawn = false;
+        } else {
+            if (lane == 0) g = atomicAdd(ticket, 1);
+            g = __shfl_sync(0xffffffffu, g, 0);
+        }
         if (g >= nGroups) break;
         const int k0 = g * R;
         const int4 *rp[R];
 #pragma unroll
         for (int r = 0; r < R; ++r) {
             const int k = k0 + r;
-            rp[r] = reinterpret_cast<const int4 *>(Sl + (int64_t)cand[k < nR ? k : nR - 1] * c.ld);
+            rp[r] = reinterpret_cast<const int4 *>(Sl + (int64_t)__ldcg(cand + (k < nR ? k : nR - 1)) * c.ld);
         }
         GV acc[R][A];                                               // running sums of this lane, [row][block of the lane]
 #pragma unroll
@@ -615,7 +650,7 @@ __device__ __noinline__ void sweep_class_sparse(const GreedyParams<SV> &prm, int
                     const int col = (int)(e[u].x & 0x0fffffffu);
 #pragma unroll
                     for (int a = 0; a < A; ++a) {
-                        const SV cv = myCov[a][col];
+                        const SV cv = __ldcg(myCov[a] + col);
                         if constexpr (Arith<SV>::kInt) {
                             const int dd = (int)e[u].y - cv;
                             d[u][a] = (ok[u] && myPart[a] >= 0 && dd > 0) ? (GV)dd : (GV)0;
@@ -699,8 +734,18 @@ __device__ __noinline__ void sweep_class_sparse(const GreedyParams<SV> &prm, int
             for (int a = 0; a < A; ++a) {
                 GV t = acc[r][a];
                 for (int off = Pp; off < 32; off <<= 1) t += __shfl_xor_sync(0xffffffffu, t, off);
-                if (slot == 0 && k0 + r < nR && myPart[a] >= 0) G[(int64_t)myPart[a] * c.ld + cand[k0 + r]] = t;
+                if (slot == 0 && k0 + r < nR && myPart[a] >= 0) G[(int64_t)myPart[a] * c.ld + __ldcg(cand + k0 + r)] = t;
             }
+        }
+        if (done != nullptr) {
+            // the row group's hit count and gains are in place before the group counts as done
+            __syncwarp();
+            if (lane == 0) {
+                if (hits) atomicAdd(&prm.hitCount[l], (unsigned long long)hits);
+                __threadfence();
+                atomicAdd(done, 1);
+            }
+            hits = 0;
         }
     }
     if (lane == 0 && hits) atomicAdd(&prm.hitCount[l], (unsigned long long)hits);
@@ -759,8 +804,8 @@ __device__ __forceinline__ void sweep_step(const GreedyParams<SV> &prm, int step
             if (threadIdx.x < P) shParts[threadIdx.x] = parts[threadIdx.x];
             __syncthreads();
             uint2 *queue = reinterpret_cast<uint2 *>(reinterpret_cast<char *>(shCover + ld4) + (threadIdx.x >> 5) * kSparseWarpBytes);
-            if (P <= 32) sweep_class_sparse<SV, 1>(prm, l, c, nR, P, shCover, shParts, queue);
-            else sweep_class_sparse<SV, 2>(prm, l, c, nR, P, shCover, shParts, queue);
+            if (P <= 32) sweep_class_sparse<SV, 1>(prm, l, c, nR, P, shCover, shParts, queue, &prm.rowCtr[l], nullptr, -1);
+            else sweep_class_sparse<SV, 2>(prm, l, c, nR, P, shCover, shParts, queue, &prm.rowCtr[l], nullptr, -1);
         } else {
             const int4 *cov = reinterpret_cast<const int4 *>(prm.cover + c.vOff);
             for (int i = threadIdx.x; i < P * ld4; i += blockDim.x) {
@@ -773,10 +818,10 @@ __device__ __forceinline__ void sweep_step(const GreedyParams<SV> &prm, int step
             }
             __syncthreads();
             switch (P) {
-            case 1: sweep_class<SV, 1, 8>(prm, l, c, nR, CS, shCover, shF, shParts, shTicket, shPart); break;
-            case 2: sweep_class<SV, 2, 8>(prm, l, c, nR, CS, shCover, shF, shParts, shTicket, shPart); break;
-            case 4: sweep_class<SV, 4, 8>(prm, l, c, nR, CS, shCover, shF, shParts, shTicket, shPart); break;
-            default: sweep_class<SV, 8, 4>(prm, l, c, nR, CS, shCover, shF, shParts, shTicket, shPart); break;
+            case 1: sweep_class<SV, 1, 8>(prm, l, c, nR, CS, shCover, shF, shParts, shTicket, shPart, &prm.rowCtr[l], nullptr, -1); break;
+            case 2: sweep_class<SV, 2, 8>(prm, l, c, nR, CS, shCover, shF, shParts, shTicket, shPart, &prm.rowCtr[l], nullptr, -1); break;
+            case 4: sweep_class<SV, 4, 8>(prm, l, c, nR, CS, shCover, shF, shParts, shTicket, shPart, &prm.rowCtr[l], nullptr, -1); break;
+            default: sweep_class<SV, 8, 4>(prm, l, c, nR, CS, shCover, shF, shParts, shTicket, shPart, &prm.rowCtr[l], nullptr, -1); break;
             }
         }
         __syncthreads();
@@ -1073,6 +1118,233 @@ __global__ void __launch_bounds__(kSweepThreads, 1) greedy_persistent_kernel(con
 }
 
 // ---------------------------------------------------------------------------------------------
+// The greedy loop without grid-wide phases.  In the kernel above every SM but one per class idles
+// while the classes make their picks.  Classes are independent, so here each class cycles on its own
+// between "being swept" and "making picks", and the picks of one class overlap the sweeps of the
+// others: CTAs [0, nPick) own the classes (class l belongs to CTA l mod nPick) and only make picks,
+// the other CTAs only sweep.  The hand-off is the class's ClassSync word:
+//   pick CTA   waits until epoch is even and done == nGroups (every row group of the published sweep
+//              has written its gains), makes epoch odd, runs the chain of picks (which also fixes
+//              the parameters of the class's next sweep), clears done, and makes epoch even again;
+//   sweep CTA  looks for a published sweep that still has tickets (the class nearest to the CTA's home
+//              position, CTAs being spread evenly over the classes; `asyncGroup` < L serves the sweeps
+//              in batches by publication order instead), reads its parameters between two reads of
+//              epoch (both must give the same even value: the parameters belong to that sweep), draws
+//              one ticket per team from the sweep's own ticket counter, and only then stages the
+//              coverage vectors and sweeps.
+// Every (class, sweep number) has a ticket counter of its own that starts at zero and is never
+// reset, so a CTA that was slow to act on what it read can only draw a ticket beyond the last row
+// group and leaves; a valid ticket is only ever drawn while the class waits for its sweep.  While a
+// class makes its picks, the CTAs at home there help the neighbouring classes.
+// All waits are bounded: a CTA that finds nothing to do for about a second sets the timeout bit, and
+// every loop leaves as soon as the status word is non-zero.
+constexpr unsigned kIdleLimit = 1u << 20;
+
+__device__ __forceinline__ int4 ld_volatile16(const void *p)
+{
+    int4 v;
+    asm volatile("ld.volatile.global.v4.s32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ int32_t ld_volatile32(const int32_t *p) { return *(const volatile int32_t *)p; }
+
+template <typename SV>
+__device__ __forceinline__ void async_pick_cta(const GreedyParams<SV> &prm, int4 *scratch)
+{
+    __shared__ int shEpoch, shFinished;
+    const int me = blockIdx.x;
+    int mine = 0;                                                   // my classes that are not finished
+    for (int l = me; l < prm.L; l += prm.nPick) mine += prm.desc[l].M > 0 ? 1 : 0;
+    unsigned idle = 0;
+    unsigned long long busy = 0;
+    while (mine > 0) {
+        bool progressed = false;
+        for (int l = me; l < prm.L; l += prm.nPick) {
+            if (threadIdx.x == 0) {
+                const int4 sy = ld_volatile16(&prm.sync[l]);           // epoch, nGroups, done, seq
+                int e = -1;
+                if (!(sy.x & 1) && sy.z == sy.y) {
+                    e = sy.x;
+                    *(volatile int32_t *)&prm.sync[l].epoch = e + 1;    // the class is mine until I publish again
+                    __threadfence();                                    // (also: the sweepers' gains are visible)
+                }
+                shEpoch = e;
+            }
+            __syncthreads();
+            const int e = shEpoch;
+            if (e < 0) { __syncthreads(); continue; }
+            progressed = true;
+            unsigned long long t0 = 0;
+            if (me == 0 && threadIdx.x == 0) t0 = global_ns();
+            pick_chain(prm, l, e >> 1, scratch, prm.smemBytes);
+            __syncthreads();                                            // all writes of the chain are issued
+            if (threadIdx.x == 0) {
+                const bool finished = prm.nR[l] == 0 || prm.jstar[l] < 0 || ld_volatile32(prm.status) != 0;
+                if (!finished) {
+                    prm.sync[l].done = 0;
+                    prm.sync[l].seq = prm.L + atomicAdd(prm.pubSeq, 1);
+                    __threadfence();                                    // parameters, coverage, candidate list before the epoch
+                    *(volatile int32_t *)&prm.sync[l].epoch = e + 2;
+                }
+                shFinished = finished ? 1 : 0;
+                if (me == 0) busy += global_ns() - t0;
+            }
+            __syncthreads();
+            if (shFinished) --mine;
+        }
+        if (progressed) {
+            idle = 0;
+        } else {
+            __nanosleep(200);
+            ++idle;
+            if ((idle & 255u) == 0) {                                   // uniform: every thread counts alike
+                if (threadIdx.x == 0) {
+                    int stop = ld_volatile32(prm.status) != 0;
+                    if (!stop && idle >= kIdleLimit) { atomicOr(prm.status, kDevTimeout); stop = 1; }
+                    shFinished = stop;
+                }
+                __syncthreads();
+                const int stop = shFinished;
+                __syncthreads();
+                if (stop) break;
+            }
+        }
+    }
+    if (me == 0 && threadIdx.x == 0) prm.phaseNs[1] = busy;
+}
+
+template <typename SV>
+__device__ __forceinline__ void async_sweep_cta(const GreedyParams<SV> &prm, int4 *shCover)
+{
+    using GV = typename Arith<SV>::GV;
+    __shared__ long long shF[kMaxSweepBatch];
+    __shared__ int32_t shParts[kSparseMax];
+    __shared__ int shTicket[kSweepThreads / 32];
+    __shared__ GV shPart[kSweepThreads];
+    __shared__ unsigned long long shBest;
+    __shared__ int shInfo[12];                                      // ok, first ticket, nR, P, CS, mode, nGroups, stop, sweep number, epoch
+    const bool clocked = blockIdx.x == prm.nPick;                   // the first sweep CTA keeps the busy clock
+    const int home = (int)(((int64_t)(blockIdx.x - prm.nPick) * prm.L) / (gridDim.x - prm.nPick));
+    unsigned idle = 0;
+    unsigned long long busy = 0;
+    for (;;) {
+        // The sweep to serve: sweeps are served in the order they were published, asyncGroup of them
+        // together; inside such a batch a CTA goes to the class nearest to its home position (CTAs spread
+        // evenly over the classes), so that a CTA visits few classes per batch.
+        if (threadIdx.x == 0) shBest = ~0ull;
+        __syncthreads();
+        for (int l = threadIdx.x; l < prm.L; l += blockDim.x) {
+            const int4 sy = ld_volatile16(&prm.sync[l]);            // epoch, nGroups, done, seq
+            if (!(sy.x & 1)) {
+                const int32_t drawn = ld_volatile32(prm.tickets + prm.desc[l].row0 + l + (sy.x >> 1));
+                if (drawn < sy.y) {
+                    int dist = l - home;
+                    if (dist < 0) dist += prm.L;
+                    const unsigned long long key = ((unsigned long long)(unsigned)(sy.w / prm.asyncGroup) << 40) |
+                                                   ((unsigned long long)(unsigned)dist << 20) | (unsigned)l;
+                    atomicMin(&shBest, key);
+                }
+            }
+        }
+        __syncthreads();
+        const unsigned long long best = shBest;
+        if (best == ~0ull) {
+            if (threadIdx.x == 0) {
+                int stop = (ld_volatile32(&prm.nSweep[3]) == 0 || ld_volatile32(prm.status) != 0) ? 1 : 0;
+                if (!stop && ++idle >= kIdleLimit) { atomicOr(prm.status, kDevTimeout); stop = 1; }
+                shInfo[7] = stop;
+            }
+            __syncthreads();
+            const int stop = shInfo[7];
+            __syncthreads();
+            if (stop) break;
+            __nanosleep(200);
+            continue;
+        }
+        const int l = (int)(unsigned)(best & 0xfffffull);
+        const ClassDesc c = prm.desc[l];
+        const int32_t *parts = prm.sweepParts + (int64_t)l * kSparseMax;
+        // Parameters of the sweep, read between two reads of the epoch.  Every load here is volatile (served
+        // by L2), and the bulk data of a sweep (coverage, threshold, candidate list) is read with ld.cg, so
+        // no stale L1 line can be seen; the barriers keep the three groups of loads in order.
+        if (threadIdx.x == 0) shInfo[9] = ld_volatile32(&prm.sync[l].epoch);
+        __syncthreads();
+        if (threadIdx.x < kSparseMax) shParts[threadIdx.x] = ld_volatile32(parts + threadIdx.x);
+        if (threadIdx.x == 64) {
+            shInfo[2] = ld_volatile32(&prm.nR[l]);
+            shInfo[3] = ld_volatile32(&prm.sweepN[l]);
+            shInfo[4] = ld_volatile32(&prm.sweepCS[l]);
+            shInfo[5] = ld_volatile32(&prm.sweepMode[l]);
+        }
+        if (threadIdx.x == 96) shInfo[6] = ld_volatile32(&prm.sync[l].nGroups);
+        if constexpr (Arith<SV>::kInt) {
+            if (threadIdx.x >= 128 && threadIdx.x < 128 + kMaxSweepBatch) {
+                int p = ld_volatile32(parts + (threadIdx.x - 128));
+                if (p < 0 || p >= prm.W) p = 0;                     // (only when the read raced with an update; discarded below)
+                shF[threadIdx.x - 128] = *(const volatile long long *)&prm.fval[(int64_t)l * prm.W + p];
+            }
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            const int e1 = shInfo[9];
+            const int e2 = ld_volatile32(&prm.sync[l].epoch);
+            int ok = (e1 == e2 && !(e1 & 1)) ? 1 : 0;
+            int first = -1;
+            if (ok) {
+                // one ticket per team, drawn before the coverage vectors are staged
+                const int teams = (kSweepThreads / 32) / (shInfo[5] ? 1 : shInfo[4]);
+                first = atomicAdd(prm.tickets + c.row0 + l + (e1 >> 1), teams);
+                if (first >= shInfo[6]) ok = 0;
+            }
+            shInfo[0] = ok;
+            shInfo[1] = first;
+            shInfo[8] = e1 >> 1;
+        }
+        __syncthreads();
+        if (!shInfo[0]) continue;                                   // another look at the sweeps
+        idle = 0;
+        unsigned long long t0 = 0;
+        if (clocked && threadIdx.x == 0) t0 = global_ns();
+        const int nR = shInfo[2], P = shInfo[3], CS = shInfo[4], first = shInfo[1];
+        const int ld4 = c.ld >> 2;
+        int32_t *ticket = prm.tickets + c.row0 + l + shInfo[8];      // the counter of this sweep alone
+        int32_t *done = &prm.sync[l].done;
+        if (shInfo[5]) {
+            const int4 *thr = reinterpret_cast<const int4 *>(prm.thr + c.vOff / prm.W);
+            for (int i = threadIdx.x; i < ld4; i += blockDim.x) shCover[i] = __ldcg(thr + i);
+            __syncthreads();
+            uint2 *queue = reinterpret_cast<uint2 *>(reinterpret_cast<char *>(shCover + ld4) + (threadIdx.x >> 5) * kSparseWarpBytes);
+            if (P <= 32) sweep_class_sparse<SV, 1>(prm, l, c, nR, P, shCover, shParts, queue, ticket, done, first);
+            else sweep_class_sparse<SV, 2>(prm, l, c, nR, P, shCover, shParts, queue, ticket, done, first);
+        } else {
+            const int4 *cov = reinterpret_cast<const int4 *>(prm.cover + c.vOff);
+            for (int i = threadIdx.x; i < P * ld4; i += blockDim.x) {
+                int p = i / ld4, cc = i - p * ld4;
+                shCover[i] = __ldcg(cov + (int64_t)shParts[p] * ld4 + cc);
+            }
+            __syncthreads();
+            switch (P) {
+            case 1: sweep_class<SV, 1, 8>(prm, l, c, nR, CS, shCover, shF, shParts, shTicket, shPart, ticket, done, first); break;
+            case 2: sweep_class<SV, 2, 8>(prm, l, c, nR, CS, shCover, shF, shParts, shTicket, shPart, ticket, done, first); break;
+            case 4: sweep_class<SV, 4, 8>(prm, l, c, nR, CS, shCover, shF, shParts, shTicket, shPart, ticket, done, first); break;
+            default: sweep_class<SV, 8, 4>(prm, l, c, nR, CS, shCover, shF, shParts, shTicket, shPart, ticket, done, first); break;
+            }
+        }
+        __syncthreads();
+        if (clocked && threadIdx.x == 0) busy += global_ns() - t0;
+    }
+    if (clocked && threadIdx.x == 0) prm.phaseNs[0] = busy;
+}
+
+template <typename SV>
+__global__ void __launch_bounds__(kSweepThreads, 1) greedy_async_kernel(const __grid_constant__ GreedyParams<SV> prm)
+{
+    extern __shared__ int4 shCover[];
+    if ((int)blockIdx.x < prm.nPick) async_pick_cta(prm, shCover);
+    else async_sweep_cta(prm, shCover);
+}
+
+// ---------------------------------------------------------------------------------------------
 // Launch with programmatic stream serialization: the next kernel's CTAs may be placed while this
 // one drains; every kernel starts with cudaGridDependencySynchronize(), so data dependencies hold.
 template <typename... KArgs, typename... Args>
@@ -1138,7 +1410,12 @@ static rcd_status run_greedy(rcd_ctx *ctx, const Sizes &sz, const Workspace &ws,
     prm.sweepWarps = ctx->smCount * (kSweepThreads / 32);
     prm.one = 1u;
     prm.sparseMinMembers = ctx->cfg.sweep_mode == 1 ? -1 : 8;
-
+    prm.sync = ws.sync;
+    prm.tickets = ws.tickets;
+    prm.pubSeq = ws.nSweep;             // (the sweep lists and their counters are not used by the asynchronous kernel)
+    prm.asyncMode = 0;
+    prm.nPick = 0;
+    prm.asyncGroup = 1;
     int maxLd = 0;
     for (const auto &c : descHost) if (c.ld > maxLd) maxLd = c.ld;
     const int64_t smemCap = (int64_t)ctx->maxSmemOptin - 20 * 1024;  // static shared of the kernels + margin
@@ -1162,6 +1439,32 @@ static rcd_status run_greedy(rcd_ctx *ctx, const Sizes &sz, const Workspace &ws,
     }
     RCD_CUDA(ctx, cudaFuncSetAttribute(sweep_kernel<SV>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
 
+    // Which form of the loop: greedy_path 1 = two launches per round, 2 = one launch, rounds with grid
+    // barriers, 3 = one launch, asynchronous classes, 0 = choose.  With few classes the pick phases of
+    // the round-based kernel leave most SMs idle, and giving every class a pick CTA of its own costs
+    // few SMs: the asynchronous kernel is chosen when there are at most a quarter as many classes as SMs.
+    const bool perSweep = ctx->cfg.profile >= 2;
+    int path = ctx->cfg.greedy_path;
+    if (perSweep || !ctx->cooperative) path = 1;
+    if (path == 0) path = (sz.L * 4 <= ctx->smCount) ? 3 : 2;
+    if (path == 3 && ctx->smCount < 2) path = 2;
+    if (path == 2 || path == 3) {
+        // one cooperative launch needs one CTA per SM resident at once
+        RCD_CUDA(ctx, cudaFuncSetAttribute(greedy_persistent_kernel<SV>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        RCD_CUDA(ctx, cudaFuncSetAttribute(greedy_async_kernel<SV>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        int perSm = 0;
+        if (path == 3) RCD_CUDA(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&perSm, greedy_async_kernel<SV>, kSweepThreads, (size_t)smem));
+        else RCD_CUDA(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&perSm, greedy_persistent_kernel<SV>, kSweepThreads, (size_t)smem));
+        if (perSm < 1) path = 1;
+    }
+    if (path == 3) {
+        prm.asyncMode = 1;
+        prm.nPick = std::min<int>(sz.L, std::max(1, ctx->smCount / 4));
+        prm.sweepWarps = (ctx->smCount - prm.nPick) * (kSweepThreads / 32);
+        prm.asyncGroup = ctx->cfg.async_group > 0 ? ctx->cfg.async_group : std::max<int>(sz.L, 1);
+    }
+
+    if (path == 3) RCD_CUDA(ctx, cudaMemsetAsync(ws.tickets, 0, (size_t)(sz.N + sz.L) * sizeof(int32_t), st));
     RCD_CUDA(ctx, cudaMemsetAsync(ws.nSweep, 0, 4 * sizeof(int32_t), st));
     RCD_CUDA(ctx, cudaMemsetAsync(ws.phaseNs, 0, 6 * sizeof(unsigned long long), st));
     ctx->phaseNsDev = ws.phaseNs;
@@ -1171,18 +1474,16 @@ static rcd_status run_greedy(rcd_ctx *ctx, const Sizes &sz, const Workspace &ws,
     ctx->kernelLaunches++;
     RCD_CUDA(ctx, cudaGetLastError());
 
-    const bool perSweep = ctx->cfg.profile >= 2;
     ctx->sweepEventsUsed = 0;
     // One cooperative launch for the whole loop when the device can hold one sweep CTA per SM at once;
     // per-sweep event timing (profile 2) needs the sweeps as separate launches.
-    bool persistent = ctx->cfg.greedy_path != 1 && !perSweep && ctx->cooperative;
-    if (persistent) {
-        RCD_CUDA(ctx, cudaFuncSetAttribute(greedy_persistent_kernel<SV>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        int perSm = 0;
-        RCD_CUDA(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&perSm, greedy_persistent_kernel<SV>, kSweepThreads, (size_t)smem));
-        if (perSm < 1) persistent = false;
-    }
-    if (persistent) {
+    const bool persistent = path != 1;
+    if (persistent && path == 3) {
+        void *args[] = {(void *)&prm};
+        RCD_CUDA(ctx, cudaLaunchCooperativeKernel((const void *)greedy_async_kernel<SV>, dim3(ctx->smCount), dim3(kSweepThreads),
+                                                  args, (size_t)smem, st));
+        ctx->kernelLaunches += 1;
+    } else if (persistent) {
         int steps = (int)sz.maxM;
         void *args[] = {(void *)&prm, (void *)&steps};
         RCD_CUDA(ctx, cudaLaunchCooperativeKernel((const void *)greedy_persistent_kernel<SV>, dim3(ctx->smCount), dim3(kSweepThreads),

@@ -26,6 +26,16 @@ enum : int {
     kDevTimeout = 8,           // a bounded wait inside a kernel ran out
 };
 
+// Hand-off word of one class between the CTA that makes its picks and the CTAs that sweep it (the
+// asynchronous greedy kernel).  `epoch` is a sequence lock: even = sweep number epoch/2 is published
+// and its parameters are stable, odd = the class belongs to its pick CTA (or is finished).
+struct ClassSync {
+    int32_t epoch;
+    int32_t nGroups;  // row groups (tickets) of the published sweep
+    int32_t done;     // row groups of the published sweep whose gains are written
+    int32_t seq;      // publication number: sweeps are served oldest first
+};
+
 // One class, as the kernels see it.  Built on the host once the class sizes are known.
 struct ClassDesc {
     int32_t M;        // samples in the class
@@ -97,6 +107,8 @@ struct Workspace {
     int32_t *sparseFrom;    // [L]
     int32_t *sweepCS;       // [L] warps per row group in the next sweep
     int32_t *rowCtr;        // [L] ticket counter over row groups of the running sweep
+    ClassSync *sync;        // [L] asynchronous kernel: hand-off words
+    int32_t *tickets;       // [N + L] asynchronous kernel: one ticket counter per (class, sweep number), never reused
     int32_t *sweepList;     // [3][L] classes that sweep in a step (three lists in rotation)
     int32_t *nSweep;        // [3] (+1 pad)
     unsigned long long *stepBytes;   // [steps+1] bytes the sweep of step t has to read

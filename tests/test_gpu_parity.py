@@ -98,7 +98,7 @@ def check_exact(rcd, orc, wl, variant="incremental", **cfg):
     return a, o, v, ref
 
 
-@pytest.mark.parametrize("path", [0, 1])        # one cooperative launch / two launches per step
+@pytest.mark.parametrize("path", [0, 1, 2, 3])  # chosen by the library / two launches per round / one launch with rounds / asynchronous
 @pytest.mark.parametrize("batch", [1, 2, 4, 8])
 def test_partition_c1_exact(rcd, orc, batch, path):
     from paper_2211_00839_b200.workloads import make_workload
@@ -128,7 +128,7 @@ def test_partition_int8_ragged_classes(rcd, orc, seed):
     caps = np.array([1, 2.5, 1, 4, 0.5, 3, 1, 1, 2], dtype=np.float64)
     wl = Workload("ragged", "int8", np.ascontiguousarray(feats[perm]), np.ascontiguousarray(labels[perm]), caps,
                   len(sizes), len(caps))
-    for batch, path in ((8, 0), (1, 0), (8, 1)):
+    for batch, path in ((8, 0), (1, 0), (8, 1), (8, 2), (8, 3), (2, 3)):
         check_exact(rcd, orc, wl, sweep_batch_max=batch, greedy_path=path)
 
 
@@ -153,6 +153,22 @@ def test_partition_c5_reduced_exact(rcd, orc):
     from paper_2211_00839_b200.workloads import make_workload
     wl = make_workload("C5", L=6, M=700, d=256)
     check_exact(rcd, orc, wl)
+
+
+@pytest.mark.parametrize("path", [2, 3])
+def test_partition_many_small_classes_every_loop_form(rcd, orc, path):
+    """More classes than pick CTAs of the asynchronous loop (a pick CTA then serves several classes), of
+    unequal sizes so that classes finish at different times; W = 64 with threshold passes."""
+    from paper_2211_00839_b200.workloads import Workload, make_workload
+    base = make_workload("C5", L=60, M=160, d=128)
+    rng = np.random.default_rng(7)
+    keep = np.ones(base.N, bool)
+    for l in range(base.L):                       # thin every class by a different amount
+        ids = np.nonzero(base.labels == l)[0]
+        keep[ids[:int(rng.integers(0, 100))]] = False
+    wl = Workload("many", "int8", np.ascontiguousarray(base.features[keep]), np.ascontiguousarray(base.labels[keep]),
+                  base.capacities, base.L, base.W)
+    check_exact(rcd, orc, wl, greedy_path=path)
 
 
 def test_partition_is_reproducible(rcd):
@@ -205,7 +221,7 @@ def test_partition_c3_reduced_float(rcd, orc):
     check_float(rcd, orc, wl)
 
 
-@pytest.mark.parametrize("batch,path", [(1, 0), (8, 0), (8, 1)])
+@pytest.mark.parametrize("batch,path", [(1, 0), (8, 0), (8, 1), (8, 2), (8, 3)])
 def test_partition_c4_reduced_float(rcd, orc, batch, path):
     from paper_2211_00839_b200.workloads import make_workload
     wl = make_workload("C4", L=5, M=500, d=256)
@@ -222,7 +238,7 @@ def run_with_profile(rcd, wl, **cfg):
         return a.cpu().numpy(), o.cpu().numpy(), v.cpu().numpy(), ctx.profile()
 
 
-@pytest.mark.parametrize("path", [0, 1])
+@pytest.mark.parametrize("path", [0, 1, 2, 3])
 def test_threshold_passes_int8_exact(rcd, orc, path):
     """Classes large enough that the sweeps switch to threshold passes: same picks as the oracle, and
     the same as with dense passes only."""
