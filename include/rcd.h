@@ -87,9 +87,9 @@ typedef struct {
     int32_t objective;         /* rcd_objective_kind used by rcd_partition / rcd_objective (default facility location) */
     int32_t sweep_mode;        /* 0 = threshold passes once the blocks have a few members (up to 64 blocks per pass);
                                   1 = dense passes only (sweep_batch_max blocks per pass) */
-    int32_t async_group;       /* greedy_path 3: sweeps published one after another that the sweep CTAs serve together,
-                                  each CTA going to the class nearest its home position; 1 = strictly oldest first;
-                                  0 = default: all classes together */
+    int32_t async_group;       /* greedy_path 3: how many sweeps (ordered by sweep number, then class) the sweep CTAs serve
+                                  together, each CTA going to the class nearest its home position; 1 = strictly in
+                                  order; 0 = default: all classes together */
     int32_t reserved[8];       /* must be 0 */
 } rcd_config;
 

@@ -113,8 +113,8 @@ static Sizes bound_sizes(const rcd_ctx *ctx, rcd_feat_dtype dtype, int64_t N, in
     sz.N = N; sz.d = d; sz.L = L; sz.W = W;
     if (Mmax > N) Mmax = N;
     sz.maxM = Mmax;
-    sz.sElems = N * (int64_t)pad4(Mmax);                  // sum M_l * ld_l <= N * pad4(Mmax)
-    sz.vElems = (int64_t)W * (N + 3LL * L);               // sum W * ld_l,  ld_l <= M_l + 3
+    sz.sElems = N * (int64_t)pad_row(Mmax);               // sum M_l * ld_l <= N * pad_row(Mmax)
+    sz.vElems = (int64_t)W * (N + 7LL * L);               // sum W * ld_l,  ld_l <= M_l + 7
     sz.nChunks = chunks_for(N);
     return sz;
 }
@@ -214,7 +214,7 @@ static rcd_status prepare(rcd_ctx *ctx, const void *features, rcd_feat_dtype dty
     for (int32_t l = 0; l < L; ++l) {
         ClassDesc c{};
         c.M = ctx->hostStage[l];
-        c.ld = pad4(c.M);
+        c.ld = pad_row(c.M);
         c.row0 = (int32_t)row;
         c.sOff = sOff;
         c.vOff = vOff;

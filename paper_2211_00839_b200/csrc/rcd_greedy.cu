@@ -86,7 +86,6 @@ struct GreedyParams {
     // asynchronous kernel (greedy_async_kernel); asyncMode = 0 everywhere else
     ClassSync *sync;            // [L] hand-off words
     int32_t *tickets;           // [N + L] ticket counter of sweep k of class l at tickets[row0_l + l + k]
-    int32_t *pubSeq;            // publication counter (orders the sweeps: oldest first)
     int32_t asyncMode;
     int32_t nPick;              // CTAs [0, nPick) make picks, the others sweep
     int32_t asyncGroup;         // sweeps published one after another that are served together (by CTA home position)
@@ -130,6 +129,12 @@ constexpr int kSparseStages = 8;                                   // threshold 
 constexpr int kSparseRingBytes = kSparseStages * kSparseRows * 512;   // rows x 32 lanes x 16 bytes per stage
 constexpr int kSparseWarpBytes = kSparseRingBytes + kSparseQueue * 8; // ring + queue
 constexpr int kSparseQueueBytes = kSparseWarpBytes * (kSweepThreads / 32);
+// The rings are the destination of 16-byte asynchronous copies whose sources (rows of S) start on 32-byte
+// boundaries: the dynamic shared memory is declared 128-byte aligned and the rings start on a 128-byte
+// boundary behind the threshold vector, so that a copy never straddles two 32-byte sectors (a ring that
+// starts 16 bytes off such a boundary doubles the sectors fetched per copy).
+__host__ __device__ inline int thr_bytes_aligned(int bytes) { return (bytes + 127) & ~127; }
+static_assert(kSparseWarpBytes % 128 == 0, "per-warp rings must keep the 128-byte alignment");
 
 template <typename SV>
 __device__ void plan_decide(const GreedyParams<SV> &prm, int l, const ClassDesc &c, int nR, int nextStep,
@@ -206,7 +211,7 @@ __device__ void plan_decide(const GreedyParams<SV> &prm, int l, const ClassDesc 
     from = __shfl_sync(0xffffffffu, from, 0);
     const int64_t together0 = max(*(volatile int32_t *)&prm.nSweep[3], 1);
     const bool sparse = prm.sparseMinMembers >= 0 && prm.batchMax > 1 && nStale > 1 && fewest >= from &&
-                        (int64_t)c.ld * (int64_t)sizeof(SV) + kSparseQueueBytes <= prm.smemBytes &&
+                        (int64_t)thr_bytes_aligned(c.ld * (int)sizeof(SV)) + kSparseQueueBytes <= prm.smemBytes &&
                         together0 * ((nR + kSparseRows - 1) / kSparseRows) * 4 >= prm.sweepWarps;
     if (sparse) cap = kSparseMax;
     // n blocks are refreshed; the dense pass is instantiated for lists of 1, 2, 4, 8, so its list is
@@ -803,7 +808,7 @@ __device__ __forceinline__ void sweep_step(const GreedyParams<SV> &prm, int step
             for (int i = threadIdx.x; i < ld4; i += blockDim.x) shCover[i] = thr[i];
             if (threadIdx.x < P) shParts[threadIdx.x] = parts[threadIdx.x];
             __syncthreads();
-            uint2 *queue = reinterpret_cast<uint2 *>(reinterpret_cast<char *>(shCover + ld4) + (threadIdx.x >> 5) * kSparseWarpBytes);
+            uint2 *queue = reinterpret_cast<uint2 *>(reinterpret_cast<char *>(shCover) + thr_bytes_aligned(c.ld * (int)sizeof(SV)) + (threadIdx.x >> 5) * kSparseWarpBytes);
             if (P <= 32) sweep_class_sparse<SV, 1>(prm, l, c, nR, P, shCover, shParts, queue, &prm.rowCtr[l], nullptr, -1);
             else sweep_class_sparse<SV, 2>(prm, l, c, nR, P, shCover, shParts, queue, &prm.rowCtr[l], nullptr, -1);
         } else {
@@ -831,7 +836,7 @@ __device__ __forceinline__ void sweep_step(const GreedyParams<SV> &prm, int step
 template <typename SV>
 __global__ void __launch_bounds__(kSweepThreads, 1) sweep_kernel(const __grid_constant__ GreedyParams<SV> prm, int step)
 {
-    extern __shared__ int4 shCover[];
+    extern __shared__ __align__(128) int4 shCover[];
     cudaGridDependencySynchronize();              // the previous launch (select / init) has finished
     cudaTriggerProgrammaticLaunchCompletion();
     sweep_step(prm, step, shCover);
@@ -1091,7 +1096,7 @@ __device__ __forceinline__ unsigned long long global_ns()
 template <typename SV>
 __global__ void __launch_bounds__(kSweepThreads, 1) greedy_persistent_kernel(const __grid_constant__ GreedyParams<SV> prm, int maxRounds)
 {
-    extern __shared__ int4 shCover[];
+    extern __shared__ __align__(128) int4 shCover[];
     __shared__ unsigned long long shClock[3];      // last stamp, sweep-phase ns, pick-phase ns (CTA 0, thread 0)
     if (blockIdx.x == 0 && threadIdx.x == 0) { shClock[0] = global_ns(); shClock[1] = 0; shClock[2] = 0; }
     for (int r = 0; r < maxRounds; ++r) {
@@ -1182,7 +1187,7 @@ __device__ __forceinline__ void async_pick_cta(const GreedyParams<SV> &prm, int4
                 const bool finished = prm.nR[l] == 0 || prm.jstar[l] < 0 || ld_volatile32(prm.status) != 0;
                 if (!finished) {
                     prm.sync[l].done = 0;
-                    prm.sync[l].seq = prm.L + atomicAdd(prm.pubSeq, 1);
+                    prm.sync[l].seq = ((e >> 1) + 1) * prm.L + l;        // sweep number first: batches follow the classes' progress
                     __threadfence();                                    // parameters, coverage, candidate list before the epoch
                     *(volatile int32_t *)&prm.sync[l].epoch = e + 2;
                 }
@@ -1228,11 +1233,14 @@ __device__ __forceinline__ void async_sweep_cta(const GreedyParams<SV> &prm, int
     unsigned idle = 0;
     unsigned long long busy = 0;
     for (;;) {
-        // The sweep to serve: sweeps are served in the order they were published, asyncGroup of them
+        // The sweep to serve: sweeps are served by order number (sweep number first), asyncGroup of them
         // together; inside such a batch a CTA goes to the class nearest to its home position (CTAs spread
-        // evenly over the classes), so that a CTA visits few classes per batch.
+        // evenly over the classes), so that a CTA visits few classes per batch.  By default a batch is
+        // every class.
         if (threadIdx.x == 0) shBest = ~0ull;
         __syncthreads();
+        unsigned long long myKey = ~0ull;
+        int myEpoch = 0;
         for (int l = threadIdx.x; l < prm.L; l += blockDim.x) {
             const int4 sy = ld_volatile16(&prm.sync[l]);            // epoch, nGroups, done, seq
             if (!(sy.x & 1)) {
@@ -1242,10 +1250,11 @@ __device__ __forceinline__ void async_sweep_cta(const GreedyParams<SV> &prm, int
                     if (dist < 0) dist += prm.L;
                     const unsigned long long key = ((unsigned long long)(unsigned)(sy.w / prm.asyncGroup) << 40) |
                                                    ((unsigned long long)(unsigned)dist << 20) | (unsigned)l;
-                    atomicMin(&shBest, key);
+                    if (key < myKey) { myKey = key; myEpoch = sy.x; }
                 }
             }
         }
+        if (myKey != ~0ull) atomicMin(&shBest, myKey);
         __syncthreads();
         const unsigned long long best = shBest;
         if (best == ~0ull) {
@@ -1263,13 +1272,18 @@ __device__ __forceinline__ void async_sweep_cta(const GreedyParams<SV> &prm, int
         }
         const int l = (int)(unsigned)(best & 0xfffffull);
         const ClassDesc c = prm.desc[l];
+        const int ld4 = c.ld >> 2;
         const int32_t *parts = prm.sweepParts + (int64_t)l * kSparseMax;
-        // Parameters of the sweep, read between two reads of the epoch.  Every load here is volatile (served
-        // by L2), and the bulk data of a sweep (coverage, threshold, candidate list) is read with ld.cg, so
-        // no stale L1 line can be seen; the barriers keep the three groups of loads in order.
-        if (threadIdx.x == 0) shInfo[9] = ld_volatile32(&prm.sync[l].epoch);
-        __syncthreads();
-        if (threadIdx.x < kSparseMax) shParts[threadIdx.x] = ld_volatile32(parts + threadIdx.x);
+        // Parameters of the sweep, read between two reads of the epoch: the first is the scan's, the second
+        // comes after the parameters.  Every load here is volatile (served by L2), and the bulk data of a
+        // sweep (coverage, threshold, candidate list) is read with ld.cg, so no stale L1 line can be seen;
+        // the barriers keep the groups of loads in order.
+        if (myKey == best) shInfo[9] = myEpoch;
+        if (threadIdx.x < kSparseMax) {
+            int bp = ld_volatile32(parts + threadIdx.x);
+            if (bp < 0 || bp >= prm.W) bp = 0;                      // (beyond the list, or a read that raced with an update)
+            shParts[threadIdx.x] = bp;
+        }
         if (threadIdx.x == 64) {
             shInfo[2] = ld_volatile32(&prm.nR[l]);
             shInfo[3] = ld_volatile32(&prm.sweepN[l]);
@@ -1280,49 +1294,55 @@ __device__ __forceinline__ void async_sweep_cta(const GreedyParams<SV> &prm, int
         if constexpr (Arith<SV>::kInt) {
             if (threadIdx.x >= 128 && threadIdx.x < 128 + kMaxSweepBatch) {
                 int p = ld_volatile32(parts + (threadIdx.x - 128));
-                if (p < 0 || p >= prm.W) p = 0;                     // (only when the read raced with an update; discarded below)
+                if (p < 0 || p >= prm.W) p = 0;
                 shF[threadIdx.x - 128] = *(const volatile long long *)&prm.fval[(int64_t)l * prm.W + p];
             }
         }
         __syncthreads();
+        // Second read of the epoch, and with it -- before its answer is known -- one ticket per team is
+        // drawn and the threshold / coverage vectors are staged.  Should the epoch turn out to have moved,
+        // the class had been taken back by its pick CTA, which happens only after every row group of the
+        // sweep is done: the tickets drawn were beyond the last row group, and what was staged is dropped.
+        const int mode = shInfo[5];
+        int P = shInfo[3], CS = shInfo[4];
+        if (CS != 1 && CS != 2 && CS != 4 && CS != 8 && CS != 16) CS = 1;
         if (threadIdx.x == 0) {
             const int e1 = shInfo[9];
+            const int teams = (kSweepThreads / 32) / (mode ? 1 : CS);
+            const int first = atomicAdd(prm.tickets + c.row0 + l + (e1 >> 1), teams);
             const int e2 = ld_volatile32(&prm.sync[l].epoch);
-            int ok = (e1 == e2 && !(e1 & 1)) ? 1 : 0;
-            int first = -1;
-            if (ok) {
-                // one ticket per team, drawn before the coverage vectors are staged
-                const int teams = (kSweepThreads / 32) / (shInfo[5] ? 1 : shInfo[4]);
-                first = atomicAdd(prm.tickets + c.row0 + l + (e1 >> 1), teams);
-                if (first >= shInfo[6]) ok = 0;
-            }
-            shInfo[0] = ok;
+            shInfo[0] = (e1 == e2 && !(e1 & 1) && first < shInfo[6]) ? 1 : 0;
             shInfo[1] = first;
             shInfo[8] = e1 >> 1;
+        }
+        if (mode) {
+            const int4 *thr = reinterpret_cast<const int4 *>(prm.thr + c.vOff / prm.W);
+            if ((int64_t)thr_bytes_aligned(c.ld * (int)sizeof(SV)) + kSparseQueueBytes <= prm.smemBytes)
+                for (int i = threadIdx.x; i < ld4; i += blockDim.x) shCover[i] = __ldcg(thr + i);
+        } else {
+            if (P != 1 && P != 2 && P != 4 && P != 8) P = 1;
+            const int4 *cov = reinterpret_cast<const int4 *>(prm.cover + c.vOff);
+            if ((int64_t)P * c.ld * (int64_t)sizeof(SV) <= prm.smemBytes) {
+                for (int i = threadIdx.x; i < P * ld4; i += blockDim.x) {
+                    int p = i / ld4, cc = i - p * ld4;
+                    shCover[i] = __ldcg(cov + (int64_t)shParts[p] * ld4 + cc);
+                }
+            }
         }
         __syncthreads();
         if (!shInfo[0]) continue;                                   // another look at the sweeps
         idle = 0;
         unsigned long long t0 = 0;
         if (clocked && threadIdx.x == 0) t0 = global_ns();
-        const int nR = shInfo[2], P = shInfo[3], CS = shInfo[4], first = shInfo[1];
-        const int ld4 = c.ld >> 2;
+        const int nR = shInfo[2], first = shInfo[1];
         int32_t *ticket = prm.tickets + c.row0 + l + shInfo[8];      // the counter of this sweep alone
         int32_t *done = &prm.sync[l].done;
-        if (shInfo[5]) {
-            const int4 *thr = reinterpret_cast<const int4 *>(prm.thr + c.vOff / prm.W);
-            for (int i = threadIdx.x; i < ld4; i += blockDim.x) shCover[i] = __ldcg(thr + i);
-            __syncthreads();
-            uint2 *queue = reinterpret_cast<uint2 *>(reinterpret_cast<char *>(shCover + ld4) + (threadIdx.x >> 5) * kSparseWarpBytes);
+        if (mode) {
+            P = shInfo[3];
+            uint2 *queue = reinterpret_cast<uint2 *>(reinterpret_cast<char *>(shCover) + thr_bytes_aligned(c.ld * (int)sizeof(SV)) + (threadIdx.x >> 5) * kSparseWarpBytes);
             if (P <= 32) sweep_class_sparse<SV, 1>(prm, l, c, nR, P, shCover, shParts, queue, ticket, done, first);
             else sweep_class_sparse<SV, 2>(prm, l, c, nR, P, shCover, shParts, queue, ticket, done, first);
         } else {
-            const int4 *cov = reinterpret_cast<const int4 *>(prm.cover + c.vOff);
-            for (int i = threadIdx.x; i < P * ld4; i += blockDim.x) {
-                int p = i / ld4, cc = i - p * ld4;
-                shCover[i] = __ldcg(cov + (int64_t)shParts[p] * ld4 + cc);
-            }
-            __syncthreads();
             switch (P) {
             case 1: sweep_class<SV, 1, 8>(prm, l, c, nR, CS, shCover, shF, shParts, shTicket, shPart, ticket, done, first); break;
             case 2: sweep_class<SV, 2, 8>(prm, l, c, nR, CS, shCover, shF, shParts, shTicket, shPart, ticket, done, first); break;
@@ -1339,7 +1359,7 @@ __device__ __forceinline__ void async_sweep_cta(const GreedyParams<SV> &prm, int
 template <typename SV>
 __global__ void __launch_bounds__(kSweepThreads, 1) greedy_async_kernel(const __grid_constant__ GreedyParams<SV> prm)
 {
-    extern __shared__ int4 shCover[];
+    extern __shared__ __align__(128) int4 shCover[];
     if ((int)blockIdx.x < prm.nPick) async_pick_cta(prm, shCover);
     else async_sweep_cta(prm, shCover);
 }
@@ -1412,7 +1432,6 @@ static rcd_status run_greedy(rcd_ctx *ctx, const Sizes &sz, const Workspace &ws,
     prm.sparseMinMembers = ctx->cfg.sweep_mode == 1 ? -1 : 8;
     prm.sync = ws.sync;
     prm.tickets = ws.tickets;
-    prm.pubSeq = ws.nSweep;             // (the sweep lists and their counters are not used by the asynchronous kernel)
     prm.asyncMode = 0;
     prm.nPick = 0;
     prm.asyncGroup = 1;
@@ -1421,7 +1440,7 @@ static rcd_status run_greedy(rcd_ctx *ctx, const Sizes &sz, const Workspace &ws,
     const int64_t smemCap = (int64_t)ctx->maxSmemOptin - 20 * 1024;  // static shared of the kernels + margin
     int64_t smem = (int64_t)batch * maxLd * (int64_t)sizeof(SV);
     if (prm.sparseMinMembers >= 0)                                   // threshold pass: one vector + the warps' rings and queues
-        smem = std::max<int64_t>(smem, (int64_t)maxLd * (int64_t)sizeof(SV) + kSparseQueueBytes);
+        smem = std::max<int64_t>(smem, (int64_t)thr_bytes_aligned(maxLd * (int)sizeof(SV)) + kSparseQueueBytes);
     if (smem > smemCap) smem = smemCap;
     if ((int64_t)maxLd * (int64_t)sizeof(SV) > smem)
         return fail(ctx, RCD_ERR_UNSUPPORTED,

@@ -33,13 +33,14 @@ struct ClassSync {
     int32_t epoch;
     int32_t nGroups;  // row groups (tickets) of the published sweep
     int32_t done;     // row groups of the published sweep whose gains are written
-    int32_t seq;      // publication number: sweeps are served oldest first
+    int32_t seq;      // order number of the published sweep (sweep number x L + class)
+    int32_t pad_[4];  // one 32-byte sector per class: the counters of two classes never share one
 };
 
 // One class, as the kernels see it.  Built on the host once the class sizes are known.
 struct ClassDesc {
     int32_t M;        // samples in the class
-    int32_t ld;       // row pitch of S and of the per-block vectors, in elements (M rounded up to 4)
+    int32_t ld;       // row pitch of S and of the per-block vectors, in elements (a multiple of 4; pad_row(M) inside rcd_partition)
     int32_t row0;     // first row of the class in class-sorted sample order
     int32_t pad_;
     int64_t sOff;     // element offset of S_l
@@ -134,6 +135,10 @@ constexpr int kGroupChunk = 1024;           // samples per chunk of the stable c
 inline size_t feat_bytes(rcd_feat_dtype t) { return t == RCD_FEAT_I8 ? 1 : 2; }
 inline size_t align_up(size_t x, size_t a = kAlign) { return (x + a - 1) / a * a; }
 inline int32_t pad4(int64_t m) { return (int32_t)((m + 3) / 4 * 4); }
+// Row pitch of S and of the per-block vectors inside rcd_partition / rcd_objective: a multiple of 8
+// elements, so that every row starts on a 32-byte boundary (one memory sector): the 16-byte pieces that
+// the sweeps copy then pair up into whole sectors.
+inline int32_t pad_row(int64_t m) { return (int32_t)((m + 7) / 8 * 8); }
 
 // Lays the workspace out at `base` (may be null to measure).  Returns total bytes.
 size_t layout_workspace(void *base, rcd_feat_dtype dtype, const Sizes &sz, Workspace *ws);

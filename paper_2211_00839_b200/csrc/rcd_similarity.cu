@@ -137,7 +137,7 @@ static rcd_status launch_similarity_generic(rcd_ctx *ctx, const void *Xs, rcd_fe
                                             const SimClasses &cls, void *S, cudaStream_t st)
 {
     const int32_t L = cls.L;
-    const int maxLd = pad4(cls.maxM), maxM = (int)cls.maxM;
+    const int maxLd = pad_row(cls.maxM), maxM = (int)cls.maxM;     // covers either row pitch (pad4 <= pad_row)
     const DescSource src = cls.src;
     if (L == 0 || maxM == 0) return RCD_OK;
     dim3 grid((maxLd + kTile - 1) / kTile, (maxM + kTile - 1) / kTile, L > 65535 ? 65535 : L);
