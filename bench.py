@@ -181,7 +181,7 @@ def run_ours(args):
     Xd, yd = Xh.to(dev), yh.to(dev)
     kind = rcd.RCD_SIM_GAUSSIAN if args.similarity == "gaussian" else rcd.RCD_SIM_DOT
     ctx = rcd.Context(local, sweep_batch_max=args.sweep_batch, profile=1, greedy_path=args.greedy_path, similarity_kind=kind,
-                      async_group=args.async_group,
+                      async_group=args.async_group, async_help_min=args.async_help_min,
                       objective=rcd.RCD_OBJ_GRAPH_CUT if args.objective == "cut" else rcd.RCD_OBJ_FACILITY)
 
     def barrier():
@@ -252,7 +252,7 @@ def run_ours(args):
     # plus the coverage vectors of the blocks refreshed (4*ld*(n_R + n) bytes), summed on the device.
     # Duration = CUDA events around the greedy loop on the launching stream (last timed step).
     peaks = load_peaks()
-    default_setup = args.sweep_batch in (0, 8) and args.async_group == 0 and args.similarity == "dot"
+    default_setup = args.sweep_batch in (0, 8) and args.async_group == 0 and args.async_help_min == 0 and args.similarity == "dot"
     loop_s = prof["greedy_ms"] * 1e-3
     achieved = prof["sweep_bytes"] / loop_s / 1e9 if loop_s > 0 else 0.0
     if args.objective != "facility":
@@ -310,7 +310,8 @@ def run_ours(args):
                          "sweep_batch_max": args.sweep_batch or 8, "similarity": args.similarity, "objective": args.objective, "sharding": "one dataset per rank, no collective"},
               "gain_evals_per_s": world * wl.L * M * (M + 1) / 2 * args.steps / (ms * 1e-3),
               "phases_ms": dict({k: prof[k] for k in ("group_ms", "similarity_ms", "greedy_ms", "total_ms")},
-                                sweep_phases_ms=prof["persistent_sweep_ns"] * 1e-6, pick_phases_ms=prof["persistent_pick_ns"] * 1e-6),
+                                sweep_phases_ms=prof["persistent_sweep_ns"] * 1e-6, pick_phases_ms=prof["persistent_pick_ns"] * 1e-6,
+                                async_lull_ms=prof["async_lull_ns"] * 1e-6, async_visits=int(prof["async_visits"]), async_attempts=int(prof["async_attempts"])),
               "similarity": similarity,
               "e2e": {"value": e2e_value, "unit": "samples/s", "h2d_bytes_per_step": int(h2d),
                       "d2h_bytes_per_step": int(d2h), "wall_ms_per_step": e2e_wall_ms / args.steps},
@@ -344,6 +345,7 @@ def main():
     ap.add_argument("--objective", default="facility", choices=["facility", "cut"], help="submodular function of Section 4 item 2")
     ap.add_argument("--greedy-path", type=int, default=0,
                     help="0 = chosen by the library, 1 = two launches per round, 2 = one launch with rounds, 3 = one launch, asynchronous classes")
+    ap.add_argument("--async-help-min", type=int, default=0, help="greedy path 3: row groups left before other classes' CTAs help (0 = default)")
     ap.add_argument("--async-group", type=int, default=0, help="greedy path 3: sweeps served together (0 = library default)")
     ap.add_argument("--ref-picks", type=int, default=150, help="picks per class in the CPU-oracle sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -90,7 +90,9 @@ typedef struct {
     int32_t async_group;       /* greedy_path 3: how many sweeps (ordered by sweep number, then class) the sweep CTAs serve
                                   together, each CTA going to the class nearest its home position; 1 = strictly in
                                   order; 0 = default: all classes together */
-    int32_t reserved[8];       /* must be 0 */
+    int32_t async_help_min;    /* greedy_path 3: row groups a sweep must have left before a sweep CTA whose home is another
+                                  class joins it; 0 = default (48) */
+    int32_t reserved[7];       /* must be 0 */
 } rcd_config;
 
 /* Timings and counters of the last rcd_partition / rcd_partition_host on a context (profile >= 1). */
@@ -113,6 +115,9 @@ typedef struct {
     int64_t threshold_hits;         /* threshold passes: elements of S above the threshold ... */
     int64_t threshold_elems;        /* ... out of this many elements compared */
     int64_t threshold_max_blocks;   /* most blocks one threshold pass refreshed */
+    int64_t async_lull_ns;          /* asynchronous form: time the first sweep CTA found no sweep with tickets left */
+    int64_t async_visits;           /* asynchronous form: times the first sweep CTA went to a class and swept there */
+    int64_t async_attempts;         /* ... and times it tried (an attempt fails when the tickets run out under way) */
 } rcd_profile;
 
 typedef struct rcd_ctx rcd_ctx;

@@ -47,7 +47,7 @@ class RcdError(RuntimeError):
 class RcdConfig(C.Structure):
     _fields_ = [("sweep_batch_max", C.c_int32), ("similarity_path", C.c_int32), ("profile", C.c_int32),
                 ("greedy_path", C.c_int32), ("similarity_kind", C.c_int32), ("objective", C.c_int32), ("sweep_mode", C.c_int32), ("async_group", C.c_int32),
-                ("reserved", C.c_int32 * 8)]
+                ("async_help_min", C.c_int32), ("reserved", C.c_int32 * 7)]
 
 
 class RcdProfile(C.Structure):
@@ -56,7 +56,8 @@ class RcdProfile(C.Structure):
                 ("sweep_bytes", C.c_int64), ("sweep_elem_ops", C.c_int64), ("kernel_launches", C.c_int64),
                 ("steps", C.c_int64), ("similarity_tc_launches", C.c_int64), ("persistent_sweep_ns", C.c_int64),
                 ("persistent_pick_ns", C.c_int64), ("threshold_hits", C.c_int64),
-                ("threshold_elems", C.c_int64), ("threshold_max_blocks", C.c_int64)]
+                ("threshold_elems", C.c_int64), ("threshold_max_blocks", C.c_int64),
+                ("async_lull_ns", C.c_int64), ("async_visits", C.c_int64), ("async_attempts", C.c_int64)]
 
 
 def _load() -> C.CDLL:
@@ -145,7 +146,7 @@ class Context:
 
     def __init__(self, device: int = 0, sweep_batch_max: int = 0, similarity_path: int = 0, profile: int = 0,
                  greedy_path: int = 0, similarity_kind: int = 0, objective: int = 0, sweep_mode: int = 0,
-                 async_group: int = 0):
+                 async_group: int = 0, async_help_min: int = 0):
         torch = _torch()
         if not torch.cuda.is_available():
             raise RcdError(4, "no CUDA device: this library has no CPU path")
@@ -160,6 +161,7 @@ class Context:
         cfg.objective = objective
         cfg.sweep_mode = sweep_mode
         cfg.async_group = async_group
+        cfg.async_help_min = async_help_min
         self.similarity_kind = similarity_kind
         self._h = C.c_void_p()
         st = lib.rcd_create(C.byref(self._h), self.device, C.byref(cfg))

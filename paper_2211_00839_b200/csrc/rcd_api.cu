@@ -89,9 +89,10 @@ size_t layout_workspace(void *base, rcd_feat_dtype dtype, const Sizes &sz, Works
     w.sweepList = c.take<int32_t>(3 * L);
     w.sync = c.take<ClassSync>(L);
     w.tickets = c.take<int32_t>(N + L);
+    w.sweepF = c.take<long long>(L * 8);
     w.stepBytes = c.take<unsigned long long>((size_t)sz.maxM + 1);
     w.stepOps = c.take<unsigned long long>((size_t)sz.maxM + 1);
-    w.phaseNs = c.take<unsigned long long>(6);      // two phase clocks, the grid-barrier counter, threshold-pass hits / elements
+    w.phaseNs = c.take<unsigned long long>(8);      // two phase clocks, the grid-barrier counter, threshold-pass hits / elements
     w.bytes = align_up(c.off);
     if (ws) *ws = w;
     return w.bytes;
@@ -292,7 +293,8 @@ rcd_status rcd_create(rcd_ctx **out, int cuda_device, const rcd_config *cfg)
         if (cfg->objective != RCD_OBJ_FACILITY && cfg->objective != RCD_OBJ_GRAPH_CUT) return RCD_ERR_INVALID_ARG;
         if (cfg->sweep_mode != 0 && cfg->sweep_mode != 1) return RCD_ERR_INVALID_ARG;
         if (cfg->async_group < 0 || cfg->async_group > 4096) return RCD_ERR_INVALID_ARG;
-        for (int i = 0; i < 8; ++i) if (cfg->reserved[i] != 0) return RCD_ERR_INVALID_ARG;
+        if (cfg->async_help_min < 0) return RCD_ERR_INVALID_ARG;
+        for (int i = 0; i < 7; ++i) if (cfg->reserved[i] != 0) return RCD_ERR_INVALID_ARG;
     }
     int count = 0;
     if (cudaGetDeviceCount(&count) != cudaSuccess || cuda_device < 0 || cuda_device >= count) {
@@ -375,13 +377,16 @@ rcd_status rcd_get_profile(rcd_ctx *ctx, rcd_profile *out)
     RCD_CUDA(ctx, cudaEventElapsedTime(&ms, ctx->evPhase[1], ctx->evPhase[2])); out->similarity_ms = ms;
     RCD_CUDA(ctx, cudaEventElapsedTime(&ms, ctx->evPhase[2], ctx->evPhase[3])); out->greedy_ms = ms;
     if (ctx->phaseNsDev) {
-        unsigned long long ns[6] = {0, 0, 0, 0, 0, 0};
+        unsigned long long ns[8] = {0, 0, 0, 0, 0, 0, 0, 0};
         RCD_CUDA(ctx, cudaMemcpy(ns, ctx->phaseNsDev, sizeof ns, cudaMemcpyDeviceToHost));
         out->persistent_sweep_ns = (int64_t)ns[0];
         out->persistent_pick_ns = (int64_t)ns[1];
         out->threshold_hits = (int64_t)ns[3];
         out->threshold_elems = (int64_t)ns[4];
         out->threshold_max_blocks = (int64_t)ns[5];
+        out->async_lull_ns = (int64_t)ns[6];
+        out->async_visits = (int64_t)(ns[7] & 0xffffffffull);
+        out->async_attempts = (int64_t)(ns[7] >> 32);
     }
     if (ctx->stepBytesDev && ctx->steps > 0) {
         std::vector<unsigned long long> bytes((size_t)ctx->steps + 1), ops((size_t)ctx->steps + 1);

@@ -70,7 +70,8 @@ struct GreedyParams {
     unsigned long long *stepBytes;
     unsigned long long *stepOps;
     unsigned long long *phaseNs;    // [0..1] time block 0 spent in sweep / pick phases (persistent kernel), [2] grid-barrier
-                                    // counter, [3..5] threshold passes: elements above the threshold / elements compared / most blocks in one pass
+                                    // counter, [3..5] threshold passes: elements above the threshold / elements compared / most blocks in one pass,
+                                    // [6..7] asynchronous kernel: ns the first sweep CTA found nothing to sweep, its visits
     unsigned *barrier;              // arrival counter of the persistent kernel's grid barrier
     int32_t *status;
     const int32_t *perm;
@@ -86,8 +87,10 @@ struct GreedyParams {
     // asynchronous kernel (greedy_async_kernel); asyncMode = 0 everywhere else
     ClassSync *sync;            // [L] hand-off words
     int32_t *tickets;           // [N + L] ticket counter of sweep k of class l at tickets[row0_l + l + k]
+    long long *sweepF;          // [L][kMaxSweepBatch] int8 features: f of the blocks a dense pass refreshes
     int32_t asyncMode;
     int32_t nPick;              // CTAs [0, nPick) make picks, the others sweep
+    int32_t helpMin;            // row groups a sweep must have left for a sweep CTA that is not at home there
     int32_t asyncGroup;         // sweeps published one after another that are served together (by CTA home position)
 };
 
@@ -266,7 +269,14 @@ __device__ void plan_decide(const GreedyParams<SV> &prm, int l, const ClassDesc 
         prm.sweepCS[l] = CS;
         prm.rowCtr[l] = 0;
         if (prm.asyncMode) {
-            prm.sync[l].nGroups = (int32_t)nGroups;        // published with the epoch by the caller
+            ClassSync &sy = prm.sync[l];                   // published with the epoch by the caller
+            sy.nGroups = (int32_t)nGroups;
+            sy.nR = nR;
+            sy.cfg = P | (CS << 8) | ((sparse ? 1 : 0) << 16);
+            if constexpr (Arith<SV>::kInt) {
+                if (!sparse)
+                    for (int k = 0; k < P; ++k) prm.sweepF[(int64_t)l * kMaxSweepBatch + k] = (long long)sh.f[parts[k]];
+            }
         } else {
             int par = nextStep % 3;
             int slot = atomicAdd(&prm.nSweep[par], 1);
@@ -308,6 +318,7 @@ __global__ void __launch_bounds__(kSelectThreads, 4) init_kernel(GreedyParams<SV
             prm.sync[l].done = 0;
             prm.sync[l].seq = l;
             prm.sync[l].nGroups = 0;                       // (plan_decide below sets it)
+
         }
     }
     __syncthreads();
@@ -875,11 +886,16 @@ __device__ __forceinline__ int4 min_int4(int4 a, int4 b)
 
 // Finishes a coverage update whose operands were copied to shared memory earlier (row v* in
 // scratch[0, ld4), the old coverage in scratch[ld4, 2 ld4)): dst[i] = max of the two.
+// thrAcc (may be null): running element-wise minimum of the coverage vectors updated in this chain.
 template <typename SV>
-__device__ __forceinline__ void fold_pending(int4 *dst, const int4 *scratch, int ld4)
+__device__ __forceinline__ void fold_pending(int4 *dst, const int4 *scratch, int ld4, int4 *thrAcc)
 {
     asm volatile("cp.async.wait_group 0;" ::: "memory");
-    for (int i = threadIdx.x; i < ld4; i += kSelectThreads) dst[i] = max_int4<SV>(scratch[ld4 + i], scratch[i]);
+    for (int i = threadIdx.x; i < ld4; i += kSelectThreads) {
+        const int4 m = max_int4<SV>(scratch[ld4 + i], scratch[i]);
+        dst[i] = m;
+        if (thrAcc) thrAcc[i] = min_int4<SV>(thrAcc[i], m);
+    }
 }
 
 // The picks of class l in round `round`, by one CTA of kSelectThreads threads: pick after pick
@@ -889,7 +905,8 @@ __device__ __forceinline__ void fold_pending(int4 *dst, const int4 *scratch, int
 // is finished.  Inside the chain nothing waits on the coverage update: a pick only needs stored
 // gains, so row v* is folded into the coverage vector while the next block is being chosen.
 template <typename SV>
-__device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, int round, int4 *scratch, int scratchBytes)
+__device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, int round, int4 *scratch, int scratchBytes,
+                                           bool planInShared = false)
 {
     using GV = typename Arith<SV>::GV;
     using FV = typename Arith<SV>::FV;
@@ -906,14 +923,31 @@ __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, i
     const int ld4 = c.ld >> 2;
     int32_t *cand = prm.cand + c.row0;
     int32_t *pos = prm.pos + c.row0;
-    plan_load(prm, l, shPlan);
-    __syncthreads();
+    __shared__ int32_t shChain[kSparseMax];         // blocks that received a sample in this chain
+    __shared__ int shChainOk;
+    if (!planInShared) {                            // (a CTA that serves one class keeps the table from its last chain)
+        plan_load(prm, l, shPlan);
+        __syncthreads();
+    }
     // Folding row v* into the coverage vector is off the critical path (a pick reads stored gains,
     // never the coverage).  When the caller lends enough shared memory, row v* and the coverage
     // vector are fetched with asynchronous copies once v* is known, and the max/store happens one
     // pick later, after the next argmax; each thread consumes exactly the pieces it copied.
     const bool defer = scratch != nullptr && (int64_t)2 * c.ld * (int64_t)sizeof(SV) <= scratchBytes;
     int4 *pendDst = nullptr;
+    // The threshold vector of a coming threshold pass is the element-wise minimum of the listed blocks'
+    // coverage.  Those blocks are, as a rule, exactly the ones that receive a sample in this chain (every
+    // other block's stored gains stay valid), and each receives one: so the minimum is taken as the
+    // updated vectors pass through fold_pending, in the third ld-sized piece of the scratch area.  A block
+    // of the chain that is not listed (it became full) only lowers the threshold, which keeps the pass exact.
+    int4 *thrAcc = (defer && (int64_t)3 * c.ld * (int64_t)sizeof(SV) <= scratchBytes) ? scratch + 2 * ld4 : nullptr;
+    if (thrAcc) {
+        int4 top;
+        if constexpr (Arith<SV>::kInt) top = make_int4(INT_MAX, INT_MAX, INT_MAX, INT_MAX);
+        else top = make_int4(0x7f800000, 0x7f800000, 0x7f800000, 0x7f800000);      // +infinity
+        for (int i = threadIdx.x; i < ld4; i += kSelectThreads) thrAcc[i] = top;
+    }
+    int chainLen = 0;
 
     for (;;) {
         const GV *G = prm.gains + c.vOff + (int64_t)j * c.ld;
@@ -942,7 +976,7 @@ __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, i
             }
         }
         if (pendDst) {                                  // finish the previous pick's coverage update
-            fold_pending<SV>(pendDst, scratch, ld4);
+            fold_pending<SV>(pendDst, scratch, ld4, thrAcc);
             pendDst = nullptr;
         }
         for (int off = 16; off > 0; off >>= 1) {
@@ -974,6 +1008,8 @@ __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, i
             __syncwarp();
         }
         __syncthreads();
+        if (threadIdx.x == 0 && chainLen < kSparseMax) shChain[chainLen] = j;
+        ++chainLen;
         const int vstar = shPick;
         if (vstar == INT_MAX || vstar < 0 || vstar >= c.M) {
             if (threadIdx.x == 0) atomicOr(prm.status, kDevBadState);
@@ -1017,24 +1053,38 @@ __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, i
         j = shPlan.nextJ;
         if (nR == 0 || j < 0 || shPlan.needSweep) break;
     }
-    if (pendDst) fold_pending<SV>(pendDst, scratch, ld4);
+    if (pendDst) fold_pending<SV>(pendDst, scratch, ld4, thrAcc);
     if (shPlan.needSweep && shPlan.sweepSparse) {
         // threshold of the coming pass: element-wise minimum of the listed blocks' coverage vectors
-        // (each thread reads back exactly the pieces of the coverage vectors it wrote itself)
         const int P = shPlan.sweepBlocks;
         const int32_t *parts = prm.sweepParts + (int64_t)l * kSparseMax;
         const int4 *cov = reinterpret_cast<const int4 *>(prm.cover + c.vOff);
         int4 *thr = reinterpret_cast<int4 *>(prm.thr + c.vOff / prm.W);
-        for (int i = threadIdx.x; i < ld4; i += kSelectThreads) {
-            int4 m = cov[(int64_t)parts[0] * ld4 + i];
-            for (int k0 = 1; k0 < P; k0 += 8) {                     // eight independent loads at a time
-                int4 t[8];
+        // is every listed block one of this chain's?  (then the running minimum is the threshold)
+        if (threadIdx.x == 0) shChainOk = (thrAcc != nullptr && chainLen <= kSparseMax) ? 1 : 0;
+        __syncthreads();
+        if (shChainOk && threadIdx.x < P) {
+            const int p = parts[threadIdx.x];
+            bool found = false;
+            for (int k = 0; k < chainLen; ++k) found = found || shChain[k] == p;
+            if (!found) shChainOk = 0;
+        }
+        __syncthreads();
+        if (shChainOk) {
+            for (int i = threadIdx.x; i < ld4; i += kSelectThreads) thr[i] = thrAcc[i];
+        } else {
+            // (each thread reads back exactly the pieces of the coverage vectors it wrote itself)
+            for (int i = threadIdx.x; i < ld4; i += kSelectThreads) {
+                int4 m = cov[(int64_t)parts[0] * ld4 + i];
+                for (int k0 = 1; k0 < P; k0 += 8) {                     // eight independent loads at a time
+                    int4 t[8];
 #pragma unroll
-                for (int u = 0; u < 8; ++u) t[u] = cov[(int64_t)parts[k0 + u < P ? k0 + u : 0] * ld4 + i];
+                    for (int u = 0; u < 8; ++u) t[u] = cov[(int64_t)parts[k0 + u < P ? k0 + u : 0] * ld4 + i];
 #pragma unroll
-                for (int u = 0; u < 8; ++u) m = min_int4<SV>(m, t[u]);
+                    for (int u = 0; u < 8; ++u) m = min_int4<SV>(m, t[u]);
+                }
+                thr[i] = m;
             }
-            thr[i] = m;
         }
     }
 }
@@ -1153,6 +1203,7 @@ __device__ __forceinline__ int4 ld_volatile16(const void *p)
 }
 __device__ __forceinline__ int32_t ld_volatile32(const int32_t *p) { return *(const volatile int32_t *)p; }
 
+
 template <typename SV>
 __device__ __forceinline__ void async_pick_cta(const GreedyParams<SV> &prm, int4 *scratch)
 {
@@ -1162,6 +1213,7 @@ __device__ __forceinline__ void async_pick_cta(const GreedyParams<SV> &prm, int4
     for (int l = me; l < prm.L; l += prm.nPick) mine += prm.desc[l].M > 0 ? 1 : 0;
     unsigned idle = 0;
     unsigned long long busy = 0;
+    bool planKept = false;
     while (mine > 0) {
         bool progressed = false;
         for (int l = me; l < prm.L; l += prm.nPick) {
@@ -1181,7 +1233,8 @@ __device__ __forceinline__ void async_pick_cta(const GreedyParams<SV> &prm, int4
             progressed = true;
             unsigned long long t0 = 0;
             if (me == 0 && threadIdx.x == 0) t0 = global_ns();
-            pick_chain(prm, l, e >> 1, scratch, prm.smemBytes);
+            pick_chain(prm, l, e >> 1, scratch, prm.smemBytes, planKept);
+            planKept = prm.nPick >= prm.L;                          // my only class: the block table stays in shared memory
             __syncthreads();                                            // all writes of the chain are issued
             if (threadIdx.x == 0) {
                 const bool finished = prm.nR[l] == 0 || prm.jstar[l] < 0 || ld_volatile32(prm.status) != 0;
@@ -1230,8 +1283,10 @@ __device__ __forceinline__ void async_sweep_cta(const GreedyParams<SV> &prm, int
     __shared__ int shInfo[12];                                      // ok, first ticket, nR, P, CS, mode, nGroups, stop, sweep number, epoch
     const bool clocked = blockIdx.x == prm.nPick;                   // the first sweep CTA keeps the busy clock
     const int home = (int)(((int64_t)(blockIdx.x - prm.nPick) * prm.L) / (gridDim.x - prm.nPick));
+    const int helpMin = ((int)(gridDim.x - prm.nPick) >= prm.L) ? prm.helpMin : 1;
     unsigned idle = 0;
-    unsigned long long busy = 0;
+    __shared__ unsigned long long shClk[5];                         // busy ns, lull ns, visits, start of the lull, start of the visit (first sweep CTA, thread 0)
+    if (threadIdx.x == 0) { shClk[0] = 0; shClk[1] = 0; shClk[2] = 0; shClk[3] = 0; shClk[4] = 0; }
     for (;;) {
         // The sweep to serve: sweeps are served by order number (sweep number first), asyncGroup of them
         // together; inside such a batch a CTA goes to the class nearest to its home position (CTAs spread
@@ -1240,18 +1295,20 @@ __device__ __forceinline__ void async_sweep_cta(const GreedyParams<SV> &prm, int
         if (threadIdx.x == 0) shBest = ~0ull;
         __syncthreads();
         unsigned long long myKey = ~0ull;
-        int myEpoch = 0;
+        int4 myA = make_int4(0, 0, 0, 0), myB = make_int4(0, 0, 0, 0);
         for (int l = threadIdx.x; l < prm.L; l += blockDim.x) {
-            const int4 sy = ld_volatile16(&prm.sync[l]);            // epoch, nGroups, done, seq
-            if (!(sy.x & 1)) {
-                const int32_t drawn = ld_volatile32(prm.tickets + prm.desc[l].row0 + l + (sy.x >> 1));
-                if (drawn < sy.y) {
-                    int dist = l - home;
-                    if (dist < 0) dist += prm.L;
-                    const unsigned long long key = ((unsigned long long)(unsigned)(sy.w / prm.asyncGroup) << 40) |
-                                                   ((unsigned long long)(unsigned)dist << 20) | (unsigned)l;
-                    if (key < myKey) { myKey = key; myEpoch = sy.x; }
-                }
+            const int4 a = ld_volatile16(&prm.sync[l]);             // epoch, nGroups, done, seq
+            const int4 b = ld_volatile16(&prm.sync[l].pad_[0]);     // -, -, nR, cfg
+            const int drawn = (a.x & 1) ? 0 : ld_volatile32(prm.tickets + prm.desc[l].row0 + l + (a.x >> 1));
+            if (!(a.x & 1) && drawn < a.y) {
+                int dist = l - home;
+                if (dist < 0) dist += prm.L;
+                // away from home only for a worthwhile number of row groups: the last few of a sweep are mostly
+                // gone by the time a helper has drawn its tickets (every class has CTAs at home when helpMin > 1)
+                if (dist != 0 && a.y - drawn < helpMin) continue;
+                const unsigned long long key = ((unsigned long long)(unsigned)(a.w / prm.asyncGroup) << 40) |
+                                               ((unsigned long long)(unsigned)dist << 20) | (unsigned)l;
+                if (key < myKey) { myKey = key; myA = a; myB = b; }
             }
         }
         if (myKey != ~0ull) atomicMin(&shBest, myKey);
@@ -1262,6 +1319,7 @@ __device__ __forceinline__ void async_sweep_cta(const GreedyParams<SV> &prm, int
                 int stop = (ld_volatile32(&prm.nSweep[3]) == 0 || ld_volatile32(prm.status) != 0) ? 1 : 0;
                 if (!stop && ++idle >= kIdleLimit) { atomicOr(prm.status, kDevTimeout); stop = 1; }
                 shInfo[7] = stop;
+                if (clocked && shClk[3] == 0) shClk[3] = global_ns();
             }
             __syncthreads();
             const int stop = shInfo[7];
@@ -1269,6 +1327,10 @@ __device__ __forceinline__ void async_sweep_cta(const GreedyParams<SV> &prm, int
             if (stop) break;
             __nanosleep(200);
             continue;
+        }
+        if (clocked && threadIdx.x == 0 && shClk[3] != 0) {
+            shClk[1] += global_ns() - shClk[3];
+            shClk[3] = 0;
         }
         const int l = (int)(unsigned)(best & 0xfffffull);
         const ClassDesc c = prm.desc[l];
@@ -1278,25 +1340,22 @@ __device__ __forceinline__ void async_sweep_cta(const GreedyParams<SV> &prm, int
         // comes after the parameters.  Every load here is volatile (served by L2), and the bulk data of a
         // sweep (coverage, threshold, candidate list) is read with ld.cg, so no stale L1 line can be seen;
         // the barriers keep the groups of loads in order.
-        if (myKey == best) shInfo[9] = myEpoch;
+        if (myKey == best) {
+            shInfo[9] = myA.x;                                      // epoch
+            shInfo[6] = myA.y;                                      // row groups
+            shInfo[2] = myB.z;                                      // unassigned samples
+            shInfo[3] = myB.w & 0xff;                               // blocks
+            shInfo[4] = (myB.w >> 8) & 0xff;                        // warps per row group
+            shInfo[5] = (myB.w >> 16) & 1;                          // threshold pass?
+        }
         if (threadIdx.x < kSparseMax) {
             int bp = ld_volatile32(parts + threadIdx.x);
             if (bp < 0 || bp >= prm.W) bp = 0;                      // (beyond the list, or a read that raced with an update)
             shParts[threadIdx.x] = bp;
         }
-        if (threadIdx.x == 64) {
-            shInfo[2] = ld_volatile32(&prm.nR[l]);
-            shInfo[3] = ld_volatile32(&prm.sweepN[l]);
-            shInfo[4] = ld_volatile32(&prm.sweepCS[l]);
-            shInfo[5] = ld_volatile32(&prm.sweepMode[l]);
-        }
-        if (threadIdx.x == 96) shInfo[6] = ld_volatile32(&prm.sync[l].nGroups);
         if constexpr (Arith<SV>::kInt) {
-            if (threadIdx.x >= 128 && threadIdx.x < 128 + kMaxSweepBatch) {
-                int p = ld_volatile32(parts + (threadIdx.x - 128));
-                if (p < 0 || p >= prm.W) p = 0;
-                shF[threadIdx.x - 128] = *(const volatile long long *)&prm.fval[(int64_t)l * prm.W + p];
-            }
+            if (threadIdx.x >= 128 && threadIdx.x < 128 + kMaxSweepBatch)
+                shF[threadIdx.x - 128] = *(const volatile long long *)&prm.sweepF[(int64_t)l * kMaxSweepBatch + (threadIdx.x - 128)];
         }
         __syncthreads();
         // Second read of the epoch, and with it -- before its answer is known -- one ticket per team is
@@ -1312,6 +1371,7 @@ __device__ __forceinline__ void async_sweep_cta(const GreedyParams<SV> &prm, int
             const int first = atomicAdd(prm.tickets + c.row0 + l + (e1 >> 1), teams);
             const int e2 = ld_volatile32(&prm.sync[l].epoch);
             shInfo[0] = (e1 == e2 && !(e1 & 1) && first < shInfo[6]) ? 1 : 0;
+            if (clocked) shClk[2] += 1ull << 32;                   // attempts (high half), visits (low half)
             shInfo[1] = first;
             shInfo[8] = e1 >> 1;
         }
@@ -1332,8 +1392,10 @@ __device__ __forceinline__ void async_sweep_cta(const GreedyParams<SV> &prm, int
         __syncthreads();
         if (!shInfo[0]) continue;                                   // another look at the sweeps
         idle = 0;
-        unsigned long long t0 = 0;
-        if (clocked && threadIdx.x == 0) t0 = global_ns();
+        if (clocked && threadIdx.x == 0) {
+            shClk[4] = global_ns();
+            shClk[2] += 1;
+        }
         const int nR = shInfo[2], first = shInfo[1];
         int32_t *ticket = prm.tickets + c.row0 + l + shInfo[8];      // the counter of this sweep alone
         int32_t *done = &prm.sync[l].done;
@@ -1351,9 +1413,11 @@ __device__ __forceinline__ void async_sweep_cta(const GreedyParams<SV> &prm, int
             }
         }
         __syncthreads();
-        if (clocked && threadIdx.x == 0) busy += global_ns() - t0;
+        if (threadIdx.x == 0) {
+            if (clocked) shClk[0] += global_ns() - shClk[4];
+        }
     }
-    if (clocked && threadIdx.x == 0) prm.phaseNs[0] = busy;
+    if (clocked && threadIdx.x == 0) { prm.phaseNs[0] = shClk[0]; prm.phaseNs[6] = shClk[1]; prm.phaseNs[7] = shClk[2]; }
 }
 
 template <typename SV>
@@ -1432,9 +1496,11 @@ static rcd_status run_greedy(rcd_ctx *ctx, const Sizes &sz, const Workspace &ws,
     prm.sparseMinMembers = ctx->cfg.sweep_mode == 1 ? -1 : 8;
     prm.sync = ws.sync;
     prm.tickets = ws.tickets;
+    prm.sweepF = ws.sweepF;
     prm.asyncMode = 0;
     prm.nPick = 0;
     prm.asyncGroup = 1;
+    prm.helpMin = 1;
     int maxLd = 0;
     for (const auto &c : descHost) if (c.ld > maxLd) maxLd = c.ld;
     const int64_t smemCap = (int64_t)ctx->maxSmemOptin - 20 * 1024;  // static shared of the kernels + margin
@@ -1480,12 +1546,13 @@ static rcd_status run_greedy(rcd_ctx *ctx, const Sizes &sz, const Workspace &ws,
         prm.asyncMode = 1;
         prm.nPick = std::min<int>(sz.L, std::max(1, ctx->smCount / 4));
         prm.sweepWarps = (ctx->smCount - prm.nPick) * (kSweepThreads / 32);
+        prm.helpMin = ctx->cfg.async_help_min > 0 ? ctx->cfg.async_help_min : 48;
         prm.asyncGroup = ctx->cfg.async_group > 0 ? ctx->cfg.async_group : std::max<int>(sz.L, 1);
     }
 
     if (path == 3) RCD_CUDA(ctx, cudaMemsetAsync(ws.tickets, 0, (size_t)(sz.N + sz.L) * sizeof(int32_t), st));
     RCD_CUDA(ctx, cudaMemsetAsync(ws.nSweep, 0, 4 * sizeof(int32_t), st));
-    RCD_CUDA(ctx, cudaMemsetAsync(ws.phaseNs, 0, 6 * sizeof(unsigned long long), st));
+    RCD_CUDA(ctx, cudaMemsetAsync(ws.phaseNs, 0, 8 * sizeof(unsigned long long), st));
     ctx->phaseNsDev = ws.phaseNs;
     RCD_CUDA(ctx, cudaMemsetAsync(ws.stepBytes, 0, (size_t)(sz.maxM + 1) * sizeof(unsigned long long), st));
     RCD_CUDA(ctx, cudaMemsetAsync(ws.stepOps, 0, (size_t)(sz.maxM + 1) * sizeof(unsigned long long), st));

@@ -31,11 +31,14 @@ enum : int {
 // and its parameters are stable, odd = the class belongs to its pick CTA (or is finished).
 struct ClassSync {
     int32_t epoch;
-    int32_t nGroups;  // row groups (tickets) of the published sweep
-    int32_t done;     // row groups of the published sweep whose gains are written
-    int32_t seq;      // order number of the published sweep (sweep number x L + class)
-    int32_t pad_[4];  // one 32-byte sector per class: the counters of two classes never share one
+    int32_t nGroups;   // row groups (tickets) of the published sweep
+    int32_t done;      // row groups of the published sweep whose gains are written
+    int32_t seq;       // order number of the published sweep (sweep number x L + class)
+    int32_t pad_[2];   // (the word fills one 32-byte sector: the counters of two classes never share one)
+    int32_t nR;        // of the published sweep: samples of the class still unassigned
+    int32_t cfg;       //   blocks it refreshes | warps per row group << 8 | (1 = threshold pass) << 16
 };
+static_assert(sizeof(ClassSync) == 32, "one 32-byte sector per class");
 
 // One class, as the kernels see it.  Built on the host once the class sizes are known.
 struct ClassDesc {
@@ -110,6 +113,7 @@ struct Workspace {
     int32_t *rowCtr;        // [L] ticket counter over row groups of the running sweep
     ClassSync *sync;        // [L] asynchronous kernel: hand-off words
     int32_t *tickets;       // [N + L] asynchronous kernel: one ticket counter per (class, sweep number), never reused
+    long long *sweepF;      // [L][8] asynchronous kernel, int8 features: f of the first blocks in the sweep's list
     int32_t *sweepList;     // [3][L] classes that sweep in a step (three lists in rotation)
     int32_t *nSweep;        // [3] (+1 pad)
     unsigned long long *stepBytes;   // [steps+1] bytes the sweep of step t has to read
