@@ -105,6 +105,7 @@ template <typename FV>
 struct PlanShared {
     FV f[kMaxBlocks];              // tracked f of every block
     int32_t room[kMaxBlocks];      // quota - count
+    int32_t quota[kMaxBlocks];
     uint8_t open[kMaxBlocks];      // bit 0: block is not full, bit 1: its stored gains are out of date
     int32_t nextJ;                 // plan_decide's answer: block of the next pick (-1: none)
     int32_t needSweep;             //                       1 = that pick must wait for a sweep
@@ -118,9 +119,11 @@ __device__ __forceinline__ void plan_load(const GreedyParams<SV> &prm, int l, Pl
     const int W = prm.W;
     for (int p = threadIdx.x; p < W; p += blockDim.x) {
         const int64_t at = (int64_t)l * W + p;
-        const int room = prm.quota[at] - prm.cnt[at];
+        const int quota = prm.quota[at];
+        const int room = quota - prm.cnt[at];
         sh.f[p] = prm.fval[at];
         sh.room[p] = room;
+        sh.quota[p] = quota;
         sh.open[p] = (uint8_t)((room > 0 ? 1 : 0) | (prm.valid[at] ? 0 : 2));
     }
 }
@@ -164,7 +167,7 @@ __device__ void plan_decide(const GreedyParams<SV> &prm, int l, const ClassDesc 
             if (bestP == INT_MAX || fp < bestF) { bestF = fp; bestP = p; }
             if (o & 2) {
                 ++nStale;
-                fewest = min(fewest, prm.quota[(int64_t)l * W + p] - sh.room[p]);
+                fewest = min(fewest, sh.quota[p] - sh.room[p]);
             }
         }
     }
@@ -203,7 +206,7 @@ __device__ void plan_decide(const GreedyParams<SV> &prm, int l, const ClassDesc 
         from = prm.sparseFrom[l];
         const unsigned long long elems = prm.sparseElems[l];
         if (elems) {
-            const unsigned long long hits = prm.hitCount[l];
+            const unsigned long long hits = *(const volatile unsigned long long *)&prm.hitCount[l];   // (added to by the sweeping CTAs)
             atomicAdd(&prm.phaseNs[3], hits);
             atomicAdd(&prm.phaseNs[4], elems);
             if (hits * 32ull > elems) { from = 2 * fewest; prm.sparseFrom[l] = from; }
@@ -904,9 +907,14 @@ __device__ __forceinline__ void fold_pending(int4 *dst, const int4 *scratch, int
 // block's stored gains are out of date -- then a sweep is scheduled for round + 1 -- or the class
 // is finished.  Inside the chain nothing waits on the coverage update: a pick only needs stored
 // gains, so row v* is folded into the coverage vector while the next block is being chosen.
+// own: 0 = the CTA may serve other classes between two chains of this one (all state is read from and
+// written to global memory); 1 / 2 = the CTA serves this class only, first / later chain: the block table,
+// the candidate list with its inverse, the dataset indices of the class's samples and the chain's loop
+// state (keep[0] = samples left, keep[1] = next block) stay in shared memory between chains, so that a
+// pick waits for one trip to memory only -- the loads of the stored gains, served by L2 (ld.cg).
 template <typename SV>
 __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, int round, int4 *scratch, int scratchBytes,
-                                           bool planInShared = false)
+                                           int own = 0, int *keep = nullptr)
 {
     using GV = typename Arith<SV>::GV;
     using FV = typename Arith<SV>::FV;
@@ -914,19 +922,39 @@ __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, i
     __shared__ GV shG[kSelectThreads / 32];
     __shared__ int shV[kSelectThreads / 32];
     __shared__ int shPick;
-    int nR = prm.nR[l];
-    if (nR == 0) return;
-    int j = prm.jstar[l];
-    if (j < 0) return;
     const ClassDesc c = prm.desc[l];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int ld4 = c.ld >> 2;
+    // resident state: behind the three ld-sized pieces of the scratch area used below
+    const bool res = own != 0 && keep != nullptr && scratch != nullptr && (int64_t)6 * c.ld * (int64_t)sizeof(SV) <= scratchBytes;
+    int32_t *shPos = reinterpret_cast<int32_t *>(scratch + 3 * ld4);
+    int32_t *shCand = shPos + c.ld;
+    int32_t *shPerm = shCand + c.ld;
+    int nR, j;
+    if (res && own == 2) {
+        nR = keep[0];
+        j = keep[1];
+    } else {
+        nR = prm.nR[l];
+        j = prm.jstar[l];
+    }
+    if (nR == 0 || j < 0) {
+        if (keep && threadIdx.x == 0) { keep[0] = nR; keep[1] = j; }
+        return;
+    }
     int32_t *cand = prm.cand + c.row0;
     int32_t *pos = prm.pos + c.row0;
     __shared__ int32_t shChain[kSparseMax];         // blocks that received a sample in this chain
     __shared__ int shChainOk;
-    if (!planInShared) {                            // (a CTA that serves one class keeps the table from its last chain)
+    if (!(res && own == 2)) {
         plan_load(prm, l, shPlan);
+        if (res) {
+            for (int v = threadIdx.x; v < c.M; v += kSelectThreads) {
+                shPos[v] = pos[v];
+                shCand[v] = cand[v];
+                shPerm[v] = prm.perm[c.row0 + v];
+            }
+        }
         __syncthreads();
     }
     // Folding row v* into the coverage vector is off the critical path (a pick reads stored gains,
@@ -967,7 +995,10 @@ __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, i
                 const int v = v0 + i * kSelectThreads;
                 ps[i] = -1;
                 g[i] = 0;
-                if (v < c.M) { g[i] = G[v]; ps[i] = pos[v]; }
+                if (v < c.M) {
+                    if (res) { g[i] = __ldcg(G + v); ps[i] = shPos[v]; }
+                    else { g[i] = G[v]; ps[i] = pos[v]; }
+                }
             }
 #pragma unroll
             for (int i = 0; i < kArgmaxBatch; ++i) {
@@ -975,6 +1006,9 @@ __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, i
                 if (ps[i] >= 0 && (bestV == INT_MAX || g[i] > bestG)) { bestG = g[i]; bestV = v; }
             }
         }
+        // (thread 0 of a CTA that owns its class has just marked the class as taken: that store is ordered
+        // before everything the chain writes; the fence completes together with the loads above)
+        if (res && chainLen == 0 && threadIdx.x == 0) __threadfence();
         if (pendDst) {                                  // finish the previous pick's coverage update
             fold_pending<SV>(pendDst, scratch, ld4, thrAcc);
             pendDst = nullptr;
@@ -1013,6 +1047,7 @@ __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, i
         const int vstar = shPick;
         if (vstar == INT_MAX || vstar < 0 || vstar >= c.M) {
             if (threadIdx.x == 0) atomicOr(prm.status, kDevBadState);
+            j = -1;
             break;
         }
         // warp 0: next block (shared memory only).  last warp: global bookkeeping of this pick.
@@ -1024,15 +1059,28 @@ __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, i
         } else if (threadIdx.x == kSelectThreads - 32) {
             const int64_t at = (int64_t)l * prm.W + j;
             prm.fval[at] = shPlan.f[j];
-            prm.cnt[at] += 1;
-            const int global = prm.perm[c.row0 + vstar];
-            prm.assignment[global] = j;
-            if (prm.order) prm.order[c.row0 + (c.M - nR)] = global;
-            const int k = pos[vstar];
-            const int lastV = cand[nR - 1];
-            cand[k] = lastV;
-            pos[lastV] = k;
-            pos[vstar] = -1;
+            prm.cnt[at] = shPlan.quota[j] - shPlan.room[j];
+            if (res) {
+                // everything this needs is in shared memory: stores only, nothing to wait for
+                const int global = shPerm[vstar];
+                prm.assignment[global] = j;
+                if (prm.order) prm.order[c.row0 + (c.M - nR)] = global;
+                const int k = shPos[vstar];
+                const int lastV = shCand[nR - 1];
+                shCand[k] = lastV;
+                shPos[lastV] = k;
+                shPos[vstar] = -1;
+                cand[k] = lastV;                                // (the sweeps read the list from global memory)
+            } else {
+                const int global = prm.perm[c.row0 + vstar];
+                prm.assignment[global] = j;
+                if (prm.order) prm.order[c.row0 + (c.M - nR)] = global;
+                const int k = pos[vstar];
+                const int lastV = cand[nR - 1];
+                cand[k] = lastV;
+                pos[lastV] = k;
+                pos[vstar] = -1;
+            }
             prm.nR[l] = nR - 1;
             if (nR == 1) atomicSub(&prm.nSweep[3], 1);        // one class fewer to finish
         }
@@ -1053,6 +1101,7 @@ __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, i
         j = shPlan.nextJ;
         if (nR == 0 || j < 0 || shPlan.needSweep) break;
     }
+    if (keep && threadIdx.x == 0) { keep[0] = nR; keep[1] = j; }     // (j = -1 after an inconsistency: the class is given up)
     if (pendDst) fold_pending<SV>(pendDst, scratch, ld4, thrAcc);
     if (shPlan.needSweep && shPlan.sweepSparse) {
         // threshold of the coming pass: element-wise minimum of the listed blocks' coverage vectors
@@ -1213,7 +1262,9 @@ __device__ __forceinline__ void async_pick_cta(const GreedyParams<SV> &prm, int4
     for (int l = me; l < prm.L; l += prm.nPick) mine += prm.desc[l].M > 0 ? 1 : 0;
     unsigned idle = 0;
     unsigned long long busy = 0;
-    bool planKept = false;
+    __shared__ int shKeep[2];
+    const bool owner = prm.nPick >= prm.L;                          // this CTA serves one class only
+    bool kept = false;
     while (mine > 0) {
         bool progressed = false;
         for (int l = me; l < prm.L; l += prm.nPick) {
@@ -1223,7 +1274,7 @@ __device__ __forceinline__ void async_pick_cta(const GreedyParams<SV> &prm, int4
                 if (!(sy.x & 1) && sy.z == sy.y) {
                     e = sy.x;
                     *(volatile int32_t *)&prm.sync[l].epoch = e + 1;    // the class is mine until I publish again
-                    __threadfence();                                    // (also: the sweepers' gains are visible)
+                    if (!owner) __threadfence();                        // (an owner's chain fences after its first loads)
                 }
                 shEpoch = e;
             }
@@ -1233,11 +1284,11 @@ __device__ __forceinline__ void async_pick_cta(const GreedyParams<SV> &prm, int4
             progressed = true;
             unsigned long long t0 = 0;
             if (me == 0 && threadIdx.x == 0) t0 = global_ns();
-            pick_chain(prm, l, e >> 1, scratch, prm.smemBytes, planKept);
-            planKept = prm.nPick >= prm.L;                          // my only class: the block table stays in shared memory
+            pick_chain(prm, l, e >> 1, scratch, prm.smemBytes, owner ? (kept ? 2 : 1) : 0, shKeep);
+            kept = true;
             __syncthreads();                                            // all writes of the chain are issued
             if (threadIdx.x == 0) {
-                const bool finished = prm.nR[l] == 0 || prm.jstar[l] < 0 || ld_volatile32(prm.status) != 0;
+                const bool finished = shKeep[0] == 0 || shKeep[1] < 0;
                 if (!finished) {
                     prm.sync[l].done = 0;
                     prm.sync[l].seq = ((e >> 1) + 1) * prm.L + l;        // sweep number first: batches follow the classes' progress
@@ -1503,7 +1554,7 @@ static rcd_status run_greedy(rcd_ctx *ctx, const Sizes &sz, const Workspace &ws,
     prm.helpMin = 1;
     int maxLd = 0;
     for (const auto &c : descHost) if (c.ld > maxLd) maxLd = c.ld;
-    const int64_t smemCap = (int64_t)ctx->maxSmemOptin - 20 * 1024;  // static shared of the kernels + margin
+    const int64_t smemCap = (int64_t)ctx->maxSmemOptin - 24 * 1024;  // static shared of the kernels + margin
     int64_t smem = (int64_t)batch * maxLd * (int64_t)sizeof(SV);
     if (prm.sparseMinMembers >= 0)                                   // threshold pass: one vector + the warps' rings and queues
         smem = std::max<int64_t>(smem, (int64_t)thr_bytes_aligned(maxLd * (int)sizeof(SV)) + kSparseQueueBytes);
