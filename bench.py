@@ -33,7 +33,7 @@ if ROOT not in sys.path:
 
 
 # DRAM bytes (read + write) of one launch of the dominant kernel under ncu, by (configuration, kernel).
-MEASURED_TRAFFIC = {}
+MEASURED_TRAFFIC = {("C2", "greedy_async_kernel"): 481.2e9}     # profiles/greedy_async_kernel_C2.md
 
 
 def load_peaks():
@@ -246,9 +246,10 @@ def run_ours(args):
     h2d = Xh.numel() * Xh.element_size() + yh.numel() * 4
     d2h = sum(t.numel() * t.element_size() for t in host_out)
 
-    # Roofline of the dominant kernel.  The whole greedy loop is ONE launch (greedy_persistent_kernel:
-    # sweep phases and pick phases separated by grid barriers); it is HBM-bound through its sweep
-    # phases.  Algorithmic bytes = for every sweep of a class, the rows of S of its unassigned samples
+    # Roofline of the dominant kernel.  The whole greedy loop is ONE launch (greedy_async_kernel when
+    # classes are few: pick CTAs and sweep CTAs hand classes back and forth; greedy_persistent_kernel
+    # otherwise: sweep phases and pick phases separated by grid barriers); it is HBM-bound through its
+    # sweeps.  Algorithmic bytes = for every sweep of a class, the rows of S of its unassigned samples
     # plus the coverage vectors of the blocks refreshed (4*ld*(n_R + n) bytes), summed on the device.
     # Duration = CUDA events around the greedy loop on the launching stream (last timed step).
     peaks = load_peaks()
@@ -268,7 +269,8 @@ def run_ours(args):
                 "traffic": MEASURED_TRAFFIC.get((args.config, kernel_name)) if default_setup else None,
                 "launch_ms": prof["greedy_ms"], "bytes_per_launch": prof["sweep_bytes"],
                 "rounds_with_sweeps": int(prof["sweep_launches"])}
-    # the same bytes against the time the kernel spends in its sweep phases (its own clock, CTA 0)
+    # the same bytes against the time the kernel spends sweeping (its own clock: the sweep phases of the
+    # round-based kernel, the busy time of the first sweep CTA of the asynchronous one)
     if prof["persistent_sweep_ns"] > 0:
         ph = prof["sweep_bytes"] / (prof["persistent_sweep_ns"] * 1e-9) / 1e9
         roofline["sweep_phases"] = {"achieved": ph, "frac": ph / peaks["hbm_gbs"], "ms": prof["persistent_sweep_ns"] * 1e-6,
