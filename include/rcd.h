@@ -92,7 +92,10 @@ typedef struct {
                                   order; 0 = default: all classes together */
     int32_t async_help_min;    /* greedy_path 3: row groups a sweep must have left before a sweep CTA whose home is another
                                   class joins it; 0 = default (48) */
-    int32_t reserved[7];       /* must be 0 */
+    int32_t threshold_from;    /* members every out-of-date block must have before a class tries threshold passes; 0 = default (8) */
+    int32_t threshold_hit_shift; /* a threshold pass that finds more than 1 element in 2^k above the threshold sends the class
+                                  back to dense passes until its blocks have twice the members; 0 = default (k = 5) */
+    int32_t reserved[5];       /* must be 0 */
 } rcd_config;
 
 /* Timings and counters of the last rcd_partition / rcd_partition_host on a context (profile >= 1). */

@@ -277,3 +277,34 @@ def objective(features: np.ndarray, labels: np.ndarray, assignment: np.ndarray, 
         for j in range(W):
             out[l, j] = f_plain(S, np.nonzero(a == j)[0], objective)
     return out
+
+
+# ----------------------------------------------------------------------------- downstream hook (Algorithm 2, initialisation)
+
+def worker_lists(assignment: np.ndarray, W: int) -> Tuple[np.ndarray, np.ndarray]:
+    """The local subset of every worker (Algorithm 2: worker i "imports the local subset xi_i from the
+    subsets A_1 .. A_N"): worker j's list is every dataset index whose block is j, in ascending order.
+    Returns (offsets [W+1], indices [N]) with worker j's list at indices[offsets[j]:offsets[j+1]].
+    Plain definition, one pass per worker."""
+    assignment = np.asarray(assignment)
+    lists = []
+    for j in range(W):
+        mine = [i for i in range(len(assignment)) if assignment[i] == j]
+        lists.append(np.asarray(mine, dtype=np.int32))
+    offsets = np.zeros(W + 1, dtype=np.int64)
+    for j in range(W):
+        offsets[j + 1] = offsets[j] + len(lists[j])
+    indices = np.concatenate(lists) if lists else np.zeros(0, np.int32)
+    return offsets, indices.astype(np.int32)
+
+
+def batch_sizes(B: int, capacities: Sequence[float]) -> np.ndarray:
+    """Per-worker batch sizes of Algorithm 2's initialisation.  The text below Algorithm 2 makes the batch
+    size of a worker proportional to its processing speed (the algorithm's own line prints the inverse
+    ratio): b_i = B * r_i / r_1 with worker 1 the reference, rounded half up to an integer, at least 1."""
+    r = [float(x) for x in capacities]
+    out = []
+    for ri in r:
+        x = float(B) * ri / r[0]
+        out.append(max(1, int(np.floor(x + 0.5))))
+    return np.asarray(out, dtype=np.int64)

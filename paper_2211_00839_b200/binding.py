@@ -47,7 +47,8 @@ class RcdError(RuntimeError):
 class RcdConfig(C.Structure):
     _fields_ = [("sweep_batch_max", C.c_int32), ("similarity_path", C.c_int32), ("profile", C.c_int32),
                 ("greedy_path", C.c_int32), ("similarity_kind", C.c_int32), ("objective", C.c_int32), ("sweep_mode", C.c_int32), ("async_group", C.c_int32),
-                ("async_help_min", C.c_int32), ("reserved", C.c_int32 * 7)]
+                ("async_help_min", C.c_int32), ("threshold_from", C.c_int32), ("threshold_hit_shift", C.c_int32),
+                ("reserved", C.c_int32 * 5)]
 
 
 class RcdProfile(C.Structure):
@@ -146,7 +147,7 @@ class Context:
 
     def __init__(self, device: int = 0, sweep_batch_max: int = 0, similarity_path: int = 0, profile: int = 0,
                  greedy_path: int = 0, similarity_kind: int = 0, objective: int = 0, sweep_mode: int = 0,
-                 async_group: int = 0, async_help_min: int = 0):
+                 async_group: int = 0, async_help_min: int = 0, threshold_from: int = 0, threshold_hit_shift: int = 0):
         torch = _torch()
         if not torch.cuda.is_available():
             raise RcdError(4, "no CUDA device: this library has no CPU path")
@@ -162,6 +163,8 @@ class Context:
         cfg.sweep_mode = sweep_mode
         cfg.async_group = async_group
         cfg.async_help_min = async_help_min
+        cfg.threshold_from = threshold_from
+        cfg.threshold_hit_shift = threshold_hit_shift
         self.similarity_kind = similarity_kind
         self._h = C.c_void_p()
         st = lib.rcd_create(C.byref(self._h), self.device, C.byref(cfg))

@@ -294,7 +294,8 @@ rcd_status rcd_create(rcd_ctx **out, int cuda_device, const rcd_config *cfg)
         if (cfg->sweep_mode != 0 && cfg->sweep_mode != 1) return RCD_ERR_INVALID_ARG;
         if (cfg->async_group < 0 || cfg->async_group > 4096) return RCD_ERR_INVALID_ARG;
         if (cfg->async_help_min < 0) return RCD_ERR_INVALID_ARG;
-        for (int i = 0; i < 7; ++i) if (cfg->reserved[i] != 0) return RCD_ERR_INVALID_ARG;
+        if (cfg->threshold_from < 0 || cfg->threshold_hit_shift < 0 || cfg->threshold_hit_shift > 30) return RCD_ERR_INVALID_ARG;
+        for (int i = 0; i < 5; ++i) if (cfg->reserved[i] != 0) return RCD_ERR_INVALID_ARG;
     }
     int count = 0;
     if (cudaGetDeviceCount(&count) != cudaSuccess || cuda_device < 0 || cuda_device >= count) {

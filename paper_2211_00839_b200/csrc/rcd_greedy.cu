@@ -83,6 +83,7 @@ struct GreedyParams {
     int32_t segIters;       // int path: chunk iterations a 32-bit partial sum can take without overflow
     int32_t sweepWarps;     // warps of one sweep launch (CTAs x 16)
     uint32_t one;           // the value 1, opaque to the compiler (see accumulate_chunk)
+    int32_t hitShift;           // a threshold pass with more than 1 element in 2^hitShift above the threshold makes the class wait
     int32_t sparseMinMembers;   // threshold passes start once every out-of-date block has this many members (<0: never)
     // asynchronous kernel (greedy_async_kernel); asyncMode = 0 everywhere else
     ClassSync *sync;            // [L] hand-off words
@@ -209,7 +210,7 @@ __device__ void plan_decide(const GreedyParams<SV> &prm, int l, const ClassDesc 
             const unsigned long long hits = *(const volatile unsigned long long *)&prm.hitCount[l];   // (added to by the sweeping CTAs)
             atomicAdd(&prm.phaseNs[3], hits);
             atomicAdd(&prm.phaseNs[4], elems);
-            if (hits * 32ull > elems) { from = 2 * fewest; prm.sparseFrom[l] = from; }
+            if ((hits << prm.hitShift) > elems) { from = 2 * fewest; prm.sparseFrom[l] = from; }
             prm.hitCount[l] = 0;
             prm.sparseElems[l] = 0;
         }
@@ -1544,7 +1545,8 @@ static rcd_status run_greedy(rcd_ctx *ctx, const Sizes &sz, const Workspace &ws,
     prm.batchMax = batch;
     prm.sweepWarps = ctx->smCount * (kSweepThreads / 32);
     prm.one = 1u;
-    prm.sparseMinMembers = ctx->cfg.sweep_mode == 1 ? -1 : 8;
+    prm.sparseMinMembers = ctx->cfg.sweep_mode == 1 ? -1 : (ctx->cfg.threshold_from > 0 ? ctx->cfg.threshold_from : 8);
+    prm.hitShift = ctx->cfg.threshold_hit_shift > 0 ? ctx->cfg.threshold_hit_shift : 5;
     prm.sync = ws.sync;
     prm.tickets = ws.tickets;
     prm.sweepF = ws.sweepF;

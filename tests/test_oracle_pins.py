@@ -517,3 +517,40 @@ def test_graph_cut_incremental_close_to_plain_in_double_and_invariants():
         assert np.array_equal(np.bincount(res.assignment[ids], minlength=4), res.quotas[l])
     again = orc.objective(wl.features, wl.labels, res.assignment, 4, wl.L, objective="cut")
     assert np.allclose(again, res.part_values, rtol=1e-12)
+
+
+# ----------------------------------------------------------------------------- downstream hook: worker lists, batch sizes
+
+def test_worker_lists_hand_example():
+    """Seven samples, three workers, written out by hand."""
+    a = np.array([2, 0, 1, 0, 2, 2, 1], dtype=np.int32)
+    off, idx = orc.worker_lists(a, 3)
+    assert off.tolist() == [0, 2, 4, 7]
+    assert idx.tolist() == [1, 3, 2, 6, 0, 4, 5]
+    off, idx = orc.worker_lists(a, 4)                      # a worker that got nothing
+    assert off.tolist() == [0, 2, 4, 7, 7]
+
+
+def test_worker_lists_are_a_stable_partition_with_quota_sizes():
+    """On a real partition: the lists are disjoint, cover the dataset, are ascending, agree with a stable
+    argsort (library routine), and worker j holds sum_l C_{l,j} samples (Algorithm 1's constraint)."""
+    from paper_2211_00839_b200.workloads import make_workload
+    wl = make_workload("C1")
+    ref = orc.partition(wl.features, wl.labels, wl.capacities, wl.L, variant="incremental")
+    off, idx = orc.worker_lists(ref.assignment, wl.W)
+    assert sorted(idx.tolist()) == list(range(wl.N))
+    assert np.array_equal(idx, np.argsort(ref.assignment, kind="stable"))
+    for j in range(wl.W):
+        mine = idx[off[j]:off[j + 1]]
+        assert np.all(np.diff(mine) > 0) and np.all(ref.assignment[mine] == j)
+        assert len(mine) == int(ref.quotas[:, j].sum())
+    assert (off[1:] - off[:-1]).tolist() == [50, 50, 100, 200]   # 2 classes x (25, 25, 50, 100)
+
+
+def test_batch_sizes_closed_forms():
+    assert orc.batch_sizes(32, [1, 1, 2, 4]).tolist() == [32, 32, 64, 128]
+    assert orc.batch_sizes(32, [2, 1, 4]).tolist() == [32, 16, 64]          # relative to worker 1
+    assert orc.batch_sizes(10, [4, 1, 3]).tolist() == [10, 3, 8]            # 2.5 -> 3, 7.5 -> 8: halves round up
+    assert orc.batch_sizes(1, [8, 1]).tolist() == [1, 1]                    # never below one sample
+    b = orc.batch_sizes(64, [1.0, 2.5, 3.5])
+    assert b.tolist() == [64, 160, 224] and b[1] / b[0] == 2.5
