@@ -232,6 +232,26 @@ RCD_API rcd_status rcd_objective(rcd_ctx *ctx, const void *features_dev, rcd_fea
                          void *part_values_dev, void *total_dev, void *workspace_dev,
                          size_t workspace_bytes, void *cuda_stream);
 
+/* ---- per-worker lists and batch sizes (Algorithm 2, initialisation: every worker imports its local subset
+ *      from the blocks A_1 .. A_N and runs with a batch size set by its capacity ratio) ------------------------ */
+
+RCD_API rcd_status rcd_worker_lists_workspace_bytes(rcd_ctx *ctx, int64_t N, int32_t W, size_t *bytes_out);
+
+/* Turns an assignment (rcd_partition's output) into one index list per worker.
+ *   assignment_dev [N]   block of every sample, each in [0, W) (anything else: RCD_ERR_INVALID_ARG)
+ *   offsets_dev    [W+1] out, int64: worker j's list is indices_dev[offsets[j] .. offsets[j+1])
+ *   indices_dev    [N]   out: dataset indices, ascending inside every list
+ * workspace_dev: 256-byte aligned, rcd_worker_lists_workspace_bytes.  Blocks once on the stream to read the W
+ * list sizes back (they fix the offsets); the lists themselves are only enqueued. */
+RCD_API rcd_status rcd_worker_lists(rcd_ctx *ctx, const int32_t *assignment_dev, int64_t N, int32_t W, int64_t *offsets_dev,
+                            int32_t *indices_dev, void *workspace_dev, size_t workspace_bytes, void *cuda_stream);
+
+/* Host-only.  Batch size of every worker for a reference batch size B of worker 1: b_j = B r_j / r_1, rounded
+ * half up, at least 1.  (The text below Algorithm 2 makes the batch size proportional to the processing speed;
+ * the algorithm's own initialisation line prints the inverse ratio, B r_1 / r_j.  This follows the text: with
+ * lists and batches both proportional to r_j every worker needs the same number of steps per epoch.) */
+RCD_API rcd_status rcd_batch_sizes(int64_t B, const double *capacities_host, int32_t W, int64_t *batch_sizes_host_out);
+
 /* ---- objective of one class without any allocation (no counterpart in the paper) ----------- */
 
 /* The paper has nothing corresponding to this entry point: it exists for callers that cannot

@@ -35,7 +35,8 @@ EXPORTS = ["rcd_create", "rcd_destroy", "rcd_last_error", "rcd_version", "rcd_sy
            "rcd_quotas", "rcd_similarity", "rcd_similarity_gaussian_workspace_bytes", "rcd_similarity_gaussian",
            "rcd_partition_workspace_bytes", "rcd_partition",
            "rcd_partition_host_workspace_bytes", "rcd_partition_host", "rcd_objective_workspace_bytes",
-           "rcd_objective", "rcd_objective_class_static"]
+           "rcd_objective", "rcd_objective_class_static",
+           "rcd_worker_lists_workspace_bytes", "rcd_worker_lists", "rcd_batch_sizes"]
 
 
 class RcdError(RuntimeError):
@@ -88,6 +89,9 @@ def _load() -> C.CDLL:
     lib.rcd_partition_host.argtypes = [vp, vp, C.c_int, i64, i64, vp, i32, vp, i32, vp, vp, vp, vp, sz, vp]
     lib.rcd_objective.argtypes = [vp, vp, C.c_int, i64, i64, vp, i32, vp, i32, vp, vp, vp, sz, vp]
     lib.rcd_objective_class_static.argtypes = [vp, vp, C.c_int, i64, i64, vp, i32, vp, vp, vp]
+    lib.rcd_worker_lists_workspace_bytes.argtypes = [vp, i64, i32, C.POINTER(sz)]
+    lib.rcd_worker_lists.argtypes = [vp, vp, i64, i32, vp, vp, vp, sz, vp]
+    lib.rcd_batch_sizes.argtypes = [i64, vp, i32, vp]
     for name in EXPORTS:
         f = getattr(lib, name)
         if name not in ("rcd_destroy", "rcd_last_error", "rcd_version"):
@@ -109,6 +113,16 @@ def rcd_quotas(M: int, capacities: Sequence[float]) -> np.ndarray:
     st = lib.rcd_quotas(int(M), r.ctypes.data_as(C.c_void_p), len(r), out.ctypes.data_as(C.c_void_p))
     if st != 0:
         raise RcdError(st, "rcd_quotas")
+    return out
+
+
+def rcd_batch_sizes(B: int, capacities: Sequence[float]) -> np.ndarray:
+    """Per-worker batch sizes b_j = B r_j / r_1 (host only; no GPU needed)."""
+    r = np.ascontiguousarray(capacities, dtype=np.float64)
+    out = np.empty(len(r), dtype=np.int64)
+    st = lib.rcd_batch_sizes(int(B), r.ctypes.data_as(C.c_void_p), len(r), out.ctypes.data_as(C.c_void_p))
+    if st != 0:
+        raise RcdError(st, "rcd_batch_sizes")
     return out
 
 
@@ -344,6 +358,22 @@ class Context:
                                       C.c_void_p(values.data_ptr()), C.c_void_p(total.data_ptr()),
                                       C.c_void_p(ws.data_ptr()), ws.numel(), self._stream()))
         return values, total
+
+
+def rcd_worker_lists(ctx: Context, assignment, W: int):
+    """assignment [N] int32 on the device -> (offsets [W+1] int64, indices [N] int32): worker j's samples are
+    indices[offsets[j]:offsets[j+1]], ascending."""
+    torch = _torch()
+    assignment = assignment.contiguous()
+    N = assignment.numel()
+    out = C.c_size_t()
+    ctx._check(lib.rcd_worker_lists_workspace_bytes(ctx._h, N, W, C.byref(out)))
+    ws = ctx.workspace(int(out.value))
+    offsets = torch.empty(W + 1, dtype=torch.int64, device=assignment.device)
+    indices = torch.empty(N, dtype=torch.int32, device=assignment.device)
+    ctx._check(lib.rcd_worker_lists(ctx._h, C.c_void_p(assignment.data_ptr()), N, W, C.c_void_p(offsets.data_ptr()),
+                                    C.c_void_p(indices.data_ptr()), C.c_void_p(ws.data_ptr()), ws.numel(), ctx._stream()))
+    return offsets, indices
 
 
 def rcd_objective_class_static(ctx: Context, S, assignment, W: int, part_values, total):

@@ -416,6 +416,96 @@ rcd_status rcd_quotas(int64_t M, const double *capacities_host, int32_t W, int32
     return RCD_OK;
 }
 
+// ---- downstream hook: per-worker index lists and batch sizes (Algorithm 2, initialisation) ----
+
+struct ListsWorkspace {
+    int32_t *status;      // [4]
+    int32_t *counts;      // [W]
+    ClassDesc *desc;      // [W] (only row0 is used: where a worker's list starts)
+    int32_t *chunkHist;   // [nChunks][W]
+    size_t bytes;
+};
+
+static size_t layout_lists(void *base, int64_t N, int32_t W, ListsWorkspace *out)
+{
+    Carver c{static_cast<unsigned char *>(base)};
+    ListsWorkspace w{};
+    const size_t Wn = (size_t)std::max<int32_t>(W, 1);
+    w.status = c.take<int32_t>(4);
+    w.counts = c.take<int32_t>(Wn);
+    w.desc = c.take<ClassDesc>(Wn);
+    w.chunkHist = c.take<int32_t>((size_t)std::max<int32_t>(chunks_for(N), 1) * Wn);
+    w.bytes = align_up(c.off);
+    if (out) *out = w;
+    return w.bytes;
+}
+
+rcd_status rcd_worker_lists_workspace_bytes(rcd_ctx *ctx, int64_t N, int32_t W, size_t *bytes_out)
+{
+    if (!ctx || !bytes_out) return RCD_ERR_INVALID_ARG;
+    if (N < 0 || N > 0x7fffffffLL || W <= 0) return fail(ctx, RCD_ERR_INVALID_ARG, "N=%lld or W=%d out of range", (long long)N, W);
+    *bytes_out = layout_lists(nullptr, N, W, nullptr);
+    return RCD_OK;
+}
+
+rcd_status rcd_worker_lists(rcd_ctx *ctx, const int32_t *assignment_dev, int64_t N, int32_t W, int64_t *offsets_dev,
+                            int32_t *indices_dev, void *workspace_dev, size_t workspace_bytes, void *cuda_stream)
+{
+    if (!ctx) return RCD_ERR_INVALID_ARG;
+    if (N < 0 || N > 0x7fffffffLL || W <= 0) return fail(ctx, RCD_ERR_INVALID_ARG, "N=%lld or W=%d out of range", (long long)N, W);
+    if (!offsets_dev || !workspace_dev || (N > 0 && (!assignment_dev || !indices_dev))) return fail(ctx, RCD_ERR_INVALID_ARG, "null device pointer");
+    if (((uintptr_t)workspace_dev) % kAlign != 0) return fail(ctx, RCD_ERR_INVALID_ARG, "workspace must be 256-byte aligned");
+    if ((size_t)W + 1 > ctx->hostStageInts) return fail(ctx, RCD_ERR_UNSUPPORTED, "W=%d exceeds the %zu blocks the context can stage", W, ctx->hostStageInts);
+    ListsWorkspace ws{};
+    const size_t need = layout_lists(workspace_dev, N, W, &ws);
+    if (workspace_bytes < need) return fail(ctx, RCD_ERR_WORKSPACE_TOO_SMALL, "workspace has %zu bytes, %zu needed", workspace_bytes, need);
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    RCD_CUDA(ctx, cudaSetDevice(ctx->device));
+    ctx->kernelLaunches = 0;
+    ctx->statusDev = ws.status;
+    RCD_CUDA(ctx, cudaMemsetAsync(ws.status, 0, 4 * sizeof(int32_t), st));
+    RCD_CUDA(ctx, cudaMemsetAsync(ws.counts, 0, (size_t)W * sizeof(int32_t), st));
+    // sizes of the lists (a histogram of the block numbers), read back: they fix where each list starts
+    rcd_status rs = launch_count_labels(ctx, assignment_dev, N, W, ws.counts, ws.status, st);
+    if (rs != RCD_OK) return rs;
+    RCD_CUDA(ctx, cudaMemcpyAsync(ctx->hostStage, ws.counts, (size_t)W * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+    RCD_CUDA(ctx, cudaMemcpyAsync(ctx->hostStage + W, ws.status, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+    RCD_CUDA(ctx, cudaStreamSynchronize(st));
+    if (ctx->hostStage[W] & kDevBadLabel) return fail(ctx, RCD_ERR_INVALID_ARG, "an assignment entry lies outside [0, %d)", W);
+    std::vector<ClassDesc> desc((size_t)W);
+    std::vector<int64_t> offsets((size_t)W + 1);
+    int64_t run = 0;
+    for (int32_t j = 0; j < W; ++j) {
+        ClassDesc c{};
+        c.M = ctx->hostStage[j];
+        c.row0 = (int32_t)run;
+        desc[(size_t)j] = c;
+        offsets[(size_t)j] = run;
+        run += c.M;
+    }
+    offsets[(size_t)W] = run;
+    if (run != N) return fail(ctx, RCD_ERR_INTERNAL, "list sizes sum to %lld, expected %lld", (long long)run, (long long)N);
+    // (pageable host memory: the runtime stages these copies before it returns)
+    RCD_CUDA(ctx, cudaMemcpyAsync(offsets_dev, offsets.data(), offsets.size() * sizeof(int64_t), cudaMemcpyHostToDevice, st));
+    RCD_CUDA(ctx, cudaMemcpyAsync(ws.desc, desc.data(), desc.size() * sizeof(ClassDesc), cudaMemcpyHostToDevice, st));
+    // a stable split by block number: inside a list the dataset indices ascend
+    return launch_stable_split(ctx, assignment_dev, N, W, chunks_for(N), ws.chunkHist, ws.desc, indices_dev, st);
+}
+
+rcd_status rcd_batch_sizes(int64_t B, const double *capacities_host, int32_t W, int64_t *batch_sizes_host_out)
+{
+    if (B <= 0 || W <= 0 || !capacities_host || !batch_sizes_host_out) return RCD_ERR_INVALID_ARG;
+    for (int32_t j = 0; j < W; ++j)
+        if (!(capacities_host[j] > 0.0) || !std::isfinite(capacities_host[j])) return RCD_ERR_INVALID_ARG;
+    for (int32_t j = 0; j < W; ++j) {
+        const double x = (double)B * capacities_host[j] / capacities_host[0];
+        if (!(x < 9.0e18)) return RCD_ERR_INVALID_ARG;
+        const int64_t b = (int64_t)std::floor(x + 0.5);
+        batch_sizes_host_out[j] = b < 1 ? 1 : b;
+    }
+    return RCD_OK;
+}
+
 rcd_status rcd_similarity(rcd_ctx *ctx, const void *X_dev, rcd_feat_dtype dtype, int64_t M, int64_t d,
                           int64_t batch, void *S_dev, int64_t ldS, void *cuda_stream)
 {

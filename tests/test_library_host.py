@@ -47,6 +47,21 @@ def test_quotas_match_oracle_and_closed_forms(binding):
         assert np.array_equal(a, orc.quotas(M, r))
 
 
+def test_batch_sizes_match_oracle_and_closed_forms(binding):
+    from oracle import rcd_oracle as orc
+    assert binding.rcd_batch_sizes(32, [1, 1, 2, 4]).tolist() == [32, 32, 64, 128]
+    assert binding.rcd_batch_sizes(10, [4, 1, 3]).tolist() == [10, 3, 8]
+    rng = np.random.default_rng(12)
+    for _ in range(200):
+        W = int(rng.integers(1, 70))
+        B = int(rng.integers(1, 2000))
+        r = np.round(rng.uniform(0.05, 9.0, size=W) * 4) / 4 + 0.25
+        assert np.array_equal(binding.rcd_batch_sizes(B, r), orc.batch_sizes(B, r))
+    for B, caps in ((0, [1.0]), (8, [1.0, 0.0]), (8, [float("nan"), 1.0])):
+        with pytest.raises(binding.RcdError):
+            binding.rcd_batch_sizes(B, caps)
+
+
 def test_quotas_reject_bad_arguments(binding):
     for caps in ([1.0, 0.0], [1.0, -2.0], [float("nan")], [float("inf"), 1.0]):
         with pytest.raises(binding.RcdError):
