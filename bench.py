@@ -131,7 +131,7 @@ def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    wl = make_workload(args.config)
+    wl = make_workload(args.config, L=args.classes or None)
     cores = min(os.cpu_count() or 1, wl.L)
     vals, walls = [], []
     for i in range(args.warmup + args.steps):
@@ -174,7 +174,7 @@ def run_ours(args):
     dev = torch.device("cuda", local)
 
     # weak scaling: every rank partitions its own dataset of the same shape (seed differs per rank)
-    wl = make_workload(args.config, seed=CONFIGS[args.config]["seed"] + 1000 * rank)
+    wl = make_workload(args.config, L=args.classes or None, seed=CONFIGS[args.config]["seed"] + 1000 * rank)
     M = wl.N // wl.L
     Xh = rcd.features_to_torch(wl.features, pin=True)
     yh = torch.from_numpy(wl.labels).pin_memory()
@@ -253,7 +253,7 @@ def run_ours(args):
     # plus the coverage vectors of the blocks refreshed (4*ld*(n_R + n) bytes), summed on the device.
     # Duration = CUDA events around the greedy loop on the launching stream (last timed step).
     peaks = load_peaks()
-    default_setup = args.sweep_batch in (0, 8) and args.async_group == 0 and args.async_help_min == 0 and args.similarity == "dot"
+    default_setup = args.classes == 0 and args.sweep_batch in (0, 8) and args.async_group == 0 and args.async_help_min == 0 and args.similarity == "dot"
     loop_s = prof["greedy_ms"] * 1e-3
     achieved = prof["sweep_bytes"] / loop_s / 1e9 if loop_s > 0 else 0.0
     if args.objective != "facility":
@@ -321,7 +321,7 @@ def run_ours(args):
               "clocks": clocks, "roofline": roofline}
 
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        base_wl = make_workload(args.config)
+        base_wl = make_workload(args.config, L=args.classes or None)
         cores = min(os.cpu_count() or 1, base_wl.L)
         r = oracle_sample(base_wl, args.ref_picks, cores)
         result["cpu_baseline"] = {
@@ -342,6 +342,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="C2", choices=["C1", "C2", "C3", "C4", "C5"])
+    ap.add_argument("--classes", type=int, default=0, help="fewer (or more) classes than the configuration names: a reduced copy for profiling")
     ap.add_argument("--sweep-batch", type=int, default=0, help="sweep_batch_max (0 = library default)")
     ap.add_argument("--similarity", default="dot", choices=["dot", "gaussian"], help="similarity of Section 4 item 2")
     ap.add_argument("--objective", default="facility", choices=["facility", "cut"], help="submodular function of Section 4 item 2")
