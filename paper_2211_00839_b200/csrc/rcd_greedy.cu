@@ -202,12 +202,15 @@ __device__ void plan_decide(const GreedyParams<SV> &prm, int l, const ClassDesc 
     // 1 element in 32 turned out to be above the threshold, the next try waits until the blocks
     // have twice the members they had.  Near the end of a class (few rows left) the dense pass,
     // which can split the columns of a row over several warps, keeps more warps busy.
+    // (everything the decision reads from global memory is loaded here, back to back: one trip, not four)
+    const int remaining = *(volatile int32_t *)&prm.nSweep[3];      // unfinished classes
     int from = 0;
     if (lane == 0) {
-        from = prm.sparseFrom[l];
-        const unsigned long long elems = prm.sparseElems[l];
+        const int fromLd = *(volatile int32_t *)&prm.sparseFrom[l];
+        const unsigned long long elems = *(volatile unsigned long long *)&prm.sparseElems[l];
+        const unsigned long long hits = *(volatile unsigned long long *)&prm.hitCount[l];     // (added to by the sweeping CTAs)
+        from = fromLd;
         if (elems) {
-            const unsigned long long hits = *(const volatile unsigned long long *)&prm.hitCount[l];   // (added to by the sweeping CTAs)
             atomicAdd(&prm.phaseNs[3], hits);
             atomicAdd(&prm.phaseNs[4], elems);
             if ((hits << prm.hitShift) > elems) { from = 2 * fewest; prm.sparseFrom[l] = from; }
@@ -216,7 +219,7 @@ __device__ void plan_decide(const GreedyParams<SV> &prm, int l, const ClassDesc 
         }
     }
     from = __shfl_sync(0xffffffffu, from, 0);
-    const int64_t together0 = max(*(volatile int32_t *)&prm.nSweep[3], 1);
+    const int64_t together0 = max(remaining, 1);
     const bool sparse = prm.sparseMinMembers >= 0 && prm.batchMax > 1 && nStale > 1 && fewest >= from &&
                         (int64_t)thr_bytes_aligned(c.ld * (int)sizeof(SV)) + kSparseQueueBytes <= prm.smemBytes &&
                         together0 * ((nR + kSparseRows - 1) / kSparseRows) * 4 >= prm.sweepWarps;
@@ -253,7 +256,7 @@ __device__ void plan_decide(const GreedyParams<SV> &prm, int l, const ClassDesc 
     // unfinished class, once per round) cover every warp of the launch, at least one 128-column chunk per warp
     const int R = sparse ? kSparseRows : rows_per_group(P);
     const int64_t nGroups = (nR + R - 1) / R;
-    const int rem = *(volatile int32_t *)&prm.nSweep[3];              // unfinished classes: they all sweep in the same round
+    const int rem = remaining;                                        // unfinished classes: they all sweep in the same round
     const int64_t together = rem > 1 ? rem : 1;
     const int chunks = (c.ld + 127) / 128;
     int CS = 1;
