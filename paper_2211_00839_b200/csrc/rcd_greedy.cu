@@ -143,9 +143,29 @@ constexpr int kSparseQueueBytes = kSparseWarpBytes * (kSweepThreads / 32);
 __host__ __device__ inline int thr_bytes_aligned(int bytes) { return (bytes + 127) & ~127; }
 static_assert(kSparseWarpBytes % 128 == 0, "per-warp rings must keep the 128-byte alignment");
 
+// What plan_decide reads from global memory when it has to schedule a sweep.  A chain of picks schedules
+// at most one (its last pick), and nothing here changes during the chain, so the chain loads it at its
+// start, under the first argmax, instead of waiting for it at the end.
+struct PlanGlobals {
+    int32_t remaining;              // unfinished classes
+    int32_t from;                   // sparseFrom[l]
+    unsigned long long elems;       // sparseElems[l]
+    unsigned long long hits;        // hitCount[l] (added to by the sweeping CTAs)
+};
+template <typename SV>
+__device__ __forceinline__ PlanGlobals plan_globals(const GreedyParams<SV> &prm, int l)
+{
+    PlanGlobals g;
+    g.remaining = *(volatile int32_t *)&prm.nSweep[3];
+    g.from = *(volatile int32_t *)&prm.sparseFrom[l];
+    g.elems = *(volatile unsigned long long *)&prm.sparseElems[l];
+    g.hits = *(volatile unsigned long long *)&prm.hitCount[l];
+    return g;
+}
+
 template <typename SV>
 __device__ void plan_decide(const GreedyParams<SV> &prm, int l, const ClassDesc &c, int nR, int nextStep,
-                            PlanShared<typename Arith<SV>::FV> &sh)
+                            PlanShared<typename Arith<SV>::FV> &sh, const PlanGlobals *pre = nullptr)
 {
     using FV = typename Arith<SV>::FV;
     const int lane = threadIdx.x & 31;
@@ -202,18 +222,19 @@ __device__ void plan_decide(const GreedyParams<SV> &prm, int l, const ClassDesc 
     // 1 element in 32 turned out to be above the threshold, the next try waits until the blocks
     // have twice the members they had.  Near the end of a class (few rows left) the dense pass,
     // which can split the columns of a row over several warps, keeps more warps busy.
-    // (everything the decision reads from global memory is loaded here, back to back: one trip, not four)
-    const int remaining = *(volatile int32_t *)&prm.nSweep[3];      // unfinished classes
+    // (everything the decision reads from global memory: loaded by the caller beforehand, or here, back to
+    // back: one trip to memory)
+    PlanGlobals g;
+    if (pre) g = *pre;
+    else g = plan_globals(prm, l);
+    const int remaining = g.remaining;
     int from = 0;
     if (lane == 0) {
-        const int fromLd = *(volatile int32_t *)&prm.sparseFrom[l];
-        const unsigned long long elems = *(volatile unsigned long long *)&prm.sparseElems[l];
-        const unsigned long long hits = *(volatile unsigned long long *)&prm.hitCount[l];     // (added to by the sweeping CTAs)
-        from = fromLd;
-        if (elems) {
-            atomicAdd(&prm.phaseNs[3], hits);
-            atomicAdd(&prm.phaseNs[4], elems);
-            if ((hits << prm.hitShift) > elems) { from = 2 * fewest; prm.sparseFrom[l] = from; }
+        from = g.from;
+        if (g.elems) {
+            atomicAdd(&prm.phaseNs[3], g.hits);
+            atomicAdd(&prm.phaseNs[4], g.elems);
+            if ((g.hits << prm.hitShift) > g.elems) { from = 2 * fewest; prm.sparseFrom[l] = from; }
             prm.hitCount[l] = 0;
             prm.sparseElems[l] = 0;
         }
@@ -233,6 +254,23 @@ __device__ void plan_decide(const GreedyParams<SV> &prm, int l, const ClassDesc 
     int32_t *parts = prm.sweepParts + (int64_t)l * kSparseMax;
     if (lane == 0) { parts[0] = jstar; valid[jstar] = 1; sh.open[jstar] = 1; }
     __syncwarp();
+    if (nStale <= cap) {
+        // every out-of-date non-full block is listed: after j* in index order (the order of the list does not
+        // enter any result: each block's gains are summed by themselves)
+        int k = 1;
+        for (int p0 = 0; p0 < W; p0 += 32) {
+            const int p = p0 + lane;
+            const bool take = p < W && sh.open[p] == 3;
+            const unsigned m = __ballot_sync(0xffffffffu, take);
+            if (take) {
+                parts[k + __popc(m & ((1u << lane) - 1u))] = p;
+                valid[p] = 1;
+                sh.open[p] = 1;
+            }
+            k += __popc(m);
+        }
+        __syncwarp();
+    } else
     for (int k = 1; k < n; ++k) {
         // next out-of-date non-full block of least f: the one most likely to be chosen soon
         FV qF = 0;
@@ -980,6 +1018,8 @@ __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, i
         for (int i = threadIdx.x; i < ld4; i += kSelectThreads) thrAcc[i] = top;
     }
     int chainLen = 0;
+    __shared__ PlanGlobals shPre;
+    if (threadIdx.x == 0) shPre = plan_globals(prm, l);     // (in flight under the first argmax; read after its barriers)
 
     for (;;) {
         const GV *G = prm.gains + c.vOff + (int64_t)j * c.ld;
@@ -1059,7 +1099,7 @@ __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, i
         const int4 *row = reinterpret_cast<const int4 *>(prm.S + c.sOff + (int64_t)vstar * c.ld);
         int4 *cov = reinterpret_cast<int4 *>(prm.cover + c.vOff + (int64_t)j * c.ld);
         if (warp == 0) {
-            plan_decide(prm, l, c, nR - 1, round + 1, shPlan);
+            plan_decide(prm, l, c, nR - 1, round + 1, shPlan, &shPre);
         } else if (threadIdx.x == kSelectThreads - 32) {
             const int64_t at = (int64_t)l * prm.W + j;
             prm.fval[at] = shPlan.f[j];
