@@ -253,6 +253,17 @@ def test_threshold_passes_int8_exact(rcd, orc, path):
     assert np.array_equal(a1, a) and np.array_equal(o1, o) and np.array_equal(v1, v)
 
 
+@pytest.mark.parametrize("knobs", [dict(greedy_path=3, async_group=1), dict(greedy_path=3, async_group=2, async_help_min=1),
+                                   dict(greedy_path=3, async_help_min=400), dict(threshold_from=1), dict(threshold_from=2, threshold_hit_shift=3),
+                                   dict(greedy_path=2, threshold_from=1, threshold_hit_shift=7), dict(greedy_path=1, threshold_from=3)])
+def test_scheduling_knobs_never_change_a_result(rcd, orc, knobs):
+    """Serving order of the asynchronous loop and the start / back-off rule of the threshold passes only move
+    work around: assignment, pick order and block values stay those of the oracle."""
+    from paper_2211_00839_b200.workloads import make_workload
+    wl = make_workload("C2", L=4, M=900)
+    check_exact(rcd, orc, wl, **knobs)
+
+
 def test_threshold_passes_many_blocks_exact(rcd, orc):
     """W = 64: one threshold pass refreshes more than 32 blocks (two blocks per lane)."""
     from paper_2211_00839_b200.workloads import make_workload
