@@ -487,6 +487,7 @@ __device__ __forceinline__ void sweep_class(const GreedyParams<SV> &prm, int l, 
     // `ticket` hands out the row groups.  firstTicket >= 0: the CTA has already drawn one ticket per
     // team (firstTicket + team); `done` (may be null) counts the row groups whose gains are written.
     bool preDrawn = firstTicket >= 0;
+    int finished = 0;                             // row groups of this sweep this team has completed
 
     for (;;) {
         int g = 0;
@@ -617,10 +618,13 @@ __device__ __forceinline__ void sweep_class(const GreedyParams<SV> &prm, int l, 
                 G[(int64_t)parts[p] * c.ld + row] = gain;
             }
         }
-        if (done != nullptr && wIn == 0) {
-            __syncwarp();
-            if (lane == 0) { __threadfence(); atomicAdd(done, 1); }
-        }
+        ++finished;
+    }
+    // The row groups this team finished are reported together, once the sweep's tickets have run out for it: the
+    // class's pick CTA only needs the total, and one fence then covers the gains of all of them.
+    if (done != nullptr && wIn == 0 && finished > 0) {
+        __syncwarp();
+        if (lane == 0) { __threadfence(); atomicAdd(done, finished); }
     }
 }
 
@@ -670,6 +674,7 @@ __device__ __noinline__ void sweep_class_sparse(const GreedyParams<SV> &prm, int
         myCov[a] = cover + (int64_t)(myPart[a] < 0 ? parts[0] : myPart[a]) * c.ld;
     }
     unsigned hits = 0;
+    int finished = 0;                                               // row groups of this sweep this warp has completed
     bool preDrawn = firstTicket >= 0;                               // one ticket per warp drawn by the CTA
     for (;;) {
         int g = 0;
@@ -798,18 +803,22 @@ __device__ __noinline__ void sweep_class_sparse(const GreedyParams<SV> &prm, int
                 if (slot == 0 && k0 + r < nR && myPart[a] >= 0) G[(int64_t)myPart[a] * c.ld + __ldcg(cand + k0 + r)] = t;
             }
         }
-        if (done != nullptr) {
-            // the row group's hit count and gains are in place before the group counts as done
+        ++finished;
+    }
+    if (done != nullptr) {
+        // The row groups this warp finished are reported together, once the sweep's tickets have run out for it (the
+        // class's pick CTA only needs the total); their hit count and gains are in place before they count as done.
+        if (finished > 0) {
             __syncwarp();
             if (lane == 0) {
                 if (hits) atomicAdd(&prm.hitCount[l], (unsigned long long)hits);
                 __threadfence();
-                atomicAdd(done, 1);
+                atomicAdd(done, finished);
             }
-            hits = 0;
         }
+    } else if (lane == 0 && hits) {
+        atomicAdd(&prm.hitCount[l], (unsigned long long)hits);
     }
-    if (lane == 0 && hits) atomicAdd(&prm.hitCount[l], (unsigned long long)hits);
 }
 
 // The sweep of greedy step `step`, run by every CTA of the launch (kSweepThreads threads each).
