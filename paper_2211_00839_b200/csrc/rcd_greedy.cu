@@ -675,24 +675,34 @@ __device__ __noinline__ void sweep_class_sparse(const GreedyParams<SV> &prm, int
     }
     unsigned hits = 0;
     int finished = 0;                                               // row groups of this sweep this warp has completed
-    bool preDrawn = firstTicket >= 0;                               // one ticket per warp drawn by the CTA
-    for (;;) {
-        int g = 0;
-        if (preDrawn) {
-            g = firstTicket + (threadIdx.x >> 5);
-            preDrawn = false;
-        } else {
-            if (lane == 0) g = atomicAdd(ticket, 1);
-            g = __shfl_sync(0xffffffffu, g, 0);
+    // The warp's ticket (firstTicket >= 0: one per warp was drawn by the CTA) and the rows it names.  The next
+    // ticket is drawn while the current rows stream, and its row indices are loaded under the drain and the
+    // stores that end a row group, so that neither trip to memory is waited for between two row groups.
+    int g = 0;
+    if (firstTicket >= 0) {
+        g = firstTicket + (threadIdx.x >> 5);
+    } else {
+        if (lane == 0) g = atomicAdd(ticket, 1);
+        g = __shfl_sync(0xffffffffu, g, 0);
+    }
+    int rowOf[R];
+#pragma unroll
+    for (int r = 0; r < R; ++r) rowOf[r] = 0;
+    if (g < nGroups) {
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            const int k = g * R + r;
+            rowOf[r] = __ldcg(cand + (k < nR ? k : nR - 1));
         }
+    }
+    for (;;) {
         if (g >= nGroups) break;
         const int k0 = g * R;
         const int4 *rp[R];
 #pragma unroll
-        for (int r = 0; r < R; ++r) {
-            const int k = k0 + r;
-            rp[r] = reinterpret_cast<const int4 *>(Sl + (int64_t)__ldcg(cand + (k < nR ? k : nR - 1)) * c.ld);
-        }
+        for (int r = 0; r < R; ++r) rp[r] = reinterpret_cast<const int4 *>(Sl + (int64_t)rowOf[r] * c.ld);
+        int gDrawn = 0;
+        if (lane == 0) gDrawn = atomicAdd(ticket, 1);
         GV acc[R][A];                                               // running sums of this lane, [row][block of the lane]
 #pragma unroll
         for (int r = 0; r < R; ++r)
@@ -793,6 +803,17 @@ __device__ __noinline__ void sweep_class_sparse(const GreedyParams<SV> &prm, int
             if (++stage == kSparseStages) stage = 0;
         }
         asm volatile("cp.async.wait_group 0;" ::: "memory");
+        const int gNext = __shfl_sync(0xffffffffu, gDrawn, 0);
+        int rowNext[R];
+#pragma unroll
+        for (int r = 0; r < R; ++r) rowNext[r] = 0;
+        if (gNext < nGroups) {
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                const int k = gNext * R + r;
+                rowNext[r] = __ldcg(cand + (k < nR ? k : nR - 1));
+            }
+        }
         if (qn) { hits += qn; drain(); }
 #pragma unroll
         for (int r = 0; r < R; ++r) {
@@ -800,10 +821,13 @@ __device__ __noinline__ void sweep_class_sparse(const GreedyParams<SV> &prm, int
             for (int a = 0; a < A; ++a) {
                 GV t = acc[r][a];
                 for (int off = Pp; off < 32; off <<= 1) t += __shfl_xor_sync(0xffffffffu, t, off);
-                if (slot == 0 && k0 + r < nR && myPart[a] >= 0) G[(int64_t)myPart[a] * c.ld + __ldcg(cand + k0 + r)] = t;
+                if (slot == 0 && k0 + r < nR && myPart[a] >= 0) G[(int64_t)myPart[a] * c.ld + rowOf[r]] = t;
             }
         }
         ++finished;
+        g = gNext;
+#pragma unroll
+        for (int r = 0; r < R; ++r) rowOf[r] = rowNext[r];
     }
     if (done != nullptr) {
         // The row groups this warp finished are reported together, once the sweep's tickets have run out for it (the
