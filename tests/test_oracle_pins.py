@@ -367,6 +367,83 @@ def test_replay_accepts_own_trace_and_flags_planted_mistakes():
     assert bad != -1
 
 
+def _replay_cases():
+    return json.load(open(os.path.join(GOLDEN, "hand_traces.json")))["replay_cases"]
+
+
+def _check_replay_case(S, q, oj, ov, objective, stats_want, first_failure, fvals):
+    for tol_text, want_bad in first_failure.items():
+        bad, stats, fv = orc.replay_class(S, q, oj, ov, float(tol_text), objective=objective)
+        assert bad == want_bad, (tol_text, bad)
+        # the deviations themselves do not depend on the tolerance, and they are the hand values, not just "small"
+        assert stats[0] == stats_want["block_mismatches"] and stats[1] == stats_want["sample_mismatches"]
+        assert stats[2] == stats_want["block_excess"][0] / stats_want["block_excess"][1]
+        assert stats[3] == stats_want["gain_deficit"][0] / stats_want["gain_deficit"][1]
+        assert fv.tolist() == fvals
+
+
+@pytest.mark.parametrize("as_float", [False, True])
+@pytest.mark.parametrize("case", _replay_cases(), ids=lambda c: c["name"])
+def test_replay_tolerance_hand_worked(case, as_float):
+    """The size of the teacher-forced checker's relative deviations, on pick sequences that deviate from
+    the greedy one by amounts computed by hand (GreedyStep's argmax, Algorithm 1's argmin over blocks):
+    a 5e-4 deficit passes at 1e-3 and fails at 1e-4 at the step that has it, and the reported worst
+    deviations equal the hand values.  A mis-scaled, swapped or wrongly normalised `rel` fails here."""
+    S = np.array(case["S"], dtype=np.float64 if as_float else np.int64)
+    fv = [float(x) for x in case["fvals"]] if as_float else case["fvals"]
+    _check_replay_case(S, case["quotas"], case["order_j"], case["order_v"], case["objective"], case["stats"],
+                       case["first_failure"], fv)
+    if "variant_b" in case:
+        b = case["variant_b"]
+        fvb = [float(x) for x in b["fvals_after"]] if as_float else b["fvals_after"]
+        _check_replay_case(S, case["quotas"], b["order_j"], b["order_v"], case["objective"], b["stats"],
+                           b["first_failure"], fvb)
+
+
+@pytest.mark.parametrize("objective", ["facility", "cut"])
+@pytest.mark.parametrize("seed", range(3))
+def test_replay_rejects_planted_mistakes(objective, seed):
+    """Both checkers against false acceptance: starting from the oracle's own trace of a random class,
+    every planted mistake is reported, at the step it was planted or (for a swap) no later than it."""
+    rng = np.random.default_rng(700 + seed)
+    M = 24
+    S = rand_sym_int(rng, M, -50, 400)
+    if objective == "cut":
+        np.fill_diagonal(S, 0)
+    q = orc.quotas(M, [1, 2, 2, 1])
+    assign, oj, ov, fv = orc.partition_class(S, q, "plain", objective=objective)
+    bad, stats, fv2 = orc.replay_class(S, q, oj, ov, 0.0, objective=objective)
+    assert bad == -1 and stats.tolist() == [0, 0, 0, 0] and np.array_equal(fv, fv2)
+    # exchange two picked samples (different gains): the earlier step is no longer the argmax
+    a, b = 3, 11
+    ov2 = ov.copy()
+    ov2[a], ov2[b] = ov2[b], ov2[a]
+    bad, stats, _ = orc.replay_class(S, q, oj, ov2, 0.0, objective=objective)
+    assert 0 <= bad <= a and stats[1] > 0 and stats[3] > 0
+    assert orc.replay_class(S, q, oj, ov2, 1e9, objective=objective)[0] == -1     # only the tolerance lets it through
+    # a sample picked twice: structural, whatever the tolerance
+    ov3 = ov.copy()
+    ov3[7] = ov3[2]
+    assert orc.replay_class(S, q, oj, ov3, 1e9, objective=objective)[0] == -(7 + 2)
+    # a block other than the argmin at a step where the values differ
+    t = next(k for k in range(4, M) if len(set(oj[:k].tolist())) == 4)
+    oj4 = oj.copy()
+    oj4[t] = (oj4[t] + 1) % 4
+    bad, stats, _ = orc.replay_class(S, q, oj4, ov, 0.0, objective=objective)
+    assert bad in (t, -(t + 2)), (bad, t)         # not the argmin (values differ), or already full
+    # a block beyond its quota: structural
+    full = int(np.argmin(q))
+    t_full = int(np.nonzero(oj == full)[0][-1])
+    later = next(k for k in range(t_full + 1, M))
+    oj5 = oj.copy()
+    oj5[later] = full
+    assert orc.replay_class(S, q, oj5, ov, 1e9, objective=objective)[0] == -(later + 2)
+    # an index out of range
+    ov6 = ov.copy()
+    ov6[5] = M
+    assert orc.replay_class(S, q, oj, ov6, 1e9, objective=objective)[0] == -(5 + 2)
+
+
 # ----------------------------------------------------------------------------- Gaussian-kernel similarity (Section 4 item 2)
 
 def test_gaussian_two_points_closed_form():
