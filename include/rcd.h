@@ -7,7 +7,8 @@
  * Conventions
  *   - "dev" pointers are CUDA device pointers on the context's device; "host"
  *     pointers are ordinary host memory.  The caller owns every buffer,
- *     including the workspace; the library never frees or keeps them.
+ *     including the workspace; the library never frees them and reads nothing of them after the
+ *     call's last kernel (the device-side status of a call is copied into the context).
  *   - `cuda_stream` is a cudaStream_t passed as void* (NULL = default stream).
  *     Unless stated otherwise a call only enqueues work on that stream and
  *     returns; outputs are valid once the stream has been synchronised.
@@ -158,14 +159,15 @@ RCD_API rcd_status rcd_quotas(int64_t M, const double *capacities_host, int32_t 
 
 /* S_b = X_b X_b^T for `batch` classes of equal size.
  *   X_dev  [batch][M][d] row-major, int8 or bf16 (16-byte aligned base)
- *   S_dev  [batch][M][ldS] row-major, int32 (I8) or fp32 (BF16); ldS >= M, ldS % 4 == 0;
+ *   S_dev  [batch][M][ldS] row-major, int32 (I8) or fp32 (BF16); ldS a multiple of 4 with
+ *          M <= ldS <= M rounded up to a multiple of 64 (anything else: RCD_ERR_INVALID_ARG);
  *          columns M..ldS-1 of every row are written as 0.
  * I8 requires 16384*d < 2^31 so that S cannot overflow int32. */
 RCD_API rcd_status rcd_similarity(rcd_ctx *ctx, const void *X_dev, rcd_feat_dtype dtype, int64_t M, int64_t d,
                           int64_t batch, void *S_dev, int64_t ldS, void *cuda_stream);
 
 /* Gaussian-kernel similarity of `batch` equal classes (see rcd_similarity_kind), whatever the context's
- * similarity_kind.  S_dev is fp32 [batch][M][ldS] (ldS = M rounded up to 4, pad columns 0);
+ * similarity_kind.  S_dev is fp32 [batch][M][ldS] (ldS as for rcd_similarity, pad columns 0);
  * sigma_dev_or_null receives the `batch` bandwidths (fp32).  It first forms the dot products like
  * rcd_similarity, then transforms them in place; the workspace holds row norms and partial sums. */
 RCD_API rcd_status rcd_similarity_gaussian_workspace_bytes(rcd_ctx *ctx, int64_t M, int64_t batch, size_t *bytes_out);
@@ -257,9 +259,10 @@ RCD_API rcd_status rcd_batch_sizes(int64_t B, const double *capacities_host, int
 /* The paper has nothing corresponding to this entry point: it exists for callers that cannot
  * allocate device memory (code running inside a fixed, pre-carved memory budget or in a region
  * where touching the CUDA allocator is not allowed) and so cannot supply the workspace that
- * rcd_objective needs.  It computes f(A_j) for the W blocks of ONE class from a similarity
- * matrix the caller already has (for instance from rcd_similarity), using a 1 MiB scratch array
- * that is built into the library instead of a workspace.
+ * rcd_objective needs.  It computes the facility-location value f(A_j) of the W blocks of ONE
+ * class from a similarity matrix the caller already has (for instance from rcd_similarity), using
+ * a 1 MiB scratch array that is built into the library instead of a workspace.  A context whose
+ * objective is RCD_OBJ_GRAPH_CUT is refused (RCD_ERR_UNSUPPORTED), not silently given other values.
  *   S_dev           [M][ldS] row-major, int32 (RCD_FEAT_I8) or fp32 (RCD_FEAT_BF16), ldS >= M
  *   assignment_dev  [M] block of each sample of the class, in [0, W); negative = in no block
  *   part_values_dev [W] int64 / double;  total_dev one int64 / double (their sum)
@@ -268,8 +271,10 @@ RCD_API rcd_status rcd_batch_sizes(int64_t B, const double *capacities_host, int
  * process exits.  All calls on a device share it: calls whose kernels overlap on the GPU race,
  * so keep them on one stream or order them with events.  It keeps the previous call's partial
  * sums; every slot a call reads has been written by that call first, so nothing needs clearing.
- * The first call on each device looks up the array's device address; make that first call
- * outside any stream capture.  No cudaMalloc/cudaFree or allocating routine is called. */
+ * The first call on each device looks up the array's device address (the lookup is serialised
+ * across host threads); make that first call outside any stream capture.  Like every call of this
+ * library it leaves the context's device current.  No cudaMalloc/cudaFree or allocating routine
+ * is called. */
 RCD_API rcd_status rcd_objective_class_static(rcd_ctx *ctx, const void *S_dev, rcd_feat_dtype dtype, int64_t M,
                                       int64_t ldS, const int32_t *assignment_dev, int32_t W,
                                       void *part_values_dev, void *total_dev, void *cuda_stream);

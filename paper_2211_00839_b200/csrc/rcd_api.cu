@@ -30,6 +30,23 @@ rcd_status cuda_fail(rcd_ctx *ctx, cudaError_t e, const char *what)
     return fail(ctx, RCD_ERR_CUDA, "CUDA error %d (%s) in %s", (int)e, cudaGetErrorString(e), what);
 }
 
+// Device-side errors of a call are collected in a status word inside the caller's workspace (the kernels'
+// target, ctx->statusDev) and copied into the context's own word when the call has enqueued its last kernel:
+// rcd_sync_status reads only the context's word, so it never touches a workspace the caller may have freed.
+static cudaError_t status_begin(rcd_ctx *ctx, cudaStream_t st)
+{
+    ctx->statusDev = ctx->statusOwn;
+    return cudaMemsetAsync(ctx->statusOwn, 0, sizeof(int32_t), st);
+}
+static cudaError_t status_publish(rcd_ctx *ctx, cudaStream_t st)
+{
+    cudaError_t e = cudaSuccess;
+    if (ctx->statusDev && ctx->statusDev != ctx->statusOwn)
+        e = cudaMemcpyAsync(ctx->statusOwn, ctx->statusDev, sizeof(int32_t), cudaMemcpyDeviceToDevice, st);
+    ctx->statusDev = ctx->statusOwn;
+    return e;
+}
+
 // Bump allocator over the caller's workspace.
 struct Carver {
     unsigned char *base;
@@ -90,6 +107,7 @@ size_t layout_workspace(void *base, rcd_feat_dtype dtype, const Sizes &sz, Works
     w.sync = c.take<ClassSync>(L);
     w.tickets = c.take<int32_t>(N + L);
     w.sweepF = c.take<long long>(L * 8);
+    w.sizesSorted = c.take<int32_t>(L);
     w.stepBytes = c.take<unsigned long long>((size_t)sz.maxM + 1);
     w.stepOps = c.take<unsigned long long>((size_t)sz.maxM + 1);
     w.phaseNs = c.take<unsigned long long>(8);      // two phase clocks, the grid-barrier counter, threshold-pass hits / elements
@@ -344,9 +362,8 @@ rcd_status rcd_sync_status(rcd_ctx *ctx, void *cuda_stream)
     if (!ctx) return RCD_ERR_INVALID_ARG;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     RCD_CUDA(ctx, cudaStreamSynchronize(st));
-    if (!ctx->statusDev) return RCD_OK;
     int32_t word = 0;
-    RCD_CUDA(ctx, cudaMemcpy(&word, ctx->statusDev, sizeof word, cudaMemcpyDeviceToHost));
+    RCD_CUDA(ctx, cudaMemcpy(&word, ctx->statusOwn, sizeof word, cudaMemcpyDeviceToHost));
     if (word == 0) return RCD_OK;
     if (word & kDevBadLabel) return fail(ctx, RCD_ERR_INVALID_ARG, "device status %d: label out of range", word);
     if (word & kDevTimeout) return fail(ctx, RCD_ERR_TIMEOUT, "device status %d: a bounded wait inside a kernel ran out", word);
@@ -462,6 +479,7 @@ rcd_status rcd_worker_lists(rcd_ctx *ctx, const int32_t *assignment_dev, int64_t
     cudaStream_t st = (cudaStream_t)cuda_stream;
     RCD_CUDA(ctx, cudaSetDevice(ctx->device));
     ctx->kernelLaunches = 0;
+    RCD_CUDA(ctx, status_begin(ctx, st));
     ctx->statusDev = ws.status;
     RCD_CUDA(ctx, cudaMemsetAsync(ws.status, 0, 4 * sizeof(int32_t), st));
     RCD_CUDA(ctx, cudaMemsetAsync(ws.counts, 0, (size_t)W * sizeof(int32_t), st));
@@ -489,7 +507,10 @@ rcd_status rcd_worker_lists(rcd_ctx *ctx, const int32_t *assignment_dev, int64_t
     RCD_CUDA(ctx, cudaMemcpyAsync(offsets_dev, offsets.data(), offsets.size() * sizeof(int64_t), cudaMemcpyHostToDevice, st));
     RCD_CUDA(ctx, cudaMemcpyAsync(ws.desc, desc.data(), desc.size() * sizeof(ClassDesc), cudaMemcpyHostToDevice, st));
     // a stable split by block number: inside a list the dataset indices ascend
-    return launch_stable_split(ctx, assignment_dev, N, W, chunks_for(N), ws.chunkHist, ws.desc, indices_dev, st);
+    rs = launch_stable_split(ctx, assignment_dev, N, W, chunks_for(N), ws.chunkHist, ws.desc, indices_dev, st);
+    if (rs != RCD_OK) return rs;
+    RCD_CUDA(ctx, status_publish(ctx, st));
+    return RCD_OK;
 }
 
 rcd_status rcd_batch_sizes(int64_t B, const double *capacities_host, int32_t W, int64_t *batch_sizes_host_out)
@@ -514,7 +535,9 @@ rcd_status rcd_similarity(rcd_ctx *ctx, const void *X_dev, rcd_feat_dtype dtype,
     if (M < 0 || batch < 0 || M > 0x7fffffffLL) return fail(ctx, RCD_ERR_INVALID_ARG, "M or batch negative");
     if (M == 0 || batch == 0) return RCD_OK;
     if (!X_dev || !S_dev) return fail(ctx, RCD_ERR_INVALID_ARG, "null device pointer");
-    if (ldS != pad4(M)) return fail(ctx, RCD_ERR_INVALID_ARG, "ldS must be M rounded up to a multiple of 4 (%d), got %lld", pad4(M), (long long)ldS);
+    if (ldS % 4 != 0 || ldS < M || ldS > (M + 63) / 64 * 64)
+        return fail(ctx, RCD_ERR_INVALID_ARG, "ldS must be a multiple of 4 in [M, M rounded up to 64] = [%lld, %lld], got %lld",
+                    (long long)M, (long long)((M + 63) / 64 * 64), (long long)ldS);
     if (M * batch > 0x7fffffffLL) return fail(ctx, RCD_ERR_INVALID_ARG, "M*batch too large");
     if (((uintptr_t)X_dev) % 16 || ((uintptr_t)S_dev) % 16) return fail(ctx, RCD_ERR_INVALID_ARG, "X and S must be 16-byte aligned");
     cudaStream_t st = (cudaStream_t)cuda_stream;
@@ -530,8 +553,7 @@ rcd_status rcd_similarity(rcd_ctx *ctx, const void *X_dev, rcd_feat_dtype dtype,
     cls.upperTiles = batch * (int64_t)cls.uniTiles;
     ctx->kernelLaunches = 0;
     ctx->tcLaunches = 0;
-    ctx->statusDev = ctx->statusOwn;
-    RCD_CUDA(ctx, cudaMemsetAsync(ctx->statusOwn, 0, sizeof(int32_t), st));
+    RCD_CUDA(ctx, status_begin(ctx, st));
     return launch_similarity(ctx, X_dev, dtype, M * batch, d, cls, S_dev, st);
 }
 
@@ -548,13 +570,18 @@ rcd_status rcd_similarity_gaussian(rcd_ctx *ctx, const void *X_dev, rcd_feat_dty
                                    void *S_dev, int64_t ldS, float *sigma_dev_or_null, void *workspace_dev,
                                    size_t workspace_bytes, void *cuda_stream)
 {
+    if (!ctx) return RCD_ERR_INVALID_ARG;
+    // every argument is checked before anything is launched or written
+    if (M > 0 && batch > 0) {
+        if (batch > 65535) return fail(ctx, RCD_ERR_UNSUPPORTED, "Gaussian similarity: more than 65535 classes");
+        if (M * batch > 0x7fffffffLL) return fail(ctx, RCD_ERR_INVALID_ARG, "M*batch too large");
+        if (!workspace_dev || ((uintptr_t)workspace_dev) % kAlign) return fail(ctx, RCD_ERR_INVALID_ARG, "workspace null or not 256-byte aligned");
+        if (workspace_bytes < gaussian_scratch_bytes(M * batch, (int32_t)batch, M))
+            return fail(ctx, RCD_ERR_WORKSPACE_TOO_SMALL, "workspace has %zu bytes, need %zu", workspace_bytes,
+                        gaussian_scratch_bytes(M * batch, (int32_t)batch, M));
+    }
     rcd_status rs = rcd_similarity(ctx, X_dev, dtype, M, d, batch, S_dev, ldS, cuda_stream);
     if (rs != RCD_OK || M == 0 || batch == 0) return rs;
-    if (batch > 65535) return fail(ctx, RCD_ERR_UNSUPPORTED, "Gaussian similarity: more than 65535 classes");
-    if (!workspace_dev || ((uintptr_t)workspace_dev) % kAlign) return fail(ctx, RCD_ERR_INVALID_ARG, "workspace null or not 256-byte aligned");
-    if (workspace_bytes < gaussian_scratch_bytes(M * batch, (int32_t)batch, M))
-        return fail(ctx, RCD_ERR_WORKSPACE_TOO_SMALL, "workspace has %zu bytes, need %zu", workspace_bytes,
-                    gaussian_scratch_bytes(M * batch, (int32_t)batch, M));
     cudaStream_t st = (cudaStream_t)cuda_stream;
     unsigned char *w = (unsigned char *)workspace_dev;
     void *norms = w;                                  w += align_up((size_t)(M * batch) * 4);
@@ -607,6 +634,7 @@ rcd_status rcd_partition(rcd_ctx *ctx, const void *features_dev, rcd_feat_dtype 
     ctx->phaseNsDev = nullptr;
     ctx->sweepEventsUsed = 0;
     const bool prof = ctx->cfg.profile >= 1;
+    RCD_CUDA(ctx, status_begin(ctx, st));
     if (prof) RCD_CUDA(ctx, cudaEventRecord(ctx->evPhase[0], st));
 
     Prepared P;
@@ -625,6 +653,7 @@ rcd_status rcd_partition(rcd_ctx *ctx, const void *features_dev, rcd_feat_dtype 
         if (P.sz.maxM == 0) RCD_CUDA(ctx, cudaMemsetAsync(part_values_dev_or_null, 0, (size_t)L * W * 8, st));
         else RCD_CUDA(ctx, cudaMemcpyAsync(part_values_dev_or_null, P.ws.fval, (size_t)L * W * 8, cudaMemcpyDeviceToDevice, st));
     }
+    RCD_CUDA(ctx, status_publish(ctx, st));
     if (prof) {
         RCD_CUDA(ctx, cudaEventRecord(ctx->evPhase[4], st));
         ctx->phaseValid = true;
@@ -725,6 +754,7 @@ rcd_status rcd_objective(rcd_ctx *ctx, const void *features_dev, rcd_feat_dtype 
     if (!workspace_dev) return fail(ctx, RCD_ERR_INVALID_ARG, "workspace is null");
     cudaStream_t st = (cudaStream_t)cuda_stream;
     RCD_CUDA(ctx, cudaSetDevice(ctx->device));
+    RCD_CUDA(ctx, status_begin(ctx, st));
     const int savedProfile = ctx->cfg.profile;
     ctx->cfg.profile = 0;
     Prepared P;
@@ -736,9 +766,13 @@ rcd_status rcd_objective(rcd_ctx *ctx, const void *features_dev, rcd_feat_dtype 
         return fail(ctx, RCD_ERR_WORKSPACE_TOO_SMALL, "workspace has %zu bytes, objective needs %zu", workspace_bytes, P.ws.bytes + scratchB);
     void *scratch = (unsigned char *)workspace_dev + P.ws.bytes;
     if (P.sz.graphCut)
-        return launch_cut_objective(ctx, P.sz, P.ws.desc, P.ws.S, P.ws.perm, assignment_dev, part_values_dev, total_dev, scratch, st);
-    return launch_objective(ctx, P.sz.floatArith ? RCD_FEAT_BF16 : RCD_FEAT_I8, P.sz, P.ws.desc, P.desc, P.ws.S, P.ws.perm, assignment_dev, part_values_dev,
-                            total_dev, scratch, st);
+        rs = launch_cut_objective(ctx, P.sz, P.ws.desc, P.ws.S, P.ws.perm, assignment_dev, part_values_dev, total_dev, scratch, st);
+    else
+        rs = launch_objective(ctx, P.sz.floatArith ? RCD_FEAT_BF16 : RCD_FEAT_I8, P.sz, P.ws.desc, P.desc, P.ws.S, P.ws.perm, assignment_dev,
+                              part_values_dev, total_dev, scratch, st);
+    if (rs != RCD_OK) return rs;
+    RCD_CUDA(ctx, status_publish(ctx, st));
+    return RCD_OK;
 }
 
 }  // extern "C"

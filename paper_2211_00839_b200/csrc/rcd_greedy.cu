@@ -24,6 +24,7 @@
 #include "rcd_internal.h"
 
 #include <limits.h>
+#include <algorithm>
 #include <type_traits>
 
 namespace rcd {
@@ -93,6 +94,9 @@ struct GreedyParams {
     int32_t nPick;              // CTAs [0, nPick) make picks, the others sweep
     int32_t helpMin;            // row groups a sweep must have left for a sweep CTA that is not at home there
     int32_t asyncGroup;         // sweeps published one after another that are served together (by CTA home position)
+    const int32_t *sizesSorted; // [L] class sizes in ascending order
+    int32_t minM;               // smallest non-empty class
+    int32_t nonEmpty;           // classes that hold at least one sample
 };
 
 __host__ __device__ inline int rows_per_group(int P) { return P == 8 ? 4 : 8; }
@@ -144,8 +148,10 @@ __host__ __device__ inline int thr_bytes_aligned(int bytes) { return (bytes + 12
 static_assert(kSparseWarpBytes % 128 == 0, "per-warp rings must keep the 128-byte alignment");
 
 // What plan_decide reads from global memory when it has to schedule a sweep.  A chain of picks schedules
-// at most one (its last pick), and nothing here changes during the chain, so the chain loads it at its
-// start, under the first argmax, instead of waiting for it at the end.
+// at most one (its last pick), so the chain loads these at its start, under the first argmax, instead of
+// waiting for them at the end.  `remaining` is decremented by other classes' chains at any time: it may only
+// steer decisions that cannot change a result (the integer path, where every sum is exact); the
+// floating-point path, whose sums depend on how a pass splits its columns, uses classes_alongside().
 struct PlanGlobals {
     int32_t remaining;              // unfinished classes
     int32_t from;                   // sparseFrom[l]
@@ -161,6 +167,21 @@ __device__ __forceinline__ PlanGlobals plan_globals(const GreedyParams<SV> &prm,
     g.elems = *(volatile unsigned long long *)&prm.sparseElems[l];
     g.hits = *(volatile unsigned long long *)&prm.hitCount[l];
     return g;
+}
+
+// How many classes are taken to be still unfinished when a class has made `made` picks: those larger than
+// `made` samples.  A function of the class's own progress and of the class sizes only, so that the shape of a
+// floating-point sweep (dense or threshold pass, warps per row group: they fix the order of its additions)
+// never depends on the timing of other classes.  Whole warp; the same value in every lane.
+template <typename SV>
+__device__ __forceinline__ int classes_alongside(const GreedyParams<SV> &prm, int made)
+{
+    if (made < prm.minM) return prm.nonEmpty;
+    const int lane = threadIdx.x & 31;
+    int n = 0;
+    for (int i = lane; i < prm.L; i += 32) n += __ldg(prm.sizesSorted + i) > made ? 1 : 0;
+    for (int off = 16; off > 0; off >>= 1) n += __shfl_xor_sync(0xffffffffu, n, off);
+    return n;
 }
 
 template <typename SV>
@@ -227,7 +248,8 @@ __device__ void plan_decide(const GreedyParams<SV> &prm, int l, const ClassDesc 
     PlanGlobals g;
     if (pre) g = *pre;
     else g = plan_globals(prm, l);
-    const int remaining = g.remaining;
+    int remaining = g.remaining;
+    if constexpr (!Arith<SV>::kInt) remaining = classes_alongside(prm, c.M - nR);
     int from = 0;
     if (lane == 0) {
         from = g.from;
@@ -1630,6 +1652,21 @@ static rcd_status run_greedy(rcd_ctx *ctx, const Sizes &sz, const Workspace &ws,
     prm.nPick = 0;
     prm.asyncGroup = 1;
     prm.helpMin = 1;
+    {
+        std::vector<int32_t> sorted;
+        sorted.reserve(descHost.size());
+        for (const auto &c : descHost) sorted.push_back(c.M);
+        std::sort(sorted.begin(), sorted.end());
+        prm.sizesSorted = ws.sizesSorted;
+        prm.nonEmpty = 0;
+        prm.minM = 0;
+        for (int32_t m : sorted) {
+            if (m <= 0) continue;
+            if (prm.nonEmpty == 0) prm.minM = m;
+            ++prm.nonEmpty;
+        }
+        RCD_CUDA(ctx, cudaMemcpyAsync(ws.sizesSorted, sorted.data(), sorted.size() * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+    }
     int maxLd = 0;
     for (const auto &c : descHost) if (c.ld > maxLd) maxLd = c.ld;
     const int64_t smemCap = (int64_t)ctx->maxSmemOptin - 24 * 1024;  // static shared of the kernels + margin

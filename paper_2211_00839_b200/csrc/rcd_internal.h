@@ -113,6 +113,7 @@ struct Workspace {
     int32_t *rowCtr;        // [L] ticket counter over row groups of the running sweep
     ClassSync *sync;        // [L] asynchronous kernel: hand-off words
     int32_t *tickets;       // [N + L] asynchronous kernel: one ticket counter per (class, sweep number), never reused
+    int32_t *sizesSorted;   // [L] class sizes, ascending
     long long *sweepF;      // [L][8] asynchronous kernel, int8 features: f of the first blocks in the sweep's list
     int32_t *sweepList;     // [3][L] classes that sweep in a step (three lists in rotation)
     int32_t *nSweep;        // [3] (+1 pad)

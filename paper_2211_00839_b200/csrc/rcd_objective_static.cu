@@ -18,6 +18,7 @@
 //     make that first call outside any stream capture.
 #include "rcd_internal.h"
 
+#include <mutex>
 #include <type_traits>
 
 namespace rcd {
@@ -31,12 +32,16 @@ constexpr int kMaxDevices = 64;
 // kernel could use; the address comes from cudaGetSymbolAddress below.
 static __device__ __align__(256) unsigned char g_objectiveScratch[kStaticScratchBytes];
 
+// One address per device, looked up once; the table is shared by every context of the process, so the
+// lookup is serialised (two contexts on two host threads may make their first call at the same time).
 static void *g_scratchAddr[kMaxDevices] = {};
+static std::mutex g_scratchLock;
 
 static rcd_status static_scratch(rcd_ctx *ctx, void **out)
 {
     if (ctx->device < 0 || ctx->device >= kMaxDevices)
         return fail(ctx, RCD_ERR_UNSUPPORTED, "device index %d beyond the %d devices this entry point tracks", ctx->device, kMaxDevices);
+    std::lock_guard<std::mutex> guard(g_scratchLock);
     if (!g_scratchAddr[ctx->device]) {
         void *p = nullptr;
         RCD_CUDA(ctx, cudaSetDevice(ctx->device));
@@ -144,6 +149,8 @@ extern "C" rcd_status rcd_objective_class_static(rcd_ctx *ctx, const void *S_dev
 {
     if (!ctx) return RCD_ERR_INVALID_ARG;
     if (dtype != RCD_FEAT_I8 && dtype != RCD_FEAT_BF16) return fail(ctx, RCD_ERR_INVALID_ARG, "unknown dtype %d", (int)dtype);
+    if (ctx->cfg.objective != RCD_OBJ_FACILITY)
+        return fail(ctx, RCD_ERR_UNSUPPORTED, "rcd_objective_class_static evaluates facility location only; this context is set to another objective");
     if (M < 0 || W <= 0 || ldS < M) return fail(ctx, RCD_ERR_INVALID_ARG, "need M >= 0, W > 0, ldS >= M");
     if (!part_values_dev || !total_dev || (M > 0 && (!S_dev || !assignment_dev)))
         return fail(ctx, RCD_ERR_INVALID_ARG, "null device pointer");

@@ -6,10 +6,26 @@ equal the oracle's run of that class alone), a replayed prefix and single late p
 not; plus properties that hold at any size (exact quotas, disjoint cover, tracked f equal to f
 recomputed from the final assignment).
 """
+import importlib.util
+import json
+import os
+from concurrent.futures import ThreadPoolExecutor
+
 import numpy as np
 import pytest
 
 pytestmark = pytest.mark.gpu
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _golden_module():
+    """The script that wrote tests/golden/fullsize_digests.json (from the oracle alone); its digest
+    functions are reused so that both sides hash the same bytes."""
+    spec = importlib.util.spec_from_file_location("make_fullsize_golden", os.path.join(GOLDEN, "make_fullsize_golden.py"))
+    mod = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(mod)
+    return mod
 
 OBJ_RTOL = 1e-4
 PICK_RTOL = 1e-3
@@ -139,3 +155,73 @@ def test_c5_many_classes_int8(rcd, orc):
         assert np.array_equal(a[ids], assign)
         assert np.array_equal(o[l * M:(l + 1) * M], ids[ov])
         assert np.array_equal(v[l], fv)
+
+
+# ----------------------------------------------------------------------------- whole trajectories at full size
+
+def _check_against_digests(rcd, orc, name):
+    """Every class of a full-size int8 configuration, bit for bit: block of every sample, pick order and
+    block values must hash to the digest the oracle's own run of that class produced (stored under
+    tests/golden by a script that calls only the oracle)."""
+    from paper_2211_00839_b200.workloads import make_workload
+    gm = _golden_module()
+    gold = json.load(open(os.path.join(GOLDEN, "fullsize_digests.json")))[name]
+    wl = make_workload(name)
+    assert gm.input_digest(wl) == gold["inputs"], "the generator no longer produces the inputs the digests were written for"
+    a, o, v, recomputed = run_full(rcd, wl)
+    groups = check_invariants(orc, wl, a, o)
+    assert np.array_equal(v, recomputed)
+    assert int(v.sum()) == gold["total_objective"]
+    bad = []
+    off = 0
+    for l, ids in enumerate(groups):
+        picked = o[off:off + len(ids)]
+        off += len(ids)
+        local = np.searchsorted(ids, picked).astype(np.int32)
+        if gm.class_digest(a[ids], local, v[l]) != gold["class_digests"][l]:
+            bad.append(l)
+    if bad:                                                           # show where the first bad class leaves the oracle's path
+        l = bad[0]
+        ids = groups[l]
+        S = orc.similarity(wl.features[ids])
+        assign, oj, ov, fv = orc.partition_class(S, orc.quotas(len(ids), wl.capacities), "incremental")
+        start = int(sum(len(g) for g in groups[:l]))
+        local = np.searchsorted(ids, o[start:start + len(ids)])
+        first = int(np.argmax(local != ov)) if np.any(local != ov) else -1
+        pytest.fail("%s: %d classes differ from the oracle (first: class %d, first differing pick %d)" % (name, len(bad), l, first))
+
+
+def test_c2_every_class_bit_exact(rcd, orc):
+    """All 10 classes of C2 (5000 picks each) in the configuration bench.py times."""
+    _check_against_digests(rcd, orc, "C2")
+
+
+def test_c5_every_class_bit_exact(rcd, orc):
+    """All 1000 classes of C5 (1300 picks each)."""
+    _check_against_digests(rcd, orc, "C5")
+
+
+def test_c3_whole_classes_teacher_forced(rcd, orc):
+    """Two whole classes of full-size C3 (5000 picks each, every one of them) replayed by the oracle in double:
+    each pick's block within 1e-3 of the least value and its sample within 1e-3 of the best gain, tracked
+    values within 1e-4 of the replayed ones.  The two replays run in two threads (the oracle is plain C)."""
+    from paper_2211_00839_b200.workloads import make_workload
+    wl = make_workload("C3")
+    a, o, v, recomputed = run_full(rcd, wl)
+    groups = check_invariants(orc, wl, a, o)
+    M = wl.N // wl.L
+
+    def replay(l):
+        ids = groups[l]
+        S = orc.similarity(wl.features[ids])
+        q = orc.quotas(M, wl.capacities)
+        picked = o[l * M:(l + 1) * M]
+        local = np.searchsorted(ids, picked).astype(np.int32)
+        return l, orc.replay_class(S, q, a[picked], local, PICK_RTOL)
+
+    with ThreadPoolExecutor(max_workers=2) as ex:
+        for l, (bad, stats, fv) in ex.map(replay, (2, 7)):
+            print("C3 class %d: %d picks replayed, block mismatches %d (worst excess %.3g), sample mismatches %d (worst deficit %.3g)"
+                  % (l, M, stats[0], stats[2], stats[1], stats[3]))
+            assert bad == -1, (l, bad, stats)
+            assert np.allclose(v[l], fv, rtol=OBJ_RTOL, atol=1e-9)

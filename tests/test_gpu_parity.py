@@ -11,6 +11,7 @@ pytestmark = pytest.mark.gpu
 
 OBJ_RTOL = 1e-4      # final objective, float configs
 PICK_RTOL = 1e-3     # a pick may differ from the oracle's only inside this relative gap
+FREE_RUN_BRANCH_RTOL = 1e-4   # totals of two runs that took different branches at a near-tie (see check_float)
 
 
 @pytest.fixture(scope="module")
@@ -180,6 +181,49 @@ def test_partition_is_reproducible(rcd):
         assert np.array_equal(x, y)
 
 
+def ragged_float_workload(sizes, d, W, seed):
+    from paper_2211_00839_b200.workloads import Workload, make_mixture, fp32_to_bf16_bits
+    rng = np.random.default_rng(seed)
+    feats, labels = [], []
+    for l, M in enumerate(sizes):
+        x = make_mixture(rng, M, d, 4, "dirichlet", "gauss", 4.0) if M else np.zeros((0, d), np.float32)
+        x = x / np.maximum(np.linalg.norm(x, axis=1, keepdims=True), 1e-30)
+        feats.append(fp32_to_bf16_bits(x.astype(np.float32)))
+        labels.append(np.full(M, l, np.int32))
+    feats = np.concatenate(feats)
+    labels = np.concatenate(labels)
+    perm = rng.permutation(len(labels))
+    caps = rng.uniform(1.0, 4.0, size=W)
+    return Workload("ragged-float", "bf16", np.ascontiguousarray(feats[perm]), np.ascontiguousarray(labels[perm]), caps,
+                    len(sizes), W)
+
+
+@pytest.mark.parametrize("path", [2, 3])
+def test_float_partition_is_reproducible_with_ragged_classes(rcd, path):
+    """fp32 gains depend on how a pass splits its columns, so the shape of a class's sweeps must not depend on
+    when OTHER classes finish: classes of very unequal sizes (the small ones finish while the large ones
+    run), both one-launch forms of the loop, several runs, bit-identical outputs."""
+    wl = ragged_float_workload([1500, 40, 700, 9, 260, 1100, 130], d=128, W=12, seed=91)
+    first = run_partition(rcd, wl, greedy_path=path)
+    for _ in range(4):
+        again = run_partition(rcd, wl, greedy_path=path)
+        for x, y in zip(first, again):
+            assert np.array_equal(x, y)
+
+
+@pytest.mark.parametrize("name,kw,W", [("C2", dict(L=3, M=1003), 7), ("C1", {}, 3)])
+def test_equal_capacities_is_the_label_balanced_partition(rcd, orc, name, kw, W):
+    """Algorithm 3 (all ratios equal): block sizes inside a class differ by at most one, and the result is the
+    oracle's, bit for bit."""
+    from paper_2211_00839_b200.workloads import Workload, make_workload
+    base = make_workload(name, **kw)
+    wl = Workload("equal", base.dtype, base.features, base.labels, np.full(W, 2.5), base.L, W)
+    a, o, v, ref = check_exact(rcd, orc, wl)
+    for l in range(wl.L):
+        sizes = np.bincount(a[wl.labels == l], minlength=W)
+        assert sizes.max() - sizes.min() <= 1 and sizes.sum() == np.count_nonzero(wl.labels == l)
+
+
 # ----------------------------------------------------------------------------- partition, bf16: tolerance rule
 
 def check_float(rcd, orc, wl, **cfg):
@@ -187,6 +231,7 @@ def check_float(rcd, orc, wl, **cfg):
     free = orc.partition(wl.features, wl.labels, wl.capacities, wl.L, variant="incremental")
     groups = orc.split_by_label(wl.labels, wl.L)
     total_replayed = 0.0
+    same_everywhere = True
     for l, ids in enumerate(groups):
         M = len(ids)
         if M == 0:
@@ -207,11 +252,19 @@ def check_float(rcd, orc, wl, **cfg):
         ref_picked = free.order[off:off + M]
         same = (picked == ref_picked) & (a[picked] == free.order_block[off:off + M])
         if not same.all():
+            same_everywhere = False
             first = int(np.argmin(same))
             bad0, stats0, _ = orc.replay_class(S, q, a[picked][:first + 1], local[:first + 1], 0.0)
             assert bad0 == first and max(stats0[2], stats0[3]) <= PICK_RTOL
     assert abs(v.sum() - total_replayed) <= OBJ_RTOL * abs(total_replayed)
-    assert abs(v.sum() - free.total) <= 5e-3 * abs(free.total)     # different near-tie branches stay close
+    # The free-running oracle: while every pick is the same, its total must agree to OBJ_RTOL as well.  Once a
+    # pick inside the 1e-3 gap has gone the other way the two runs are different (both valid) trajectories; on the
+    # synthetic workloads their totals still agree to OBJ_RTOL (measured: below 1e-6), which is what is asserted.
+    free_dev = abs(v.sum() - free.total) / abs(free.total)
+    print("free-run deviation %.3g (%s), replayed deviation %.3g" % (
+        free_dev, "same picks" if same_everywhere else "a near-tie went the other way",
+        abs(v.sum() - total_replayed) / abs(total_replayed)))
+    assert free_dev <= (OBJ_RTOL if same_everywhere else FREE_RUN_BRANCH_RTOL)
     return a, o, v
 
 

@@ -15,11 +15,12 @@ import pytest
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("name,M,d,W", [("C2", 700, 128, 8), ("C4", 450, 96, 32)])
+@pytest.mark.parametrize("name,M,d,W", [("C2", 700, 128, 8), ("C4", 450, 96, 32), ("C5", 300, 128, 64)])
 def test_static_scratch_objective_matches_workspace_objective_twice(name, M, d, W):
     import torch
     from paper_2211_00839_b200 import binding as rcd
     from paper_2211_00839_b200.workloads import make_workload
+    from oracle import rcd_oracle as orc
 
     dev = torch.device("cuda", 0)
     with rcd.Context(0) as ctx:
@@ -36,12 +37,71 @@ def test_static_scratch_objective_matches_workspace_objective_twice(name, M, d, 
             total = torch.full((1,), -7, dtype=vdt, device=dev)
             rcd.rcd_objective_class_static(ctx, S, assignment, W, vals, total)
             ctx.sync_status()
+            # ... and the oracle's plain definition of f on the same class
+            So = orc.similarity(wl.features)
+            a_host = assignment.cpu().numpy()
+            plain = np.array([orc.f_plain(So, np.nonzero(a_host == j)[0]) for j in range(W)])
             if wl.dtype == "int8":
                 assert torch.equal(vals, want_vals[0]), "call %d" % call
                 assert int(total[0]) == int(want_total[0])
+                assert np.array_equal(vals.cpu().numpy(), plain)
             else:
                 assert torch.allclose(vals, want_vals[0], rtol=1e-5, atol=1e-7), "call %d" % call
                 assert float(total[0]) == pytest.approx(float(want_total[0]), rel=1e-5)
+                assert np.allclose(vals.cpu().numpy(), plain, rtol=1e-5, atol=1e-7)
+
+
+def test_static_scratch_at_its_size_limit():
+    """ceil(M/64) * W * 8 exactly 1 MiB is served (and equals the plain definition); one row block more is refused."""
+    import ctypes as C
+    import torch
+    from paper_2211_00839_b200 import binding as rcd
+    from oracle import rcd_oracle as orc
+    dev = torch.device("cuda", 0)
+    W = 1024
+    M = 64 * 128                                     # 128 row blocks * 1024 * 8 bytes = 1 MiB
+    rng = np.random.default_rng(31)
+    d = 16
+    X = rng.integers(-20, 21, size=(M, d)).astype(np.int8)
+    a_host = rng.integers(-1, W, size=M).astype(np.int32)
+    with rcd.Context(0) as ctx:
+        S = ctx.rcd_similarity(torch.from_numpy(X).to(dev))[0]
+        a = torch.from_numpy(a_host).to(dev)
+        vals = torch.full((W,), -7, dtype=torch.int64, device=dev)
+        total = torch.full((1,), -7, dtype=torch.int64, device=dev)
+        rcd.rcd_objective_class_static(ctx, S, a, W, vals, total)
+        ctx.sync_status()
+        So = orc.similarity(X)
+        # plain definition, vectorised per block: sum over rows of the clamped maximum over the block's members
+        want = np.zeros(W, dtype=np.int64)
+        for j in range(W):
+            mem = np.nonzero(a_host == j)[0]
+            if len(mem):
+                want[j] = np.maximum(So[:, mem].max(axis=1), 0).sum()
+        for j in (0, 1, 511, 1023):
+            assert want[j] == orc.f_plain(So, np.nonzero(a_host == j)[0])
+        assert np.array_equal(vals.cpu().numpy(), want) and int(total[0]) == int(want.sum())
+        Mbig = M + 1                                 # one more row block: 129 * 1024 * 8 > 1 MiB
+        st = rcd.lib.rcd_objective_class_static(ctx._h, C.c_void_p(S.data_ptr()), rcd.RCD_FEAT_I8, Mbig, Mbig,
+                                                C.c_void_p(a.data_ptr()), W, C.c_void_p(vals.data_ptr()),
+                                                C.c_void_p(total.data_ptr()), None)
+        assert st == 2
+
+
+def test_static_scratch_refuses_a_graph_cut_context():
+    import ctypes as C
+    import torch
+    from paper_2211_00839_b200 import binding as rcd
+    dev = torch.device("cuda", 0)
+    with rcd.Context(0, objective=rcd.RCD_OBJ_GRAPH_CUT) as ctx:
+        S = torch.zeros((8, 8), dtype=torch.int32, device=dev)
+        a = torch.zeros(8, dtype=torch.int32, device=dev)
+        vals = torch.zeros(2, dtype=torch.int64, device=dev)
+        total = torch.zeros(1, dtype=torch.int64, device=dev)
+        st = rcd.lib.rcd_objective_class_static(ctx._h, C.c_void_p(S.data_ptr()), rcd.RCD_FEAT_I8, 8, 8,
+                                                C.c_void_p(a.data_ptr()), 2, C.c_void_p(vals.data_ptr()),
+                                                C.c_void_p(total.data_ptr()), None)
+        assert st == 2 and b"facility" in rcd.lib.rcd_last_error(ctx._h)
 
 
 def test_static_scratch_rejects_sizes_beyond_its_array():
