@@ -94,6 +94,40 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
+def measure_yardsticks(rcd, ctx, dev, dtype_code):
+    """Times the library's own yardstick kernels with CUDA events: L2-resident and HBM read sweeps (GB/s) and the
+    tensor-core peak loop for the feature dtype (TFLOP/s or TOP/s).  Best of three after one warm-up each."""
+    import torch
+    out = {}
+    l2 = int(torch.cuda.get_device_properties(dev).L2_cache_size)
+
+    def best_of(fn, reps=3):
+        fn()
+        torch.cuda.synchronize(dev)
+        best = None
+        for _ in range(reps):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            work = fn()
+            e1.record()
+            torch.cuda.synchronize(dev)
+            ms = e0.elapsed_time(e1)
+            rate = work / (ms * 1e-3)
+            best = rate if best is None or rate > best else best
+        return best
+
+    small = torch.empty(l2 // 2, dtype=torch.uint8, device=dev).fill_(1)
+    out["l2_read_gbs"] = best_of(lambda: rcd.rcd_yardstick_read(ctx, small, repeats=300)) / 1e9
+    out["l2_read_buffer_mb"] = small.numel() / 1e6
+    big = torch.empty(4 << 30, dtype=torch.uint8, device=dev).fill_(1)
+    out["hbm_read_gbs"] = best_of(lambda: rcd.rcd_yardstick_read(ctx, big, repeats=1)) / 1e9
+    del small, big
+    out["mma_tflops"] = best_of(lambda: rcd.rcd_yardstick_mma(ctx, dtype_code, 20000)) / 1e12
+    ctx.sync_status()
+    out["mma_dtype"] = "int8" if dtype_code == rcd.RCD_FEAT_I8 else "bf16"
+    return out
+
+
 def oracle_sample(wl, picks: int, threads: int):
     """Times the CPU oracle on a bounded sample: `threads` classes, one per thread, similarity in
     full and the first `picks` picks of Algorithm 1; the oracle's cost per pick is constant (it
@@ -173,15 +207,18 @@ def run_ours(args):
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
 
-    # weak scaling: every rank partitions its own dataset of the same shape (seed differs per rank)
-    wl = make_workload(args.config, L=args.classes or None, seed=CONFIGS[args.config]["seed"] + 1000 * rank)
+    # replicas (default; weak scaling): every rank partitions its own dataset of the same shape (seed differs per rank).
+    # --sharding classes (strong scaling): ONE dataset, its classes sharded over the ranks by M^3, one all-gather of
+    # the assignment at the end of every step.
+    by_classes = args.sharding == "classes"
+    wl = make_workload(args.config, L=args.classes or None, seed=CONFIGS[args.config]["seed"] + (0 if by_classes else 1000 * rank))
     M = wl.N // wl.L
     Xh = rcd.features_to_torch(wl.features, pin=True)
     yh = torch.from_numpy(wl.labels).pin_memory()
     Xd, yd = Xh.to(dev), yh.to(dev)
     kind = rcd.RCD_SIM_GAUSSIAN if args.similarity == "gaussian" else rcd.RCD_SIM_DOT
     ctx = rcd.Context(local, sweep_batch_max=args.sweep_batch, profile=1, greedy_path=args.greedy_path, similarity_kind=kind,
-                      async_group=args.async_group, async_help_min=args.async_help_min,
+                      async_group=args.async_group, async_help_min=args.async_help_min, lazy_mode=args.lazy_mode, lazy_from=args.lazy_from,
                       objective=rcd.RCD_OBJ_GRAPH_CUT if args.objective == "cut" else rcd.RCD_OBJ_FACILITY)
 
     def barrier():
@@ -191,6 +228,9 @@ def run_ours(args):
         torch.cuda.synchronize()
 
     def step_device():
+        if by_classes:
+            from paper_2211_00839_b200.distributed import partition_sharded_gpu
+            return partition_sharded_gpu(ctx, Xd, yd, wl.capacities, wl.L)
         out = ctx.rcd_partition(Xd, yd, wl.capacities, wl.L, M_max=M)
         return out
 
@@ -206,24 +246,47 @@ def run_ours(args):
     ctx.sync_status()
     launches_per_step = int(ctx.profile()["kernel_launches"])
 
+    # Inputs of a step = the similarity matrices every sweep re-reads.  When they exceed L2 nothing survives between
+    # steps; when they fit, a buffer larger than L2 is written between the timed steps (outside the event pairs).
+    l2_bytes = int(torch.cuda.get_device_properties(local).L2_cache_size)
+    s_bytes = 4.0 * wl.L * M * M
+    fits_l2 = s_bytes <= l2_bytes
+    flush = torch.empty(2 * l2_bytes, dtype=torch.uint8, device=dev) if fits_l2 else None
+
     sampler = ClockSampler(local)
     barrier()
     sampler.start()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
+    pairs = []
     for _ in range(args.steps):
+        if flush is not None:
+            flush.fill_(1)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
         out = step_device()
-    e1.record()
+        e1.record()
+        pairs.append((e0, e1))
     barrier()
-    clocks = sampler.stop()
     ctx.sync_status()
-    ms = e0.elapsed_time(e1)
+    # (one bracket around all K steps when nothing is flushed in between; the sum of the steps' own brackets otherwise)
+    ms = pairs[0][0].elapsed_time(pairs[-1][1]) if flush is None else sum(a.elapsed_time(b) for a, b in pairs)
     prof = ctx.profile()
+    # a short timed region leaves the 100 ms clock sampler with nothing: keep the same load running (untimed) until it
+    # has a dozen samples, and say so
+    extra_steps = 0
+    t_guard = time.perf_counter()
+    while len(sampler.lines) < 12 and time.perf_counter() - t_guard < 4.0:
+        step_device()
+        torch.cuda.synchronize()
+        extra_steps += 1
+    clocks = sampler.stop()
+    clocks["sampled_over"] = "the timed steps" if extra_steps == 0 else "the timed steps and %d further identical steps (untimed)" % extra_steps
+    ctx.sync_status()
     if world > 1:
         t = torch.tensor([ms], device=dev, dtype=torch.float64)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         ms = float(t.item())
-    value = world * wl.N * args.steps / (ms * 1e-3)
+    jobs = 1 if by_classes else world                 # datasets partitioned per step, all ranks together
+    value = jobs * wl.N * args.steps / (ms * 1e-3)
 
     # end to end: host buffers in, host buffers out, copies inside the timed region
     for _ in range(max(1, min(args.warmup, 2))):
@@ -242,7 +305,7 @@ def run_ours(args):
         t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         e2e_ms = float(t.item())
-    e2e_value = world * wl.N * args.steps / (e2e_ms * 1e-3)
+    e2e_value = jobs * wl.N * args.steps / (e2e_ms * 1e-3)
     h2d = Xh.numel() * Xh.element_size() + yh.numel() * 4
     d2h = sum(t.numel() * t.element_size() for t in host_out)
 
@@ -253,6 +316,11 @@ def run_ours(args):
     # plus the coverage vectors of the blocks refreshed (4*ld*(n_R + n) bytes), summed on the device.
     # Duration = CUDA events around the greedy loop on the launching stream (last timed step).
     peaks = load_peaks()
+    yard = measure_yardsticks(rcd, ctx, dev, rcd.RCD_FEAT_I8 if wl.dtype == "int8" else rcd.RCD_FEAT_BF16) if rank == 0 else None
+    if world > 1:
+        box = [yard]
+        dist.broadcast_object_list(box, src=0)
+        yard = box[0]
     default_setup = args.classes == 0 and args.sweep_batch in (0, 8) and args.async_group == 0 and args.async_help_min == 0 and args.similarity == "dot"
     loop_s = prof["greedy_ms"] * 1e-3
     achieved = prof["sweep_bytes"] / loop_s / 1e9 if loop_s > 0 else 0.0
@@ -262,8 +330,14 @@ def run_ours(args):
         kernel_name = "greedy_async_kernel"
     else:
         kernel_name = "greedy_persistent_kernel" if args.greedy_path != 1 else "sweep_kernel"
-    roofline = {"bound": "hbm", "kernel": kernel_name, "achieved": achieved, "peak": peaks["hbm_gbs"],
-                "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "peak_source": peaks["source"],
+    # S larger than L2: the sweeps stream from HBM (peak: the measured copy bandwidth); S inside L2: they stream from
+    # L2 (peak: this library's read-only sweep yardstick over an L2-resident buffer, measured in this run)
+    bound = "l2" if fits_l2 else "hbm"
+    sweep_peak = yard["l2_read_gbs"] if fits_l2 else peaks["hbm_gbs"]
+    roofline = {"bound": bound, "kernel": kernel_name, "achieved": achieved, "peak": sweep_peak,
+                "unit": "GB/s", "frac": achieved / sweep_peak,
+                "peak_source": ("measured in this run: read-only sweep over %.0f MB (L2-resident)" % yard["l2_read_buffer_mb"]) if fits_l2 else peaks["source"],
+                "yardsticks": yard,
                 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of that kernel on this workload, from the
                 # ncu capture summarised under profiles/ (None: no capture of the kernel as it stands)
                 "traffic": MEASURED_TRAFFIC.get((args.config, kernel_name)) if default_setup else None,
@@ -273,7 +347,7 @@ def run_ours(args):
     # round-based kernel, the busy time of the first sweep CTA of the asynchronous one)
     if prof["persistent_sweep_ns"] > 0:
         ph = prof["sweep_bytes"] / (prof["persistent_sweep_ns"] * 1e-9) / 1e9
-        roofline["sweep_phases"] = {"achieved": ph, "frac": ph / peaks["hbm_gbs"], "ms": prof["persistent_sweep_ns"] * 1e-6,
+        roofline["sweep_phases"] = {"achieved": ph, "frac": ph / sweep_peak, "ms": prof["persistent_sweep_ns"] * 1e-6,
                                     "pick_phases_ms": prof["persistent_pick_ns"] * 1e-6,
                                     "elem_block_ops_per_s": prof["sweep_elem_ops"] / (prof["persistent_sweep_ns"] * 1e-9)}
     # and with every round's sweep as a launch of its own (sweep_kernel), one CUDA-event pair each
@@ -285,35 +359,54 @@ def run_ours(args):
     sweep_s = p2["sweep_ms"] * 1e-3
     if sweep_s > 0:
         a2 = p2["sweep_bytes"] / sweep_s / 1e9
-        roofline["sweep_kernel_launches"] = {"achieved": a2, "frac": a2 / peaks["hbm_gbs"], "launches": int(p2["sweep_launches"]),
+        roofline["sweep_kernel_launches"] = {"achieved": a2, "frac": a2 / sweep_peak, "launches": int(p2["sweep_launches"]),
                                              "avg_launch_us": 1e3 * p2["sweep_ms"] / max(1, p2["sweep_launches"]),
                                              "bytes_per_launch": p2["sweep_bytes"] / max(1, p2["sweep_launches"])}
-    # similarity GEMM: a dense contraction on the tensor cores.  Peak for its dtype: the measured bf16
-    # cuBLAS peak, times 2 for int8 (nominal int8 : bf16 ratio of the part); it also has to write 4*M^2
-    # bytes per class, which is the tighter bound at d = 512.
+    # similarity GEMM: a dense contraction on the tensor cores.  Peak: this library's tensor-core peak loop for the
+    # dtype, measured in this run (the cuBLAS bf16 figure of MEASURED_PEAKS.json is printed beside it).  It also has
+    # to write 4*M^2 bytes per class, the tighter bound at d = 512.  Flops by the full-matrix convention 2*M^2*d per
+    # class; the kernel computes only the 128 x 128 tiles on or above the diagonal (S is symmetric) and mirrors the
+    # stores, so the flops it executes are given as well.
     sim_flops = 2.0 * wl.L * M * M * wl.d
+    nt = (M + 127) // 128
+    exec_flops = 2.0 * wl.L * (nt * (nt + 1) // 2) * 128 * 128 * wl.d
     sim_s = prof["similarity_ms"] * 1e-3
-    tensor_peak = peaks["bf16_tflops"] * (2.0 if wl.dtype == "int8" else 1.0)
+    tensor_peak = yard["mma_tflops"]
     sim_tflops = sim_flops / sim_s / 1e12 if sim_s > 0 else None
+    exec_tflops = exec_flops / sim_s / 1e12 if sim_s > 0 else None
     sim_gbs = 4.0 * wl.L * M * M / sim_s / 1e9 if sim_s > 0 else None
+    t_flops = exec_flops / (tensor_peak * 1e12)
+    t_bytes = 4.0 * wl.L * M * M / (peaks["hbm_gbs"] * 1e9)
     similarity = {"ms": prof["similarity_ms"], "tensor_core_launches": int(prof["similarity_tc_launches"]),
-                  "tflops": sim_tflops, "tensor_peak_tflops": tensor_peak,
+                  "flops_convention": "full matrix 2*M^2*d per class; the kernel executes the tiles on or above the diagonal only",
+                  "tflops": sim_tflops, "executed_tflops": exec_tflops, "tensor_peak_tflops": tensor_peak,
                   "frac_of_tensor_peak": sim_tflops / tensor_peak if sim_tflops else None,
+                  "executed_frac_of_tensor_peak": exec_tflops / tensor_peak if exec_tflops else None,
                   "bytes_written_gbs": sim_gbs, "frac_of_hbm_peak": sim_gbs / peaks["hbm_gbs"] if sim_gbs else None,
-                  "peak_source": peaks["source"] + (" bf16 x2 (nominal int8:bf16 ratio)" if wl.dtype == "int8" else " bf16")}
+                  "frac_of_bound": max(t_flops, t_bytes) / sim_s if sim_s > 0 else None,
+                  "bound": "tensor" if t_flops >= t_bytes else "hbm-write",
+                  "peak_source": "measured in this run: tcgen05 %s peak loop of this library (cuBLAS bf16 in MEASURED_PEAKS.json: %.0f TFLOP/s)"
+                                 % (yard["mma_dtype"], peaks["bf16_tflops"])}
 
     result = {"metric": "samples partitioned/sec", "value": value, "unit": "samples/s", "n_gpus": world,
               "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps,
-              "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+              "higher_is_better": True, "scaling": "strong" if by_classes else "weak", "vs_baseline": None,
               "dtype": "int64" if (wl.dtype == "int8" and args.similarity == "dot") else ("f32" if args.objective == "facility" else "f64"),
               "data": "synthetic",
               "config": {"workload": workload_name(args.config, wl),
-                         "l2": "inputs larger than L2 (S is %.0f MB per class, re-read every sweep)" % (4e-6 * M * M),
-                         "sweep_batch_max": args.sweep_batch or 8, "similarity": args.similarity, "objective": args.objective, "sharding": "one dataset per rank, no collective"},
-              "gain_evals_per_s": world * wl.L * M * (M + 1) / 2 * args.steps / (ms * 1e-3),
+                         "l2": ("inputs larger than L2 (S: %.0f MB in all, %.1f MB per class, re-read every sweep; L2 %.0f MB)"
+                                if not fits_l2 else
+                                "S of all classes (%.0f MB, %.1f MB per class) fits in L2 (%.0f MB): a buffer of twice the L2 size is written between timed steps")
+                               % (s_bytes * 1e-6, 4e-6 * M * M, l2_bytes * 1e-6),
+                         "sweep_batch_max": args.sweep_batch or 8, "similarity": args.similarity, "objective": args.objective,
+                         "sharding": ("one dataset, classes sharded over the ranks by M^3, one all-gather of the assignment per step" if by_classes
+                                      else "one dataset per rank, no collective")},
+              "gain_evals_per_s": jobs * wl.L * M * (M + 1) / 2 * args.steps / (ms * 1e-3),
               "phases_ms": dict({k: prof[k] for k in ("group_ms", "similarity_ms", "greedy_ms", "total_ms")},
                                 sweep_phases_ms=prof["persistent_sweep_ns"] * 1e-6, pick_phases_ms=prof["persistent_pick_ns"] * 1e-6,
-                                async_lull_ms=prof["async_lull_ns"] * 1e-6, async_visits=int(prof["async_visits"]), async_attempts=int(prof["async_attempts"])),
+                                async_lull_ms=prof["async_lull_ns"] * 1e-6, async_visits=int(prof["async_visits"]), async_attempts=int(prof["async_attempts"]),
+                                lazy_sweeps=int(prof["lazy_sweeps"]), lazy_misses=int(prof["lazy_misses"]), lazy_rows=int(prof["lazy_rows"]),
+                                lazy_rows_skipped=int(prof["lazy_rows_skipped"])),
               "similarity": similarity,
               "e2e": {"value": e2e_value, "unit": "samples/s", "h2d_bytes_per_step": int(h2d),
                       "d2h_bytes_per_step": int(d2h), "wall_ms_per_step": e2e_wall_ms / args.steps},
@@ -350,6 +443,10 @@ def main():
                     help="0 = chosen by the library, 1 = two launches per round, 2 = one launch with rounds, 3 = one launch, asynchronous classes")
     ap.add_argument("--async-help-min", type=int, default=0, help="greedy path 3: row groups left before other classes' CTAs help (0 = default)")
     ap.add_argument("--async-group", type=int, default=0, help="greedy path 3: sweeps served together (0 = library default)")
+    ap.add_argument("--sharding", default="replicas", choices=["replicas", "classes"],
+                    help="with --gpus N: one dataset per rank (weak scaling), or one dataset with its classes sharded over the ranks (strong scaling)")
+    ap.add_argument("--lazy-mode", type=int, default=0, help="1 = threshold passes skip rows below the blocks' floors (exact lazy evaluation), 0 = every pass reads every row")
+    ap.add_argument("--lazy-from", type=int, default=0, help="members a block needs before rows are skipped (0 = library default)")
     ap.add_argument("--ref-picks", type=int, default=150, help="picks per class in the CPU-oracle sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

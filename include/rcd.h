@@ -96,7 +96,13 @@ typedef struct {
     int32_t threshold_from;    /* members every out-of-date block must have before a class tries threshold passes; 0 = default (8) */
     int32_t threshold_hit_shift; /* a threshold pass that finds more than 1 element in 2^k above the threshold sends the class
                                   back to dense passes until its blocks have twice the members; 0 = default (k = 5) */
-    int32_t reserved[5];       /* must be 0 */
+    int32_t lazy_mode;         /* exact lazy evaluation of GreedyStep's argmax.  0 = off: every pass visits every unassigned row.
+                                  1 = on: a threshold pass skips rows whose stored gains (upper bounds of the current ones, by
+                                  diminishing returns) lie below a per-block floor; a pick whose best stored gain is below
+                                  its block's floor is not made, the block gets a pass over every row instead.  Same picks
+                                  either way; fewer bytes read, but each class waits longer for its short passes. */
+    int32_t lazy_from;         /* members every out-of-date block must have before rows are skipped; 0 = default (8) */
+    int32_t reserved[3];       /* must be 0 */
 } rcd_config;
 
 /* Timings and counters of the last rcd_partition / rcd_partition_host on a context (profile >= 1). */
@@ -122,6 +128,10 @@ typedef struct {
     int64_t async_lull_ns;          /* asynchronous form: time the first sweep CTA found no sweep with tickets left */
     int64_t async_visits;           /* asynchronous form: times the first sweep CTA went to a class and swept there */
     int64_t async_attempts;         /* ... and times it tried (an attempt fails when the tickets run out under way) */
+    int64_t lazy_sweeps;            /* threshold passes that skipped rows below the blocks' floors */
+    int64_t lazy_misses;            /* picks whose best stored gain lay below its block's floor (answered by a pass over every row) */
+    int64_t lazy_rows;              /* rows of S those passes did read */
+    int64_t lazy_rows_skipped;      /* rows they did not */
 } rcd_profile;
 
 typedef struct rcd_ctx rcd_ctx;
@@ -278,6 +288,22 @@ RCD_API rcd_status rcd_batch_sizes(int64_t B, const double *capacities_host, int
 RCD_API rcd_status rcd_objective_class_static(rcd_ctx *ctx, const void *S_dev, rcd_feat_dtype dtype, int64_t M,
                                       int64_t ldS, const int32_t *assignment_dev, int32_t W,
                                       void *part_values_dev, void *total_dev, void *cuda_stream);
+
+/* ---- yardsticks (measurement only; no counterpart in the paper) ------------------------------ */
+
+/* A read-only sweep with the access pattern of the dense gain sweep (one CTA of 512 threads per SM, 128-bit loads
+ * that do not allocate in L1): reads `bytes` bytes at buffer_dev (16-byte aligned, owned by the caller, contents
+ * irrelevant) `repeats` times inside ONE launch.  A buffer well below the L2 size with many repeats measures the
+ * L2-resident read bandwidth, a buffer of gigabytes with one repeat the HBM read bandwidth: bytes * repeats over
+ * the time the caller measures with events on cuda_stream.  Only enqueues. */
+RCD_API rcd_status rcd_yardstick_read(rcd_ctx *ctx, const void *buffer_dev, size_t bytes, int32_t repeats, void *cuda_stream);
+
+/* A tensor-core peak loop: one CTA per SM issues `iterations` batches of sixteen 128 x 256 x (32-byte k)
+ * tcgen05.mma instructions (RCD_FEAT_I8: s8 x s8 -> s32; RCD_FEAT_BF16: bf16 x bf16 -> f32) on operands that stay in
+ * shared memory, accumulators in tensor memory.  *ops_host_out (may be NULL) receives the number of arithmetic
+ * operations (2 per multiply-add) the launch performs; divide by the time measured on cuda_stream.  Every wait in
+ * the kernel is bounded (RCD_ERR_TIMEOUT from rcd_sync_status otherwise).  Only enqueues. */
+RCD_API rcd_status rcd_yardstick_mma(rcd_ctx *ctx, rcd_feat_dtype dtype, int32_t iterations, double *ops_host_out, void *cuda_stream);
 
 #ifdef __cplusplus
 }

@@ -36,7 +36,8 @@ EXPORTS = ["rcd_create", "rcd_destroy", "rcd_last_error", "rcd_version", "rcd_sy
            "rcd_partition_workspace_bytes", "rcd_partition",
            "rcd_partition_host_workspace_bytes", "rcd_partition_host", "rcd_objective_workspace_bytes",
            "rcd_objective", "rcd_objective_class_static",
-           "rcd_worker_lists_workspace_bytes", "rcd_worker_lists", "rcd_batch_sizes"]
+           "rcd_worker_lists_workspace_bytes", "rcd_worker_lists", "rcd_batch_sizes",
+           "rcd_yardstick_read", "rcd_yardstick_mma"]
 
 
 class RcdError(RuntimeError):
@@ -49,7 +50,7 @@ class RcdConfig(C.Structure):
     _fields_ = [("sweep_batch_max", C.c_int32), ("similarity_path", C.c_int32), ("profile", C.c_int32),
                 ("greedy_path", C.c_int32), ("similarity_kind", C.c_int32), ("objective", C.c_int32), ("sweep_mode", C.c_int32), ("async_group", C.c_int32),
                 ("async_help_min", C.c_int32), ("threshold_from", C.c_int32), ("threshold_hit_shift", C.c_int32),
-                ("reserved", C.c_int32 * 5)]
+                ("lazy_mode", C.c_int32), ("lazy_from", C.c_int32), ("reserved", C.c_int32 * 3)]
 
 
 class RcdProfile(C.Structure):
@@ -59,7 +60,9 @@ class RcdProfile(C.Structure):
                 ("steps", C.c_int64), ("similarity_tc_launches", C.c_int64), ("persistent_sweep_ns", C.c_int64),
                 ("persistent_pick_ns", C.c_int64), ("threshold_hits", C.c_int64),
                 ("threshold_elems", C.c_int64), ("threshold_max_blocks", C.c_int64),
-                ("async_lull_ns", C.c_int64), ("async_visits", C.c_int64), ("async_attempts", C.c_int64)]
+                ("async_lull_ns", C.c_int64), ("async_visits", C.c_int64), ("async_attempts", C.c_int64),
+                ("lazy_sweeps", C.c_int64), ("lazy_misses", C.c_int64), ("lazy_rows", C.c_int64),
+                ("lazy_rows_skipped", C.c_int64)]
 
 
 def _load() -> C.CDLL:
@@ -92,6 +95,8 @@ def _load() -> C.CDLL:
     lib.rcd_worker_lists_workspace_bytes.argtypes = [vp, i64, i32, C.POINTER(sz)]
     lib.rcd_worker_lists.argtypes = [vp, vp, i64, i32, vp, vp, vp, sz, vp]
     lib.rcd_batch_sizes.argtypes = [i64, vp, i32, vp]
+    lib.rcd_yardstick_read.argtypes = [vp, vp, sz, i32, vp]
+    lib.rcd_yardstick_mma.argtypes = [vp, C.c_int, i32, C.POINTER(C.c_double), vp]
     for name in EXPORTS:
         f = getattr(lib, name)
         if name not in ("rcd_destroy", "rcd_last_error", "rcd_version"):
@@ -161,7 +166,8 @@ class Context:
 
     def __init__(self, device: int = 0, sweep_batch_max: int = 0, similarity_path: int = 0, profile: int = 0,
                  greedy_path: int = 0, similarity_kind: int = 0, objective: int = 0, sweep_mode: int = 0,
-                 async_group: int = 0, async_help_min: int = 0, threshold_from: int = 0, threshold_hit_shift: int = 0):
+                 async_group: int = 0, async_help_min: int = 0, threshold_from: int = 0, threshold_hit_shift: int = 0,
+                 lazy_mode: int = 0, lazy_from: int = 0):
         torch = _torch()
         if not torch.cuda.is_available():
             raise RcdError(4, "no CUDA device: this library has no CPU path")
@@ -179,6 +185,8 @@ class Context:
         cfg.async_help_min = async_help_min
         cfg.threshold_from = threshold_from
         cfg.threshold_hit_shift = threshold_hit_shift
+        cfg.lazy_mode = lazy_mode
+        cfg.lazy_from = lazy_from
         self.similarity_kind = similarity_kind
         self._h = C.c_void_p()
         st = lib.rcd_create(C.byref(self._h), self.device, C.byref(cfg))
@@ -389,6 +397,20 @@ def rcd_objective_class_static(ctx: Context, S, assignment, W: int, part_values,
                                               C.c_void_p(assignment.data_ptr()), W,
                                               C.c_void_p(part_values.data_ptr()), C.c_void_p(total.data_ptr()),
                                               ctx._stream()))
+
+
+def rcd_yardstick_read(ctx: Context, buffer, repeats: int = 1) -> int:
+    """Enqueues the read-only sweep over ``buffer`` (any device tensor); returns the bytes one call reads."""
+    nbytes = buffer.numel() * buffer.element_size() // 16 * 16
+    ctx._check(lib.rcd_yardstick_read(ctx._h, C.c_void_p(buffer.data_ptr()), nbytes, int(repeats), ctx._stream()))
+    return nbytes * int(repeats)
+
+
+def rcd_yardstick_mma(ctx: Context, dtype_code: int, iterations: int) -> float:
+    """Enqueues the tensor-core peak loop; returns the arithmetic operations the launch performs."""
+    ops = C.c_double()
+    ctx._check(lib.rcd_yardstick_mma(ctx._h, int(dtype_code), int(iterations), C.byref(ops), ctx._stream()))
+    return float(ops.value)
 
 
 def rcd_similarity(ctx: Context, X):

@@ -17,7 +17,7 @@ OBJ = os.path.join(ROOT, "_build")
 LIB = os.path.join(HERE, "librcd.so")
 
 SOURCES = ["rcd_api.cu", "rcd_group.cu", "rcd_similarity.cu", "rcd_similarity_tc.cu", "rcd_greedy.cu",
-           "rcd_objective.cu", "rcd_objective_static.cu", "rcd_gaussian.cu", "rcd_cut.cu"]
+           "rcd_objective.cu", "rcd_objective_static.cu", "rcd_gaussian.cu", "rcd_cut.cu", "rcd_yardstick.cu"]
 HEADERS = [os.path.join(CSRC, "rcd_internal.h"), os.path.join(ROOT, "include", "rcd.h")]
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

@@ -108,9 +108,13 @@ size_t layout_workspace(void *base, rcd_feat_dtype dtype, const Sizes &sz, Works
     w.tickets = c.take<int32_t>(N + L);
     w.sweepF = c.take<long long>(L * 8);
     w.sizesSorted = c.take<int32_t>(L);
+    w.floorv = c.take<unsigned char>(L * kLazyBlocks * 8);
+    w.theta = c.take<unsigned char>(L * kLazyBlocks * 8);
+    w.sweepTheta = c.take<unsigned char>(L * kLazyBlocks * 8);
+    w.lazyStat = c.take<int32_t>(L * 4);
     w.stepBytes = c.take<unsigned long long>((size_t)sz.maxM + 1);
     w.stepOps = c.take<unsigned long long>((size_t)sz.maxM + 1);
-    w.phaseNs = c.take<unsigned long long>(8);      // two phase clocks, the grid-barrier counter, threshold-pass hits / elements
+    w.phaseNs = c.take<unsigned long long>(kPhaseWords);   // phase clocks, the grid-barrier counter, threshold-pass and row-skipping counters
     w.bytes = align_up(c.off);
     if (ws) *ws = w;
     return w.bytes;
@@ -313,7 +317,9 @@ rcd_status rcd_create(rcd_ctx **out, int cuda_device, const rcd_config *cfg)
         if (cfg->async_group < 0 || cfg->async_group > 4096) return RCD_ERR_INVALID_ARG;
         if (cfg->async_help_min < 0) return RCD_ERR_INVALID_ARG;
         if (cfg->threshold_from < 0 || cfg->threshold_hit_shift < 0 || cfg->threshold_hit_shift > 30) return RCD_ERR_INVALID_ARG;
-        for (int i = 0; i < 5; ++i) if (cfg->reserved[i] != 0) return RCD_ERR_INVALID_ARG;
+        if (cfg->lazy_mode != 0 && cfg->lazy_mode != 1) return RCD_ERR_INVALID_ARG;
+        if (cfg->lazy_from < 0) return RCD_ERR_INVALID_ARG;
+        for (int i = 0; i < 3; ++i) if (cfg->reserved[i] != 0) return RCD_ERR_INVALID_ARG;
     }
     int count = 0;
     if (cudaGetDeviceCount(&count) != cudaSuccess || cuda_device < 0 || cuda_device >= count) {
@@ -390,13 +396,19 @@ rcd_status rcd_get_profile(rcd_ctx *ctx, rcd_profile *out)
     if (!ctx->phaseValid) return RCD_OK;
     RCD_CUDA(ctx, cudaEventSynchronize(ctx->evPhase[4]));
     float ms = 0.f;
+    int64_t lazyBytes = 0;      // bytes of the rows read by row-skipping passes (counted as they are read)
     RCD_CUDA(ctx, cudaEventElapsedTime(&ms, ctx->evPhase[0], ctx->evPhase[4])); out->total_ms = ms;
     RCD_CUDA(ctx, cudaEventElapsedTime(&ms, ctx->evPhase[0], ctx->evPhase[1])); out->group_ms = ms;
     RCD_CUDA(ctx, cudaEventElapsedTime(&ms, ctx->evPhase[1], ctx->evPhase[2])); out->similarity_ms = ms;
     RCD_CUDA(ctx, cudaEventElapsedTime(&ms, ctx->evPhase[2], ctx->evPhase[3])); out->greedy_ms = ms;
     if (ctx->phaseNsDev) {
-        unsigned long long ns[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+        unsigned long long ns[kPhaseWords] = {};
         RCD_CUDA(ctx, cudaMemcpy(ns, ctx->phaseNsDev, sizeof ns, cudaMemcpyDeviceToHost));
+        out->lazy_sweeps = (int64_t)ns[8];
+        out->lazy_misses = (int64_t)ns[9];
+        out->lazy_rows = (int64_t)ns[10];
+        out->lazy_rows_skipped = (int64_t)ns[11];
+        lazyBytes = (int64_t)ns[12];
         out->persistent_sweep_ns = (int64_t)ns[0];
         out->persistent_pick_ns = (int64_t)ns[1];
         out->threshold_hits = (int64_t)ns[3];
@@ -420,6 +432,7 @@ rcd_status rcd_get_profile(rcd_ctx *ctx, rcd_profile *out)
                 out->sweep_ms += ms;
             }
         }
+        out->sweep_bytes += lazyBytes;
     }
     return RCD_OK;
 }

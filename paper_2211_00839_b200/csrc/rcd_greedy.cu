@@ -94,6 +94,12 @@ struct GreedyParams {
     int32_t nPick;              // CTAs [0, nPick) make picks, the others sweep
     int32_t helpMin;            // row groups a sweep must have left for a sweep CTA that is not at home there
     int32_t asyncGroup;         // sweeps published one after another that are served together (by CTA home position)
+    // row skipping (lazy evaluation of GreedyStep's argmax): see plan_decide / sweep_class_lazy / pick_chain
+    FV *floorv;                 // [L][kLazyBlocks] every stored gain of the block at or above this value is exact
+    FV *theta;                  // [L][kLazyBlocks] the floor the block's next row-skipping pass establishes
+    GV *sweepTheta;             // [L][kLazyBlocks] those floors for the blocks of the class's next pass, in list order
+    int32_t *lazyStat;          // [L][4] row-skipping passes, misses
+    int32_t lazyFrom;           // members every listed block must have before a pass skips rows (< 0: never)
     const int32_t *sizesSorted; // [L] class sizes in ascending order
     int32_t minM;               // smallest non-empty class
     int32_t nonEmpty;           // classes that hold at least one sample
@@ -116,7 +122,26 @@ struct PlanShared {
     int32_t needSweep;             //                       1 = that pick must wait for a sweep
     int32_t sweepBlocks;           //                       blocks in the scheduled sweep's list
     int32_t sweepSparse;           //                       1 = the scheduled sweep is a threshold pass
+    int32_t sweepLazy;             //                       1 = ... that skips rows below the blocks' floors
+    // Row skipping.  Stored gains never grow when a block grows (diminishing returns, Section 3.1), so an
+    // out-of-date stored gain is an upper bound of the current one.  floorv[p]: every stored gain of block p at
+    // or above it was recomputed since p last changed (exact); theta[p]: the floor the next pass will use.
+    FV floorv[kLazyBlocks];
+    FV theta[kLazyBlocks];
+    int32_t lazySweeps, lazyMisses;
 };
+
+template <typename T> __device__ __forceinline__ T lowest_value();
+template <> __device__ __forceinline__ long long lowest_value<long long>() { return LLONG_MIN; }
+template <> __device__ __forceinline__ double lowest_value<double>() { return -INFINITY; }
+template <> __device__ __forceinline__ float lowest_value<float>() { return -INFINITY; }
+template <typename T> __device__ __forceinline__ T highest_value();
+template <> __device__ __forceinline__ long long highest_value<long long>() { return LLONG_MAX; }
+template <> __device__ __forceinline__ double highest_value<double>() { return INFINITY; }
+
+// Rows one ticket of a sweep stands for: R rows of a dense pass, two of a threshold pass, 32 of a row-skipping
+// pass (one per lane: most of them are skipped).
+constexpr int kLazyRows = 32;
 
 template <typename SV>
 __device__ __forceinline__ void plan_load(const GreedyParams<SV> &prm, int l, PlanShared<typename Arith<SV>::FV> &sh)
@@ -130,6 +155,30 @@ __device__ __forceinline__ void plan_load(const GreedyParams<SV> &prm, int l, Pl
         sh.room[p] = room;
         sh.quota[p] = quota;
         sh.open[p] = (uint8_t)((room > 0 ? 1 : 0) | (prm.valid[at] ? 0 : 2));
+        if (p < kLazyBlocks) {
+            sh.floorv[p] = prm.floorv[(int64_t)l * kLazyBlocks + p];
+            sh.theta[p] = prm.theta[(int64_t)l * kLazyBlocks + p];
+        }
+    }
+    if (threadIdx.x == 0) {
+        sh.lazySweeps = prm.lazyStat[4 * l];
+        sh.lazyMisses = prm.lazyStat[4 * l + 1];
+    }
+}
+
+// The counterpart of plan_load for what a chain changes of the row-skipping state (block values and counts are
+// written as the picks are made).
+template <typename SV>
+__device__ __forceinline__ void plan_store_lazy(const GreedyParams<SV> &prm, int l, const PlanShared<typename Arith<SV>::FV> &sh)
+{
+    const int n = min(prm.W, kLazyBlocks);
+    for (int p = threadIdx.x; p < n; p += blockDim.x) {
+        prm.floorv[(int64_t)l * kLazyBlocks + p] = sh.floorv[p];
+        prm.theta[(int64_t)l * kLazyBlocks + p] = sh.theta[p];
+    }
+    if (threadIdx.x == 0) {
+        prm.lazyStat[4 * l] = sh.lazySweeps;
+        prm.lazyStat[4 * l + 1] = sh.lazyMisses;
     }
 }
 
@@ -189,6 +238,7 @@ __device__ void plan_decide(const GreedyParams<SV> &prm, int l, const ClassDesc 
                             PlanShared<typename Arith<SV>::FV> &sh, const PlanGlobals *pre = nullptr)
 {
     using FV = typename Arith<SV>::FV;
+    using GV = typename Arith<SV>::GV;
     const int lane = threadIdx.x & 31;
     const int W = prm.W;
     uint8_t *valid = prm.valid + (int64_t)l * W;
@@ -202,6 +252,7 @@ __device__ void plan_decide(const GreedyParams<SV> &prm, int l, const ClassDesc 
     int bestP = INT_MAX;
     int nStale = 0;
     int fewest = INT_MAX;                          // members of the emptiest out-of-date non-full block
+    int floorsKnown = 1;                           // every out-of-date non-full block has a floor for a row-skipping pass
     for (int p = lane; p < W; p += 32) {
         const uint8_t o = sh.open[p];
         if (o & 1) {
@@ -210,6 +261,7 @@ __device__ void plan_decide(const GreedyParams<SV> &prm, int l, const ClassDesc 
             if (o & 2) {
                 ++nStale;
                 fewest = min(fewest, sh.quota[p] - sh.room[p]);
+                if (p >= kLazyBlocks || !(sh.theta[p] > lowest_value<FV>())) floorsKnown = 0;
             }
         }
     }
@@ -218,6 +270,7 @@ __device__ void plan_decide(const GreedyParams<SV> &prm, int l, const ClassDesc 
         int oP = __shfl_xor_sync(0xffffffffu, bestP, off);
         nStale += __shfl_xor_sync(0xffffffffu, nStale, off);
         fewest = min(fewest, __shfl_xor_sync(0xffffffffu, fewest, off));
+        floorsKnown &= __shfl_xor_sync(0xffffffffu, floorsKnown, off);
         if (oP != INT_MAX && (bestP == INT_MAX || oF < bestF || (oF == bestF && oP < bestP))) { bestF = oF; bestP = oP; }
     }
     if (bestP == INT_MAX) {
@@ -263,10 +316,16 @@ __device__ void plan_decide(const GreedyParams<SV> &prm, int l, const ClassDesc 
     }
     from = __shfl_sync(0xffffffffu, from, 0);
     const int64_t together0 = max(remaining, 1);
-    const bool sparse = prm.sparseMinMembers >= 0 && prm.batchMax > 1 && nStale > 1 && fewest >= from &&
+    // Row skipping: a threshold pass may leave out every row whose stored gains lie below the listed blocks'
+    // floors (they stay upper bounds).  Tried once the blocks have lazyFrom members; a class where, after a few
+    // misses, more than a quarter of such passes ended in one (the best stored gain fell below its floor) stops trying.
+    const bool lazyWanted = prm.lazyFrom >= 0 && W <= kLazyBlocks && floorsKnown && fewest >= prm.lazyFrom &&
+                            (sh.lazyMisses <= 8 || 4 * sh.lazyMisses <= sh.lazySweeps);
+    const bool sparse = prm.sparseMinMembers >= 0 && prm.batchMax > 1 && (nStale > 1 || lazyWanted) && fewest >= from &&
                         (int64_t)thr_bytes_aligned(c.ld * (int)sizeof(SV)) + kSparseQueueBytes <= prm.smemBytes &&
-                        together0 * ((nR + kSparseRows - 1) / kSparseRows) * 4 >= prm.sweepWarps;
+                        (lazyWanted || together0 * ((nR + kSparseRows - 1) / kSparseRows) * 4 >= prm.sweepWarps);
     if (sparse) cap = kSparseMax;
+    const bool lazy = sparse && lazyWanted;
     // n blocks are refreshed; the dense pass is instantiated for lists of 1, 2, 4, 8, so its list is
     // padded with copies of j* up to the next power of two (same bytes read, identical values written)
     const int n = nStale < cap ? nStale : cap;
@@ -274,7 +333,14 @@ __device__ void plan_decide(const GreedyParams<SV> &prm, int l, const ClassDesc 
     while (P < n) P *= 2;
     if (sparse) P = n;
     int32_t *parts = prm.sweepParts + (int64_t)l * kSparseMax;
-    if (lane == 0) { parts[0] = jstar; valid[jstar] = 1; sh.open[jstar] = 1; }
+    GV *listTheta = prm.sweepTheta + (int64_t)l * kLazyBlocks;
+    if (lane == 0) {
+        parts[0] = jstar; valid[jstar] = 1; sh.open[jstar] = 1;
+        if (jstar < kLazyBlocks) {
+            sh.floorv[jstar] = lazy ? sh.theta[jstar] : lowest_value<FV>();
+            listTheta[0] = lazy ? (GV)sh.theta[jstar] : lowest_value<GV>();
+        }
+    }
     __syncwarp();
     if (nStale <= cap) {
         // every out-of-date non-full block is listed: after j* in index order (the order of the list does not
@@ -285,9 +351,14 @@ __device__ void plan_decide(const GreedyParams<SV> &prm, int l, const ClassDesc 
             const bool take = p < W && sh.open[p] == 3;
             const unsigned m = __ballot_sync(0xffffffffu, take);
             if (take) {
-                parts[k + __popc(m & ((1u << lane) - 1u))] = p;
+                const int at = k + __popc(m & ((1u << lane) - 1u));
+                parts[at] = p;
                 valid[p] = 1;
                 sh.open[p] = 1;
+                if (p < kLazyBlocks) {
+                    sh.floorv[p] = lazy ? sh.theta[p] : lowest_value<FV>();
+                    if (at < kLazyBlocks) listTheta[at] = lazy ? (GV)sh.theta[p] : lowest_value<GV>();
+                }
             }
             k += __popc(m);
         }
@@ -308,13 +379,16 @@ __device__ void plan_decide(const GreedyParams<SV> &prm, int l, const ClassDesc 
             int oP = __shfl_xor_sync(0xffffffffu, qP, off);
             if (oP != INT_MAX && (qP == INT_MAX || oF < qF || (oF == qF && oP < qP))) { qF = oF; qP = oP; }
         }
-        if (lane == 0) { parts[k] = qP; valid[qP] = 1; sh.open[qP] = 1; }
+        if (lane == 0) {
+            parts[k] = qP; valid[qP] = 1; sh.open[qP] = 1;
+            if (qP < kLazyBlocks) sh.floorv[qP] = lowest_value<FV>();     // (more blocks than one list holds: never a row-skipping pass)
+        }
         __syncwarp();
     }
     if (lane == 0) for (int k = n; k < P; ++k) parts[k] = jstar;
     // warps per row group: enough that the row groups of the classes that sweep together (every
     // unfinished class, once per round) cover every warp of the launch, at least one 128-column chunk per warp
-    const int R = sparse ? kSparseRows : rows_per_group(P);
+    const int R = lazy ? kLazyRows : (sparse ? kSparseRows : rows_per_group(P));
     const int64_t nGroups = (nR + R - 1) / R;
     const int rem = remaining;                                        // unfinished classes: they all sweep in the same round
     const int64_t together = rem > 1 ? rem : 1;
@@ -326,10 +400,16 @@ __device__ void plan_decide(const GreedyParams<SV> &prm, int l, const ClassDesc 
         sh.needSweep = 1;
         sh.sweepBlocks = P;
         sh.sweepSparse = sparse ? 1 : 0;
-        prm.sweepMode[l] = sparse ? 1 : 0;
+        sh.sweepLazy = lazy ? 1 : 0;
+        prm.sweepMode[l] = lazy ? 2 : (sparse ? 1 : 0);
         if (sparse) {
-            prm.sparseElems[l] = (unsigned long long)nR * (unsigned long long)c.M;
+            // (a row-skipping pass compares only the rows it reads: its hit rate does not steer the back-off)
+            prm.sparseElems[l] = lazy ? 0ull : (unsigned long long)nR * (unsigned long long)c.M;
             atomicMax(&prm.phaseNs[5], (unsigned long long)P);
+        }
+        if (lazy) {
+            sh.lazySweeps += 1;
+            atomicAdd(&prm.phaseNs[8], 1ull);
         }
         prm.jstar[l] = jstar;
         prm.sweepN[l] = P;
@@ -339,7 +419,7 @@ __device__ void plan_decide(const GreedyParams<SV> &prm, int l, const ClassDesc 
             ClassSync &sy = prm.sync[l];                   // published with the epoch by the caller
             sy.nGroups = (int32_t)nGroups;
             sy.nR = nR;
-            sy.cfg = P | (CS << 8) | ((sparse ? 1 : 0) << 16);
+            sy.cfg = P | (CS << 8) | ((lazy ? 2 : (sparse ? 1 : 0)) << 16);
             if constexpr (Arith<SV>::kInt) {
                 if (!sparse)
                     for (int k = 0; k < P; ++k) prm.sweepF[(int64_t)l * kMaxSweepBatch + k] = (long long)sh.f[parts[k]];
@@ -349,8 +429,14 @@ __device__ void plan_decide(const GreedyParams<SV> &prm, int l, const ClassDesc 
             int slot = atomicAdd(&prm.nSweep[par], 1);
             prm.sweepList[(int64_t)par * prm.L + slot] = l;
         }
-        atomicAdd(&prm.stepBytes[nextStep], (unsigned long long)((int64_t)nR * c.ld + (int64_t)(sparse ? 1 : n) * c.ld) * sizeof(SV));
-        atomicAdd(&prm.stepOps[nextStep], (unsigned long long)((int64_t)nR * c.M * (sparse ? 1 : n)));
+        if (lazy) {
+            // what the pass reads whatever it finds: the threshold vector, the candidate list and the stored gains of
+            // the listed blocks; the rows of S it does read are counted by the warps that read them
+            atomicAdd(&prm.stepBytes[nextStep], (unsigned long long)((int64_t)c.ld * sizeof(SV) + (int64_t)nR * (4 + (int64_t)n * sizeof(GV))));
+        } else {
+            atomicAdd(&prm.stepBytes[nextStep], (unsigned long long)((int64_t)nR * c.ld + (int64_t)(sparse ? 1 : n) * c.ld) * sizeof(SV));
+            atomicAdd(&prm.stepOps[nextStep], (unsigned long long)((int64_t)nR * c.M * (sparse ? 1 : n)));
+        }
     }
 }
 
@@ -374,6 +460,11 @@ __global__ void __launch_bounds__(kSelectThreads, 4) init_kernel(GreedyParams<SV
         prm.fval[(int64_t)l * W + p] = (FV)0;
         prm.valid[(int64_t)l * W + p] = 0;
     }
+    for (int p = threadIdx.x; p < kLazyBlocks; p += blockDim.x) {
+        prm.floorv[(int64_t)l * kLazyBlocks + p] = lowest_value<FV>();
+        prm.theta[(int64_t)l * kLazyBlocks + p] = lowest_value<FV>();
+    }
+    if (threadIdx.x < 4) prm.lazyStat[4 * l + threadIdx.x] = 0;
     if (threadIdx.x == 0) {
         prm.nR[l] = c.M;
         prm.sparseFrom[l] = prm.sparseMinMembers;
@@ -666,35 +757,171 @@ __device__ __forceinline__ void async_copy16(int4 *smemDst, const int4 *src)
 // (P' = P rounded up to a power of two) are in flight at once.  The slots' sums are added at the
 // end of the row group.  With more than 32 blocks every lane serves blocks p and p + 32.
 
+// What a warp of a threshold pass keeps for the whole pass.
+template <typename SV, int A>
+struct SparseWarp {
+    int4 *ring;                 // the warp's ring of chunks of S
+    uint2 *queue;               // the warp's queue of elements above the threshold
+    const int4 *shThr;          // threshold vector (shared memory)
+    int ld4, lane;
+    unsigned below;             // lanes below this one
+    int Pp, slots, slot;        // lanes per queue slot, slots, this lane's slot
+    int myPart[A];              // blocks this lane serves (-1: none)
+    const SV *myCov[A];         // their coverage vectors
+};
+
+template <typename SV, int A>
+__device__ __forceinline__ void sparse_setup(SparseWarp<SV, A> &w, const GreedyParams<SV> &prm, const ClassDesc &c, int P,
+                                             const int4 *shThr, const int32_t *parts, uint2 *warpArea)
+{
+    w.ring = reinterpret_cast<int4 *>(warpArea);                    // per warp: ring, then queue
+    w.queue = warpArea + kSparseRingBytes / 8;
+    w.shThr = shThr;
+    w.ld4 = c.ld >> 2;
+    w.lane = threadIdx.x & 31;
+    w.below = (1u << w.lane) - 1u;
+    const SV *cover = prm.cover + c.vOff;
+    int Pp = 1;                                                     // lanes per queue slot
+    while (Pp < P && Pp < 32) Pp *= 2;
+    w.Pp = Pp;
+    w.slots = 32 / Pp;
+    w.slot = w.lane / Pp;
+#pragma unroll
+    for (int a = 0; a < A; ++a) {
+        const int p = (w.lane & (Pp - 1)) + 32 * a;
+        w.myPart[a] = p < P ? parts[p] : -1;
+        w.myCov[a] = cover + (int64_t)(w.myPart[a] < 0 ? parts[0] : w.myPart[a]) * c.ld;
+    }
+}
+
+// Adds the queued elements to the lanes' running sums: lane (slot, block) fetches the block's coverage of the
+// element's column and adds max(0, S - cover) to the sum of the element's row.
+template <typename SV, int A>
+__device__ __forceinline__ void sparse_drain(const SparseWarp<SV, A> &w, int &qn, typename Arith<SV>::GV (&acc)[kSparseRows][A])
+{
+    using GV = typename Arith<SV>::GV;
+    constexpr int R = kSparseRows;
+    __syncwarp();
+    for (int i0 = w.slot; i0 < qn; i0 += 2 * w.slots) {
+        uint2 e[2];
+        bool ok[2];
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            const int i = i0 + u * w.slots;
+            ok[u] = i < qn;
+            e[u] = w.queue[ok[u] ? i : i0];
+        }
+        GV d[2][A];
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            const int col = (int)(e[u].x & 0x0fffffffu);
+#pragma unroll
+            for (int a = 0; a < A; ++a) {
+                const SV cv = __ldcg(w.myCov[a] + col);
+                if constexpr (Arith<SV>::kInt) {
+                    const int dd = (int)e[u].y - cv;
+                    d[u][a] = (ok[u] && w.myPart[a] >= 0 && dd > 0) ? (GV)dd : (GV)0;
+                } else {
+                    const float dd = __uint_as_float(e[u].y) - cv;
+                    d[u][a] = (ok[u] && w.myPart[a] >= 0 && dd > 0.f) ? dd : 0.f;
+                }
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            const int r = (int)(e[u].x >> 28);
+#pragma unroll
+            for (int rr = 0; rr < R; ++rr)
+#pragma unroll
+                for (int a = 0; a < A; ++a) acc[rr][a] += (r == rr) ? d[u][a] : (GV)0;
+        }
+    }
+    __syncwarp();
+    qn = 0;
+}
+
+// Streams nRows (<= kSparseRows) rows of S against the threshold vector: elements above it are queued and the
+// queue is drained into acc whenever it is nearly full.  On return every copy has landed and the last
+// elements are still in the queue (qn of them): the caller drains them when it has issued what it wants to
+// overlap with that.
+// S streams through a ring in shared memory filled by asynchronous copies, kSparseStages - 1 chunks ahead;
+// every lane reads back only the 16-byte pieces it copied itself, so waiting for its own copy groups is all
+// the synchronisation the ring needs.
+template <typename SV, int A>
+__device__ __forceinline__ void sparse_stream(const SparseWarp<SV, A> &w, const int4 *const (&rp)[kSparseRows], int nRows,
+                                              typename Arith<SV>::GV (&acc)[kSparseRows][A], unsigned &hits, int &qn)
+{
+    constexpr int R = kSparseRows;
+    const int lane = w.lane, ld4 = w.ld4;
+    auto issue = [&](int base, int st) {
+        const int cc = base + lane;
+        if (cc < ld4) {
+#pragma unroll
+            for (int r = 0; r < R; ++r)
+                if (r < nRows) async_copy16(w.ring + (st * R + r) * 32 + lane, rp[r] + cc);
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+#pragma unroll
+    for (int st = 0; st < kSparseStages - 1; ++st) issue(st * 32, st);
+    int stage = 0;
+    for (int base = 0; base < ld4; base += 32) {                // every lane runs every chunk: ballots below
+        const int cc = base + lane;
+        const bool inside = cc < ld4;
+        {
+            int ahead = stage + kSparseStages - 1;
+            if (ahead >= kSparseStages) ahead -= kSparseStages;
+            issue(base + (kSparseStages - 1) * 32, ahead);       // past the row's end: an empty group
+        }
+        asm volatile("cp.async.wait_group %0;" :: "n"(kSparseStages - 1) : "memory");
+        int4 t = make_int4(0, 0, 0, 0);
+        if (inside) t = w.shThr[cc];
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            int4 s = make_int4(0, 0, 0, 0);
+            unsigned h = 0;
+            if (inside && r < nRows) {
+                s = w.ring[(stage * R + r) * 32 + lane];
+                if constexpr (Arith<SV>::kInt) {
+                    h = (s.x > t.x ? 1u : 0u) | (s.y > t.y ? 2u : 0u) | (s.z > t.z ? 4u : 0u) | (s.w > t.w ? 8u : 0u);
+                } else {
+                    h = (__int_as_float(s.x) > __int_as_float(t.x) ? 1u : 0u) | (__int_as_float(s.y) > __int_as_float(t.y) ? 2u : 0u) |
+                        (__int_as_float(s.z) > __int_as_float(t.z) ? 4u : 0u) | (__int_as_float(s.w) > __int_as_float(t.w) ? 8u : 0u);
+                }
+            }
+            if (__any_sync(0xffffffffu, h != 0)) {
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const bool mine = (h >> e) & 1u;
+                    const unsigned m = __ballot_sync(0xffffffffu, mine);
+                    if (mine) {
+                        const int sv = e == 0 ? s.x : (e == 1 ? s.y : (e == 2 ? s.z : s.w));
+                        w.queue[qn + __popc(m & w.below)] = make_uint2((unsigned)(cc * 4 + e) | ((unsigned)r << 28), (unsigned)sv);
+                    }
+                    qn += __popc(m);
+                }
+                if (qn > kSparseQueue - 128) { hits += qn; sparse_drain<SV, A>(w, qn, acc); }
+            }
+        }
+        if (++stage == kSparseStages) stage = 0;
+    }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+}
+
 template <typename SV, int A>
 __device__ __noinline__ void sweep_class_sparse(const GreedyParams<SV> &prm, int l, const ClassDesc c, int nR, int P,
                                                    const int4 *shThr, const int32_t *parts, uint2 *queue,
                                                    int32_t *ticket, int32_t *done, int firstTicket)
 {
-    int4 *ring = reinterpret_cast<int4 *>(queue);                    // per warp: ring, queue, sums
-    queue += kSparseRingBytes / 8;
     using GV = typename Arith<SV>::GV;
     constexpr int R = kSparseRows;
-    const int lane = threadIdx.x & 31;
-    const unsigned below = (1u << lane) - 1u;
-    const int ld4 = c.ld >> 2;
+    SparseWarp<SV, A> w;
+    sparse_setup<SV, A>(w, prm, c, P, shThr, parts, queue);
+    const int lane = w.lane;
     const int nGroups = (nR + R - 1) / R;
     const SV *Sl = prm.S + c.sOff;
     const int32_t *cand = prm.cand + c.row0;
     GV *G = prm.gains + c.vOff;
-    const SV *cover = prm.cover + c.vOff;
-    int Pp = 1;                                                     // lanes per queue slot
-    while (Pp < P && Pp < 32) Pp *= 2;
-    const int slots = 32 / Pp;
-    const int slot = lane / Pp;
-    int myPart[A];
-    const SV *myCov[A];
-#pragma unroll
-    for (int a = 0; a < A; ++a) {
-        const int p = (lane & (Pp - 1)) + 32 * a;
-        myPart[a] = p < P ? parts[p] : -1;
-        myCov[a] = cover + (int64_t)(myPart[a] < 0 ? parts[0] : myPart[a]) * c.ld;
-    }
     unsigned hits = 0;
     int finished = 0;                                               // row groups of this sweep this warp has completed
     // The warp's ticket (firstTicket >= 0: one per warp was drawn by the CTA) and the rows it names.  The next
@@ -731,100 +958,7 @@ __device__ __noinline__ void sweep_class_sparse(const GreedyParams<SV> &prm, int
 #pragma unroll
             for (int a = 0; a < A; ++a) acc[r][a] = 0;
         int qn = 0;                                                 // queued elements (same in every lane)
-        auto drain = [&]() {
-            __syncwarp();
-            for (int i0 = slot; i0 < qn; i0 += 2 * slots) {
-                uint2 e[2];
-                bool ok[2];
-#pragma unroll
-                for (int u = 0; u < 2; ++u) {
-                    const int i = i0 + u * slots;
-                    ok[u] = i < qn;
-                    e[u] = queue[ok[u] ? i : i0];
-                }
-                GV d[2][A];
-#pragma unroll
-                for (int u = 0; u < 2; ++u) {
-                    const int col = (int)(e[u].x & 0x0fffffffu);
-#pragma unroll
-                    for (int a = 0; a < A; ++a) {
-                        const SV cv = __ldcg(myCov[a] + col);
-                        if constexpr (Arith<SV>::kInt) {
-                            const int dd = (int)e[u].y - cv;
-                            d[u][a] = (ok[u] && myPart[a] >= 0 && dd > 0) ? (GV)dd : (GV)0;
-                        } else {
-                            const float dd = __uint_as_float(e[u].y) - cv;
-                            d[u][a] = (ok[u] && myPart[a] >= 0 && dd > 0.f) ? dd : 0.f;
-                        }
-                    }
-                }
-#pragma unroll
-                for (int u = 0; u < 2; ++u) {
-                    const int r = (int)(e[u].x >> 28);
-#pragma unroll
-                    for (int rr = 0; rr < R; ++rr)
-#pragma unroll
-                        for (int a = 0; a < A; ++a) acc[rr][a] += (r == rr) ? d[u][a] : (GV)0;
-                }
-            }
-            __syncwarp();
-            qn = 0;
-        };
-        // S streams through a ring in shared memory filled by asynchronous copies, kSparseStages - 1
-        // chunks ahead; every lane reads back only the 16-byte pieces it copied itself, so waiting
-        // for its own copy groups is all the synchronisation the ring needs
-        auto issue = [&](int base, int st) {
-            const int cc = base + lane;
-            if (cc < ld4) {
-#pragma unroll
-                for (int r = 0; r < R; ++r) async_copy16(ring + (st * R + r) * 32 + lane, rp[r] + cc);
-            }
-            asm volatile("cp.async.commit_group;" ::: "memory");
-        };
-#pragma unroll
-        for (int st = 0; st < kSparseStages - 1; ++st) issue(st * 32, st);
-        int stage = 0;
-        for (int base = 0; base < ld4; base += 32) {                // every lane runs every chunk: ballots below
-            const int cc = base + lane;
-            const bool inside = cc < ld4;
-            {
-                int ahead = stage + kSparseStages - 1;
-                if (ahead >= kSparseStages) ahead -= kSparseStages;
-                issue(base + (kSparseStages - 1) * 32, ahead);       // past the row's end: an empty group
-            }
-            asm volatile("cp.async.wait_group %0;" :: "n"(kSparseStages - 1) : "memory");
-            int4 t = make_int4(0, 0, 0, 0);
-            if (inside) t = shThr[cc];
-#pragma unroll
-            for (int r = 0; r < R; ++r) {
-                int4 s = make_int4(0, 0, 0, 0);
-                unsigned h = 0;
-                if (inside) {
-                    s = ring[(stage * R + r) * 32 + lane];
-                    if constexpr (Arith<SV>::kInt) {
-                        h = (s.x > t.x ? 1u : 0u) | (s.y > t.y ? 2u : 0u) | (s.z > t.z ? 4u : 0u) | (s.w > t.w ? 8u : 0u);
-                    } else {
-                        h = (__int_as_float(s.x) > __int_as_float(t.x) ? 1u : 0u) | (__int_as_float(s.y) > __int_as_float(t.y) ? 2u : 0u) |
-                            (__int_as_float(s.z) > __int_as_float(t.z) ? 4u : 0u) | (__int_as_float(s.w) > __int_as_float(t.w) ? 8u : 0u);
-                    }
-                }
-                if (__any_sync(0xffffffffu, h != 0)) {
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const bool mine = (h >> e) & 1u;
-                        const unsigned m = __ballot_sync(0xffffffffu, mine);
-                        if (mine) {
-                            const int sv = e == 0 ? s.x : (e == 1 ? s.y : (e == 2 ? s.z : s.w));
-                            queue[qn + __popc(m & below)] = make_uint2((unsigned)(cc * 4 + e) | ((unsigned)r << 28), (unsigned)sv);
-                        }
-                        qn += __popc(m);
-                    }
-                    if (qn > kSparseQueue - 128) { hits += qn; drain(); }
-                }
-            }
-            if (++stage == kSparseStages) stage = 0;
-        }
-        asm volatile("cp.async.wait_group 0;" ::: "memory");
+        sparse_stream<SV, A>(w, rp, R, acc, hits, qn);
         const int gNext = __shfl_sync(0xffffffffu, gDrawn, 0);
         int rowNext[R];
 #pragma unroll
@@ -836,14 +970,14 @@ __device__ __noinline__ void sweep_class_sparse(const GreedyParams<SV> &prm, int
                 rowNext[r] = __ldcg(cand + (k < nR ? k : nR - 1));
             }
         }
-        if (qn) { hits += qn; drain(); }
+        if (qn) { hits += qn; sparse_drain<SV, A>(w, qn, acc); }
 #pragma unroll
         for (int r = 0; r < R; ++r) {
 #pragma unroll
             for (int a = 0; a < A; ++a) {
                 GV t = acc[r][a];
-                for (int off = Pp; off < 32; off <<= 1) t += __shfl_xor_sync(0xffffffffu, t, off);
-                if (slot == 0 && k0 + r < nR && myPart[a] >= 0) G[(int64_t)myPart[a] * c.ld + rowOf[r]] = t;
+                for (int off = w.Pp; off < 32; off <<= 1) t += __shfl_xor_sync(0xffffffffu, t, off);
+                if (w.slot == 0 && k0 + r < nR && w.myPart[a] >= 0) G[(int64_t)w.myPart[a] * c.ld + rowOf[r]] = t;
             }
         }
         ++finished;
@@ -867,6 +1001,101 @@ __device__ __noinline__ void sweep_class_sparse(const GreedyParams<SV> &prm, int
     }
 }
 
+// Row-skipping threshold pass (the exact lazy rule for GreedyStep's argmax).  A stored gain of a block that has
+// grown since it was computed is an upper bound of the current gain (diminishing returns), so a row whose
+// stored gains lie below the floors of all listed blocks (shTheta[k] for parts[k]) cannot be needed before
+// those floors are lowered: it is left out and keeps its upper bounds.  Every other row is recomputed for all
+// listed blocks, exactly as in sweep_class_sparse.  Afterwards every stored gain of parts[k] at or above
+// shTheta[k] is exact: an entry that was not recomputed was below the floor and still is.
+// A ticket stands for kLazyRows consecutive entries of the candidate list, one per lane; the lanes look their
+// rows' stored gains up, and the warp then streams the rows that are needed, two at a time.
+template <typename SV, int A>
+__device__ __noinline__ void sweep_class_lazy(const GreedyParams<SV> &prm, int l, const ClassDesc c, int nR, int P,
+                                                 const int4 *shThr, const int32_t *parts, const typename Arith<SV>::GV *shTheta,
+                                                 uint2 *queue, int32_t *ticket, int32_t *done, int firstTicket)
+{
+    using GV = typename Arith<SV>::GV;
+    constexpr int R = kSparseRows;
+    SparseWarp<SV, A> w;
+    sparse_setup<SV, A>(w, prm, c, P, shThr, parts, queue);
+    const int lane = w.lane;
+    const int nTickets = (nR + kLazyRows - 1) / kLazyRows;
+    const SV *Sl = prm.S + c.sOff;
+    const int32_t *cand = prm.cand + c.row0;
+    GV *G = prm.gains + c.vOff;
+    unsigned hits = 0;
+    int finished = 0, rowsRead = 0, rowsSeen = 0;
+    int g = 0;
+    if (firstTicket >= 0) {
+        g = firstTicket + (threadIdx.x >> 5);
+    } else {
+        if (lane == 0) g = atomicAdd(ticket, 1);
+        g = __shfl_sync(0xffffffffu, g, 0);
+    }
+    while (g < nTickets) {
+        int gDrawn = 0;
+        if (lane == 0) gDrawn = atomicAdd(ticket, 1);               // (the next ticket: in flight under this one's work)
+        const int k = g * kLazyRows + lane;
+        const int v = k < nR ? __ldcg(cand + k) : -1;
+        bool need = false;
+        if (v >= 0) {
+            for (int k0 = 0; k0 < P; k0 += 4) {                     // four independent look-ups at a time
+                GV b[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) b[u] = __ldcg(G + (int64_t)parts[k0 + u < P ? k0 + u : 0] * c.ld + v);
+#pragma unroll
+                for (int u = 0; u < 4; ++u) need = need || (k0 + u < P && b[u] >= shTheta[k0 + u]);
+            }
+        }
+        unsigned mask = __ballot_sync(0xffffffffu, need);
+        rowsSeen += __popc(__ballot_sync(0xffffffffu, v >= 0));
+        while (mask) {
+            const int i0 = __ffs(mask) - 1;
+            mask &= mask - 1;
+            int i1 = i0, nRows = 1;
+            if (mask) { i1 = __ffs(mask) - 1; mask &= mask - 1; nRows = 2; }
+            int rowOf[R];
+            rowOf[0] = __shfl_sync(0xffffffffu, v, i0);
+            rowOf[1] = __shfl_sync(0xffffffffu, v, i1);
+            const int4 *rp[R];
+#pragma unroll
+            for (int r = 0; r < R; ++r) rp[r] = reinterpret_cast<const int4 *>(Sl + (int64_t)rowOf[r] * c.ld);
+            GV acc[R][A];
+#pragma unroll
+            for (int r = 0; r < R; ++r)
+#pragma unroll
+                for (int a = 0; a < A; ++a) acc[r][a] = 0;
+            int qn = 0;
+            sparse_stream<SV, A>(w, rp, nRows, acc, hits, qn);
+            if (qn) { hits += qn; sparse_drain<SV, A>(w, qn, acc); }
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+#pragma unroll
+                for (int a = 0; a < A; ++a) {
+                    GV t = acc[r][a];
+                    for (int off = w.Pp; off < 32; off <<= 1) t += __shfl_xor_sync(0xffffffffu, t, off);
+                    if (w.slot == 0 && r < nRows && w.myPart[a] >= 0) G[(int64_t)w.myPart[a] * c.ld + rowOf[r]] = t;
+                }
+            }
+            rowsRead += nRows;
+        }
+        ++finished;
+        g = __shfl_sync(0xffffffffu, gDrawn, 0);
+    }
+    if (finished > 0) {
+        __syncwarp();
+        if (lane == 0) {
+            atomicAdd(&prm.phaseNs[10], (unsigned long long)rowsRead);
+            atomicAdd(&prm.phaseNs[11], (unsigned long long)(rowsSeen - rowsRead));
+            atomicAdd(&prm.phaseNs[12], (unsigned long long)rowsRead * (unsigned long long)c.ld * sizeof(SV));
+            if (done != nullptr) {
+                __threadfence();                                    // the gains are in place before the tickets count as done
+                atomicAdd(done, finished);
+            }
+        }
+    }
+}
+
 // The sweep of greedy step `step`, run by every CTA of the launch (kSweepThreads threads each).
 template <typename SV>
 __device__ __forceinline__ void sweep_step(const GreedyParams<SV> &prm, int step, int4 *shCover)
@@ -874,6 +1103,7 @@ __device__ __forceinline__ void sweep_step(const GreedyParams<SV> &prm, int step
     using GV = typename Arith<SV>::GV;
     __shared__ long long shF[kMaxSweepBatch];
     __shared__ int32_t shParts[kSparseMax];
+    __shared__ GV shTheta[kLazyBlocks];
     __shared__ int shTicket[kSweepThreads / 32];
     __shared__ GV shPart[kSweepThreads];
     __shared__ int shGo;
@@ -893,7 +1123,8 @@ __device__ __forceinline__ void sweep_step(const GreedyParams<SV> &prm, int step
         __syncthreads();
         for (int s = threadIdx.x; s < nS; s += blockDim.x) {
             const int ls = prm.sweepList[(int64_t)par * prm.L + s];
-            const int Rs = prm.sweepMode[ls] ? kSparseRows : rows_per_group(prm.sweepN[ls]);
+            const int ms = prm.sweepMode[ls];
+            const int Rs = ms == 2 ? kLazyRows : (ms ? kSparseRows : rows_per_group(prm.sweepN[ls]));
             const int groups = (prm.nR[ls] + Rs - 1) / Rs;
             if (*(volatile int32_t *)&prm.rowCtr[ls] < groups) {
                 int dist = s - start;
@@ -917,10 +1148,17 @@ __device__ __forceinline__ void sweep_step(const GreedyParams<SV> &prm, int step
             // threshold pass: one vector in shared memory, the blocks' coverage stays in global memory
             const int4 *thr = reinterpret_cast<const int4 *>(prm.thr + c.vOff / prm.W);
             for (int i = threadIdx.x; i < ld4; i += blockDim.x) shCover[i] = thr[i];
-            if (threadIdx.x < P) shParts[threadIdx.x] = parts[threadIdx.x];
+            const bool lazy = prm.sweepMode[l] == 2;
+            if (threadIdx.x < P) {
+                shParts[threadIdx.x] = parts[threadIdx.x];
+                if (lazy) shTheta[threadIdx.x] = prm.sweepTheta[(int64_t)l * kLazyBlocks + threadIdx.x];
+            }
             __syncthreads();
             uint2 *queue = reinterpret_cast<uint2 *>(reinterpret_cast<char *>(shCover) + thr_bytes_aligned(c.ld * (int)sizeof(SV)) + (threadIdx.x >> 5) * kSparseWarpBytes);
-            if (P <= 32) sweep_class_sparse<SV, 1>(prm, l, c, nR, P, shCover, shParts, queue, &prm.rowCtr[l], nullptr, -1);
+            if (lazy) {
+                if (P <= 32) sweep_class_lazy<SV, 1>(prm, l, c, nR, P, shCover, shParts, shTheta, queue, &prm.rowCtr[l], nullptr, -1);
+                else sweep_class_lazy<SV, 2>(prm, l, c, nR, P, shCover, shParts, shTheta, queue, &prm.rowCtr[l], nullptr, -1);
+            } else if (P <= 32) sweep_class_sparse<SV, 1>(prm, l, c, nR, P, shCover, shParts, queue, &prm.rowCtr[l], nullptr, -1);
             else sweep_class_sparse<SV, 2>(prm, l, c, nR, P, shCover, shParts, queue, &prm.rowCtr[l], nullptr, -1);
         } else {
             const int4 *cov = reinterpret_cast<const int4 *>(prm.cover + c.vOff);
@@ -1009,6 +1247,7 @@ __device__ __forceinline__ void fold_pending(int4 *dst, const int4 *scratch, int
 // the candidate list with its inverse, the dataset indices of the class's samples and the chain's loop
 // state (keep[0] = samples left, keep[1] = next block) stay in shared memory between chains, so that a
 // pick waits for one trip to memory only -- the loads of the stored gains, served by L2 (ld.cg).
+constexpr int kPickMiss = -2;      // shPick: the best stored gain was not known to be exact
 template <typename SV>
 __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, int round, int4 *scratch, int scratchBytes,
                                            int own = 0, int *keep = nullptr)
@@ -1122,25 +1361,47 @@ __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, i
         if (warp == 0) {
             bestG = lane < kSelectThreads / 32 ? shG[lane] : (GV)0;
             bestV = lane < kSelectThreads / 32 ? shV[lane] : INT_MAX;
+            // The least of the warps' best stored gains: at least one unassigned sample per warp lies at or above it,
+            // so a later row-skipping pass with this floor recomputes the few dozen best-placed candidates of the block.
+            FV low = bestV != INT_MAX ? (FV)bestG : highest_value<FV>();
             for (int off = 16; off > 0; off >>= 1) {
                 GV oG = __shfl_xor_sync(0xffffffffu, bestG, off);
                 int oV = __shfl_xor_sync(0xffffffffu, bestV, off);
+                const FV oLow = __shfl_xor_sync(0xffffffffu, low, off);
+                if (oLow < low) low = oLow;
                 if (oV != INT_MAX && (bestV == INT_MAX || oG > bestG || (oG == bestG && oV < bestV))) { bestG = oG; bestV = oV; }
             }
             if (lane == 0) {
                 shPick = bestV;
-                // block j has received a sample: value, room, and its stored gains are now out of date
-                if (bestV != INT_MAX) {
+                if (bestV != INT_MAX && j < kLazyBlocks && (FV)bestG < shPlan.floorv[j]) {
+                    // A miss: the best stored gain lies below the floor of the block's last pass, so it may be an
+                    // upper bound only.  Nothing is picked; the block asks for a pass over every row.
+                    shPick = kPickMiss;
+                    shPlan.open[j] = (uint8_t)(shPlan.open[j] | 2);
+                    shPlan.theta[j] = lowest_value<FV>();
+                    shPlan.lazyMisses += 1;
+                    atomicAdd(&prm.phaseNs[9], 1ull);
+                    prm.valid[(int64_t)l * prm.W + j] = 0;
+                } else if (bestV != INT_MAX) {
+                    // block j has received a sample: value, room, and its stored gains are now out of date
                     shPlan.f[j] += (FV)bestG;
                     const int room = shPlan.room[j] - 1;
                     shPlan.room[j] = room;
                     shPlan.open[j] = (uint8_t)((room > 0 ? 1 : 0) | 2);
+                    if (j < kLazyBlocks) shPlan.theta[j] = low;
                     prm.valid[(int64_t)l * prm.W + j] = 0;     // (plan_decide, same lane, may set it again)
                 }
             }
             __syncwarp();
         }
         __syncthreads();
+        if (shPick == kPickMiss) {
+            // (the chain ends here: its last act is to schedule the pass this block needs)
+            if (warp == 0) plan_decide(prm, l, c, nR, round + 1, shPlan, &shPre);
+            __syncthreads();
+            j = shPlan.nextJ;
+            break;
+        }
         if (threadIdx.x == 0 && chainLen < kSparseMax) shChain[chainLen] = j;
         ++chainLen;
         const int vstar = shPick;
@@ -1201,6 +1462,7 @@ __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, i
         if (nR == 0 || j < 0 || shPlan.needSweep) break;
     }
     if (keep && threadIdx.x == 0) { keep[0] = nR; keep[1] = j; }     // (j = -1 after an inconsistency: the class is given up)
+    if (!res) plan_store_lazy(prm, l, shPlan);                       // (a CTA that owns its class keeps this state in shared memory)
     if (pendDst) fold_pending<SV>(pendDst, scratch, ld4, thrAcc);
     if (shPlan.needSweep && shPlan.sweepSparse) {
         // threshold of the coming pass: element-wise minimum of the listed blocks' coverage vectors
@@ -1427,6 +1689,7 @@ __device__ __forceinline__ void async_sweep_cta(const GreedyParams<SV> &prm, int
     using GV = typename Arith<SV>::GV;
     __shared__ long long shF[kMaxSweepBatch];
     __shared__ int32_t shParts[kSparseMax];
+    __shared__ GV shTheta[kLazyBlocks];
     __shared__ int shTicket[kSweepThreads / 32];
     __shared__ GV shPart[kSweepThreads];
     __shared__ unsigned long long shBest;
@@ -1496,12 +1759,14 @@ __device__ __forceinline__ void async_sweep_cta(const GreedyParams<SV> &prm, int
             shInfo[2] = myB.z;                                      // unassigned samples
             shInfo[3] = myB.w & 0xff;                               // blocks
             shInfo[4] = (myB.w >> 8) & 0xff;                        // warps per row group
-            shInfo[5] = (myB.w >> 16) & 1;                          // threshold pass?
+            shInfo[5] = (myB.w >> 16) & 3;                          // 1 = threshold pass, 2 = one that skips rows
         }
         if (threadIdx.x < kSparseMax) {
             int bp = ld_volatile32(parts + threadIdx.x);
             if (bp < 0 || bp >= prm.W) bp = 0;                      // (beyond the list, or a read that raced with an update)
             shParts[threadIdx.x] = bp;
+        } else if (threadIdx.x >= 256 && threadIdx.x < 256 + kLazyBlocks) {
+            shTheta[threadIdx.x - 256] = *(const volatile GV *)&prm.sweepTheta[(int64_t)l * kLazyBlocks + (threadIdx.x - 256)];
         }
         if constexpr (Arith<SV>::kInt) {
             if (threadIdx.x >= 128 && threadIdx.x < 128 + kMaxSweepBatch)
@@ -1551,8 +1816,12 @@ __device__ __forceinline__ void async_sweep_cta(const GreedyParams<SV> &prm, int
         int32_t *done = &prm.sync[l].done;
         if (mode) {
             P = shInfo[3];
+            if (P < 1 || P > kSparseMax) P = 1;
             uint2 *queue = reinterpret_cast<uint2 *>(reinterpret_cast<char *>(shCover) + thr_bytes_aligned(c.ld * (int)sizeof(SV)) + (threadIdx.x >> 5) * kSparseWarpBytes);
-            if (P <= 32) sweep_class_sparse<SV, 1>(prm, l, c, nR, P, shCover, shParts, queue, ticket, done, first);
+            if (mode == 2) {
+                if (P <= 32) sweep_class_lazy<SV, 1>(prm, l, c, nR, P, shCover, shParts, shTheta, queue, ticket, done, first);
+                else sweep_class_lazy<SV, 2>(prm, l, c, nR, P, shCover, shParts, shTheta, queue, ticket, done, first);
+            } else if (P <= 32) sweep_class_sparse<SV, 1>(prm, l, c, nR, P, shCover, shParts, queue, ticket, done, first);
             else sweep_class_sparse<SV, 2>(prm, l, c, nR, P, shCover, shParts, queue, ticket, done, first);
         } else {
             switch (P) {
@@ -1645,6 +1914,11 @@ static rcd_status run_greedy(rcd_ctx *ctx, const Sizes &sz, const Workspace &ws,
     prm.one = 1u;
     prm.sparseMinMembers = ctx->cfg.sweep_mode == 1 ? -1 : (ctx->cfg.threshold_from > 0 ? ctx->cfg.threshold_from : 8);
     prm.hitShift = ctx->cfg.threshold_hit_shift > 0 ? ctx->cfg.threshold_hit_shift : 5;
+    prm.floorv = (FV *)ws.floorv;
+    prm.theta = (FV *)ws.theta;
+    prm.sweepTheta = (GV *)ws.sweepTheta;
+    prm.lazyStat = ws.lazyStat;
+    prm.lazyFrom = (ctx->cfg.lazy_mode != 1 || ctx->cfg.sweep_mode == 1) ? -1 : (ctx->cfg.lazy_from > 0 ? ctx->cfg.lazy_from : 8);
     prm.sync = ws.sync;
     prm.tickets = ws.tickets;
     prm.sweepF = ws.sweepF;
@@ -1718,7 +1992,7 @@ static rcd_status run_greedy(rcd_ctx *ctx, const Sizes &sz, const Workspace &ws,
 
     if (path == 3) RCD_CUDA(ctx, cudaMemsetAsync(ws.tickets, 0, (size_t)(sz.N + sz.L) * sizeof(int32_t), st));
     RCD_CUDA(ctx, cudaMemsetAsync(ws.nSweep, 0, 4 * sizeof(int32_t), st));
-    RCD_CUDA(ctx, cudaMemsetAsync(ws.phaseNs, 0, 8 * sizeof(unsigned long long), st));
+    RCD_CUDA(ctx, cudaMemsetAsync(ws.phaseNs, 0, kPhaseWords * sizeof(unsigned long long), st));
     ctx->phaseNsDev = ws.phaseNs;
     RCD_CUDA(ctx, cudaMemsetAsync(ws.stepBytes, 0, (size_t)(sz.maxM + 1) * sizeof(unsigned long long), st));
     RCD_CUDA(ctx, cudaMemsetAsync(ws.stepOps, 0, (size_t)(sz.maxM + 1) * sizeof(unsigned long long), st));

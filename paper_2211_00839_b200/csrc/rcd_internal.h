@@ -15,6 +15,8 @@ constexpr int kMaxSweepBatch = 8;          // blocks refreshed by one dense pass
 constexpr int kSparseMax = 64;             // blocks refreshed by one threshold pass over S
 constexpr int kSweepThreads = 512;         // sweep CTA: 16 warps, one CTA per SM
 constexpr int kSelectThreads = 512;        // pick/update CTA: one per class
+constexpr int kLazyBlocks = 64;            // row skipping keeps a floor per block for classes of up to this many blocks
+constexpr int kPhaseWords = 16;            // 64-bit counters a greedy launch keeps (phase clocks, barrier, pass statistics)
 constexpr size_t kAlign = 256;
 
 // Device-side status bits (OR-ed into the status word).
@@ -114,6 +116,10 @@ struct Workspace {
     ClassSync *sync;        // [L] asynchronous kernel: hand-off words
     int32_t *tickets;       // [N + L] asynchronous kernel: one ticket counter per (class, sweep number), never reused
     int32_t *sizesSorted;   // [L] class sizes, ascending
+    void *floorv;           // [L][kLazyBlocks] per block: every stored gain at or above it is exact (int64 / double)
+    void *theta;            // [L][kLazyBlocks] per block: floor its next row-skipping pass will establish
+    void *sweepTheta;       // [L][kLazyBlocks] floors of the blocks the class's next pass lists, in list order (int64 / fp32)
+    int32_t *lazyStat;      // [L][4] row-skipping passes of the class, misses, members needed before rows are skipped
     long long *sweepF;      // [L][8] asynchronous kernel, int8 features: f of the first blocks in the sweep's list
     int32_t *sweepList;     // [3][L] classes that sweep in a step (three lists in rotation)
     int32_t *nSweep;        // [3] (+1 pad)

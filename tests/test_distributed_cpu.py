@@ -34,6 +34,17 @@ def _worker(rank, world, port, out_dir):
 
         got = partition_sharded(wl.features, wl.labels, wl.capacities, wl.L, single_device)
         np.save(os.path.join(out_dir, "rank%d.npy" % rank), got)
+
+        # the tensor form (the one the GPU path uses, here on CPU tensors over gloo)
+        import torch
+        from paper_2211_00839_b200.distributed import partition_sharded_tensors
+
+        def single_device_t(f, y, caps, L):
+            return torch.from_numpy(orc.partition(f.numpy(), y.numpy(), caps, L, variant="incremental").assignment)
+
+        got_t = partition_sharded_tensors(torch.from_numpy(wl.features), torch.from_numpy(wl.labels), wl.capacities, wl.L,
+                                          single_device_t)
+        np.save(os.path.join(out_dir, "rank%d_t.npy" % rank), got_t.numpy())
     finally:
         dist.destroy_process_group()
 
@@ -51,3 +62,5 @@ def test_two_ranks_reproduce_the_single_process_partition(tmp_path):
     for r in range(2):
         got = np.load(os.path.join(str(tmp_path), "rank%d.npy" % r))
         assert np.array_equal(got, want)
+        got_t = np.load(os.path.join(str(tmp_path), "rank%d_t.npy" % r))
+        assert np.array_equal(got_t, want)

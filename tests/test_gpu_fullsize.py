@@ -43,10 +43,10 @@ def orc():
     return rcd_oracle
 
 
-def run_full(rcd, wl):
+def run_full(rcd, wl, **cfg):
     import torch
     dev = torch.device("cuda", 0)
-    with rcd.Context(0) as ctx:
+    with rcd.Context(0, **cfg) as ctx:
         X = rcd.features_to_torch(wl.features, device=dev)
         y = torch.from_numpy(wl.labels).to(dev)
         M = wl.N // wl.L
@@ -159,7 +159,7 @@ def test_c5_many_classes_int8(rcd, orc):
 
 # ----------------------------------------------------------------------------- whole trajectories at full size
 
-def _check_against_digests(rcd, orc, name):
+def _check_against_digests(rcd, orc, name, **cfg):
     """Every class of a full-size int8 configuration, bit for bit: block of every sample, pick order and
     block values must hash to the digest the oracle's own run of that class produced (stored under
     tests/golden by a script that calls only the oracle)."""
@@ -168,7 +168,7 @@ def _check_against_digests(rcd, orc, name):
     gold = json.load(open(os.path.join(GOLDEN, "fullsize_digests.json")))[name]
     wl = make_workload(name)
     assert gm.input_digest(wl) == gold["inputs"], "the generator no longer produces the inputs the digests were written for"
-    a, o, v, recomputed = run_full(rcd, wl)
+    a, o, v, recomputed = run_full(rcd, wl, **cfg)
     groups = check_invariants(orc, wl, a, o)
     assert np.array_equal(v, recomputed)
     assert int(v.sum()) == gold["total_objective"]
@@ -194,6 +194,11 @@ def _check_against_digests(rcd, orc, name):
 def test_c2_every_class_bit_exact(rcd, orc):
     """All 10 classes of C2 (5000 picks each) in the configuration bench.py times."""
     _check_against_digests(rcd, orc, "C2")
+
+
+def test_c2_every_class_bit_exact_with_lazy_evaluation(rcd, orc):
+    """The same 10 x 5000 picks with row-skipping passes switched on."""
+    _check_against_digests(rcd, orc, "C2", lazy_mode=1)
 
 
 def test_c5_every_class_bit_exact(rcd, orc):

@@ -339,6 +339,56 @@ def test_threshold_passes_float(rcd, orc):
     check_float(rcd, orc, wl, sweep_mode=1)
 
 
+# ----------------------------------------------------------------------------- exact lazy evaluation (row-skipping passes)
+
+@pytest.mark.parametrize("path", [0, 1, 2, 3])
+def test_lazy_evaluation_int8_exact(rcd, orc, path):
+    """Row-skipping threshold passes (stored gains as upper bounds, a floor per block): rows are skipped, some picks
+    miss and are answered by a pass over every row, and every pick is still the oracle's."""
+    from paper_2211_00839_b200.workloads import make_workload
+    wl = make_workload("C2", L=3, M=1200)
+    ref = orc.partition(wl.features, wl.labels, wl.capacities, wl.L, variant="incremental")
+    a, o, v, prof = run_with_profile(rcd, wl, greedy_path=path, lazy_mode=1, lazy_from=2)
+    assert prof["lazy_sweeps"] > 0 and prof["lazy_rows_skipped"] > prof["lazy_rows"] > 0 and prof["lazy_misses"] > 0
+    assert np.array_equal(a, ref.assignment) and np.array_equal(o, ref.order) and np.array_equal(v, ref.part_values)
+    a0, o0, v0, prof0 = run_with_profile(rcd, wl, greedy_path=path)
+    assert prof0["lazy_sweeps"] == 0 and prof0["lazy_rows"] == 0
+    assert prof["sweep_bytes"] < prof0["sweep_bytes"]
+
+
+@pytest.mark.parametrize("lazy_from", [1, 8])
+def test_lazy_evaluation_many_blocks_and_ragged_classes_exact(rcd, orc, lazy_from):
+    """W = 64 (two blocks per lane in a pass), classes of unequal sizes, more classes than pick CTAs."""
+    from paper_2211_00839_b200.workloads import Workload, make_workload
+    wl = make_workload("C5", L=3, M=1300, d=128)
+    ref = orc.partition(wl.features, wl.labels, wl.capacities, wl.L, variant="incremental")
+    a, o, v, prof = run_with_profile(rcd, wl, lazy_mode=1, lazy_from=lazy_from)
+    assert prof["lazy_sweeps"] > 0
+    assert np.array_equal(a, ref.assignment) and np.array_equal(o, ref.order) and np.array_equal(v, ref.part_values)
+    base = make_workload("C2", L=40, M=300, d=64)
+    rng = np.random.default_rng(17)
+    keep = np.ones(base.N, bool)
+    for l in range(base.L):
+        ids = np.nonzero(base.labels == l)[0]
+        keep[ids[:int(rng.integers(0, 200))]] = False
+    wl = Workload("ragged-lazy", "int8", np.ascontiguousarray(base.features[keep]), np.ascontiguousarray(base.labels[keep]),
+                  base.capacities, base.L, base.W)
+    for path in (2, 3):
+        check_exact(rcd, orc, wl, greedy_path=path, lazy_mode=1, lazy_from=lazy_from)
+
+
+def test_lazy_evaluation_float(rcd, orc):
+    from paper_2211_00839_b200.workloads import make_workload
+    wl = make_workload("C3", L=2, M=900, d=512)
+    with rcd.Context(0, profile=1, lazy_mode=1, lazy_from=2) as ctx:
+        X, y = to_device(rcd, wl)
+        ctx.rcd_partition(X, y, wl.capacities, wl.L)
+        ctx.sync_status()
+        assert ctx.profile()["lazy_sweeps"] > 0
+    check_float(rcd, orc, wl, lazy_mode=1, lazy_from=2)
+    check_float(rcd, orc, wl, lazy_mode=1, greedy_path=2)
+
+
 # ----------------------------------------------------------------------------- objective
 
 @pytest.mark.parametrize("name,L,M,d", [("C1", 2, 200, 64), ("C5", 3, 300, 128), ("C4", 3, 250, 96)])
