@@ -218,7 +218,7 @@ def run_ours(args):
     Xd, yd = Xh.to(dev), yh.to(dev)
     kind = rcd.RCD_SIM_GAUSSIAN if args.similarity == "gaussian" else rcd.RCD_SIM_DOT
     ctx = rcd.Context(local, sweep_batch_max=args.sweep_batch, profile=1, greedy_path=args.greedy_path, similarity_kind=kind,
-                      async_group=args.async_group, async_help_min=args.async_help_min, lazy_mode=args.lazy_mode, lazy_from=args.lazy_from,
+                      async_group=args.async_group, async_help_min=args.async_help_min, lazy_mode=args.lazy_mode, lazy_from=args.lazy_from, dense_ring=args.dense_ring,
                       objective=rcd.RCD_OBJ_GRAPH_CUT if args.objective == "cut" else rcd.RCD_OBJ_FACILITY)
 
     def barrier():
@@ -324,12 +324,12 @@ def run_ours(args):
     default_setup = args.classes == 0 and args.sweep_batch in (0, 8) and args.async_group == 0 and args.async_help_min == 0 and args.similarity == "dot"
     loop_s = prof["greedy_ms"] * 1e-3
     achieved = prof["sweep_bytes"] / loop_s / 1e9 if loop_s > 0 else 0.0
+    sms = torch.cuda.get_device_properties(local).multi_processor_count
+    path = args.greedy_path if args.greedy_path else (3 if wl.L * 4 <= sms else 4)
     if args.objective != "facility":
         kernel_name = "cut_chain_kernel"
-    elif args.greedy_path == 3 or (args.greedy_path == 0 and wl.L * 4 <= torch.cuda.get_device_properties(local).multi_processor_count):
-        kernel_name = "greedy_async_kernel"
     else:
-        kernel_name = "greedy_persistent_kernel" if args.greedy_path != 1 else "sweep_kernel"
+        kernel_name = {1: "sweep_kernel", 2: "greedy_persistent_kernel", 3: "greedy_async_kernel", 4: "greedy_owner_kernel"}[path]
     # S larger than L2: the sweeps stream from HBM (peak: the measured copy bandwidth); S inside L2: they stream from
     # L2 (peak: this library's read-only sweep yardstick over an L2-resident buffer, measured in this run)
     bound = "l2" if fits_l2 else "hbm"
@@ -406,7 +406,8 @@ def run_ours(args):
                                 sweep_phases_ms=prof["persistent_sweep_ns"] * 1e-6, pick_phases_ms=prof["persistent_pick_ns"] * 1e-6,
                                 async_lull_ms=prof["async_lull_ns"] * 1e-6, async_visits=int(prof["async_visits"]), async_attempts=int(prof["async_attempts"]),
                                 lazy_sweeps=int(prof["lazy_sweeps"]), lazy_misses=int(prof["lazy_misses"]), lazy_rows=int(prof["lazy_rows"]),
-                                lazy_rows_skipped=int(prof["lazy_rows_skipped"])),
+                                lazy_rows_skipped=int(prof["lazy_rows_skipped"]),
+                                threshold_pass_ms=prof["threshold_pass_ns"] * 1e-6, threshold_pass_gb=prof["threshold_pass_bytes"] * 1e-9),
               "similarity": similarity,
               "e2e": {"value": e2e_value, "unit": "samples/s", "h2d_bytes_per_step": int(h2d),
                       "d2h_bytes_per_step": int(d2h), "wall_ms_per_step": e2e_wall_ms / args.steps},
@@ -440,12 +441,13 @@ def main():
     ap.add_argument("--similarity", default="dot", choices=["dot", "gaussian"], help="similarity of Section 4 item 2")
     ap.add_argument("--objective", default="facility", choices=["facility", "cut"], help="submodular function of Section 4 item 2")
     ap.add_argument("--greedy-path", type=int, default=0,
-                    help="0 = chosen by the library, 1 = two launches per round, 2 = one launch with rounds, 3 = one launch, asynchronous classes")
+                    help="0 = chosen by the library, 1 = two launches per round, 2 = one launch with rounds, 3 = one launch, asynchronous classes, 4 = one CTA per class")
     ap.add_argument("--async-help-min", type=int, default=0, help="greedy path 3: row groups left before other classes' CTAs help (0 = default)")
     ap.add_argument("--async-group", type=int, default=0, help="greedy path 3: sweeps served together (0 = library default)")
     ap.add_argument("--sharding", default="replicas", choices=["replicas", "classes"],
                     help="with --gpus N: one dataset per rank (weak scaling), or one dataset with its classes sharded over the ranks (strong scaling)")
     ap.add_argument("--lazy-mode", type=int, default=0, help="1 = threshold passes skip rows below the blocks' floors (exact lazy evaluation), 0 = every pass reads every row")
+    ap.add_argument("--dense-ring", type=int, default=0, help="0 = dense passes stream through shared-memory rings where they fit, 2 = never")
     ap.add_argument("--lazy-from", type=int, default=0, help="members a block needs before rows are skipped (0 = library default)")
     ap.add_argument("--ref-picks", type=int, default=150, help="picks per class in the CPU-oracle sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")

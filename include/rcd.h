@@ -77,12 +77,13 @@ typedef struct {
     int32_t sweep_batch_max;   /* blocks whose gains one pass over S may refresh: 1,2,4 or 8; 0 = default (8) */
     int32_t similarity_path;   /* 0 = tensor-core kernel when the shape allows, 2 = always the generic kernel */
     int32_t profile;           /* 0 off; 1 time the phases of rcd_partition; 2 also time every sweep launch */
-    int32_t greedy_path;       /* form of the greedy loop.  0 = choose: one cooperative launch when the device allows,
-                                  asynchronous classes (3) when there are at most a quarter as many classes as SMs,
-                                  else rounds (2);  1 = two launches per round (always used with profile 2);
-                                  2 = one launch, rounds of a sweep phase and a pick phase separated by grid barriers;
-                                  3 = one launch, every class cycles between sweep and picks on its own: some CTAs
-                                  only make picks, the others only sweep, so picks overlap other classes' sweeps.
+    int32_t greedy_path;       /* form of the greedy loop.  0 = choose: asynchronous classes (3) when there are at most a quarter
+                                  as many classes as SMs, else one CTA per class (4);  1 = two launches per round (always
+                                  used with profile 2);  2 = one cooperative launch, rounds of a sweep phase and a pick phase
+                                  separated by grid barriers;  3 = one cooperative launch, every class cycles between sweep and
+                                  picks on its own: some CTAs only make picks, the others only sweep, so picks overlap other
+                                  classes' sweeps;  4 = one launch, every CTA draws a class and runs it from its first pick
+                                  to its last (no barrier, no hand-off; picks of one SM overlap sweeps of the others).
                                   All forms make the same picks. */
     int32_t similarity_kind;   /* rcd_similarity_kind used by rcd_partition / rcd_objective (default RCD_SIM_DOT) */
     int32_t objective;         /* rcd_objective_kind used by rcd_partition / rcd_objective (default facility location) */
@@ -102,7 +103,9 @@ typedef struct {
                                   its block's floor is not made, the block gets a pass over every row instead.  Same picks
                                   either way; fewer bytes read, but each class waits longer for its short passes. */
     int32_t lazy_from;         /* members every out-of-date block must have before rows are skipped; 0 = default (8) */
-    int32_t reserved[3];       /* must be 0 */
+    int32_t dense_ring;        /* 0 = 8-block dense passes stream S through per-warp rings of asynchronous copies in shared
+                                  memory when the coverage vectors leave room for them; 2 = never (one register buffer ahead) */
+    int32_t reserved[2];       /* must be 0 */
 } rcd_config;
 
 /* Timings and counters of the last rcd_partition / rcd_partition_host on a context (profile >= 1). */
@@ -132,6 +135,8 @@ typedef struct {
     int64_t lazy_misses;            /* picks whose best stored gain lay below its block's floor (answered by a pass over every row) */
     int64_t lazy_rows;              /* rows of S those passes did read */
     int64_t lazy_rows_skipped;      /* rows they did not */
+    int64_t threshold_pass_ns;      /* one CTA per class: time the first CTA spent in threshold passes (part of persistent_sweep_ns) */
+    int64_t threshold_pass_bytes;   /* bytes of S and threshold vectors the (row-visiting) threshold passes had to read (part of sweep_bytes) */
 } rcd_profile;
 
 typedef struct rcd_ctx rcd_ctx;

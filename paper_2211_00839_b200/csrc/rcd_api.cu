@@ -108,6 +108,7 @@ size_t layout_workspace(void *base, rcd_feat_dtype dtype, const Sizes &sz, Works
     w.tickets = c.take<int32_t>(N + L);
     w.sweepF = c.take<long long>(L * 8);
     w.sizesSorted = c.take<int32_t>(L);
+    w.classOrder = c.take<int32_t>(L);
     w.floorv = c.take<unsigned char>(L * kLazyBlocks * 8);
     w.theta = c.take<unsigned char>(L * kLazyBlocks * 8);
     w.sweepTheta = c.take<unsigned char>(L * kLazyBlocks * 8);
@@ -310,7 +311,7 @@ rcd_status rcd_create(rcd_ctx **out, int cuda_device, const rcd_config *cfg)
             return RCD_ERR_INVALID_ARG;
         if (cfg->similarity_path != 0 && cfg->similarity_path != 2) return RCD_ERR_INVALID_ARG;
         if (cfg->profile < 0 || cfg->profile > 2) return RCD_ERR_INVALID_ARG;
-        if (cfg->greedy_path < 0 || cfg->greedy_path > 3) return RCD_ERR_INVALID_ARG;
+        if (cfg->greedy_path < 0 || cfg->greedy_path > 4) return RCD_ERR_INVALID_ARG;
         if (cfg->similarity_kind != RCD_SIM_DOT && cfg->similarity_kind != RCD_SIM_GAUSSIAN) return RCD_ERR_INVALID_ARG;
         if (cfg->objective != RCD_OBJ_FACILITY && cfg->objective != RCD_OBJ_GRAPH_CUT) return RCD_ERR_INVALID_ARG;
         if (cfg->sweep_mode != 0 && cfg->sweep_mode != 1) return RCD_ERR_INVALID_ARG;
@@ -319,7 +320,8 @@ rcd_status rcd_create(rcd_ctx **out, int cuda_device, const rcd_config *cfg)
         if (cfg->threshold_from < 0 || cfg->threshold_hit_shift < 0 || cfg->threshold_hit_shift > 30) return RCD_ERR_INVALID_ARG;
         if (cfg->lazy_mode != 0 && cfg->lazy_mode != 1) return RCD_ERR_INVALID_ARG;
         if (cfg->lazy_from < 0) return RCD_ERR_INVALID_ARG;
-        for (int i = 0; i < 3; ++i) if (cfg->reserved[i] != 0) return RCD_ERR_INVALID_ARG;
+        if (cfg->dense_ring != 0 && cfg->dense_ring != 2) return RCD_ERR_INVALID_ARG;
+        for (int i = 0; i < 2; ++i) if (cfg->reserved[i] != 0) return RCD_ERR_INVALID_ARG;
     }
     int count = 0;
     if (cudaGetDeviceCount(&count) != cudaSuccess || cuda_device < 0 || cuda_device >= count) {
@@ -409,6 +411,8 @@ rcd_status rcd_get_profile(rcd_ctx *ctx, rcd_profile *out)
         out->lazy_rows = (int64_t)ns[10];
         out->lazy_rows_skipped = (int64_t)ns[11];
         lazyBytes = (int64_t)ns[12];
+        out->threshold_pass_ns = (int64_t)ns[13];
+        out->threshold_pass_bytes = (int64_t)ns[14];
         out->persistent_sweep_ns = (int64_t)ns[0];
         out->persistent_pick_ns = (int64_t)ns[1];
         out->threshold_hits = (int64_t)ns[3];

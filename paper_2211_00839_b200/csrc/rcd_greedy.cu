@@ -100,6 +100,8 @@ struct GreedyParams {
     GV *sweepTheta;             // [L][kLazyBlocks] those floors for the blocks of the class's next pass, in list order
     int32_t *lazyStat;          // [L][4] row-skipping passes, misses
     int32_t lazyFrom;           // members every listed block must have before a pass skips rows (< 0: never)
+    int32_t denseRing;          // 8-block dense passes stream through shared-memory rings when the coverage vectors leave room
+    const int32_t *classOrder;  // [L] classes by descending size (the order in which the one-CTA-per-class loop draws them)
     const int32_t *sizesSorted; // [L] class sizes in ascending order
     int32_t minM;               // smallest non-empty class
     int32_t nonEmpty;           // classes that hold at least one sample
@@ -303,6 +305,7 @@ __device__ void plan_decide(const GreedyParams<SV> &prm, int l, const ClassDesc 
     else g = plan_globals(prm, l);
     int remaining = g.remaining;
     if constexpr (!Arith<SV>::kInt) remaining = classes_alongside(prm, c.M - nR);
+    if (prm.asyncMode == 2) remaining = 1;                   // the class has its CTA to itself
     int from = 0;
     if (lane == 0) {
         from = g.from;
@@ -415,7 +418,9 @@ __device__ void plan_decide(const GreedyParams<SV> &prm, int l, const ClassDesc 
         prm.sweepN[l] = P;
         prm.sweepCS[l] = CS;
         prm.rowCtr[l] = 0;
-        if (prm.asyncMode) {
+        if (prm.asyncMode == 2) {
+            // (one CTA runs the class from its first pick to its last: nothing to publish)
+        } else if (prm.asyncMode) {
             ClassSync &sy = prm.sync[l];                   // published with the epoch by the caller
             sy.nGroups = (int32_t)nGroups;
             sy.nR = nR;
@@ -436,6 +441,7 @@ __device__ void plan_decide(const GreedyParams<SV> &prm, int l, const ClassDesc 
         } else {
             atomicAdd(&prm.stepBytes[nextStep], (unsigned long long)((int64_t)nR * c.ld + (int64_t)(sparse ? 1 : n) * c.ld) * sizeof(SV));
             atomicAdd(&prm.stepOps[nextStep], (unsigned long long)((int64_t)nR * c.M * (sparse ? 1 : n)));
+            if (sparse) atomicAdd(&prm.phaseNs[14], (unsigned long long)((int64_t)nR * c.ld + c.ld) * sizeof(SV));
         }
     }
 }
@@ -471,7 +477,7 @@ __global__ void __launch_bounds__(kSelectThreads, 4) init_kernel(GreedyParams<SV
         prm.sparseElems[l] = 0;
         prm.hitCount[l] = 0;
         if (c.M > 0) atomicAdd(&prm.nSweep[3], 1);         // classes still to finish
-        if (prm.asyncMode) {
+        if (prm.asyncMode == 1) {
             prm.sync[l].epoch = c.M > 0 ? 0 : 1;           // sweep 0 is published by this kernel
             prm.sync[l].done = 0;
             prm.sync[l].seq = l;
@@ -577,11 +583,24 @@ __device__ __forceinline__ void accumulate_chunk(uint32_t one, const int4 (&s)[R
 // from the class's ticket counter and its warps take interleaved 128-column chunks of those rows,
 // so that a sweep with few rows left still spreads over every warp of the GPU.  Per-warp partial
 // sums meet in shared memory and are added in warp order (fixed, reproducible).
-template <typename SV, int P, int R>
+// 16 bytes global -> shared without passing through registers (completion: cp.async.wait_group).
+__device__ __forceinline__ void async_copy16(int4 *smemDst, const int4 *src)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" :: "r"((uint32_t)__cvta_generic_to_shared(smemDst)), "l"(src) : "memory");
+}
+
+// kRing: the rows stream through a per-warp ring of asynchronous copies in shared memory (`ring`, kDenseStages
+// chunks of R rows per warp) instead of one register buffer ahead: a warp of a CTA that sweeps a class alone has
+// a few hundred instructions of work per chunk, far less than a trip to memory takes, so it needs several
+// chunks in flight to keep its issue slots busy.  Each lane reads back only the pieces it copied itself.
+constexpr int kDenseStages = 4;
+__host__ __device__ inline int dense_ring_bytes(int R) { return (kSweepThreads / 32) * kDenseStages * R * 512; }
+
+template <typename SV, int P, int R, bool kRing = false>
 __device__ __forceinline__ void sweep_class(const GreedyParams<SV> &prm, int l, const ClassDesc &c, int nR, int CS,
                                             const int4 *shCover, const long long *shF, const int32_t *parts,
                                             int *shTicket, typename Arith<SV>::GV *shPart,
-                                            int32_t *ticket, int32_t *done, int firstTicket)
+                                            int32_t *ticket, int32_t *done, int firstTicket, int4 *ring = nullptr)
 {
     using GV = typename Arith<SV>::GV;
     using AccT = typename std::conditional<Arith<SV>::kInt, uint32_t, float>::type;
@@ -627,6 +646,39 @@ __device__ __forceinline__ void sweep_class(const GreedyParams<SV> &prm, int l, 
         }
         GV total;
         const int first = wIn * 32 + lane;
+        // (kRing) this lane's chunks c0, c0 + stride, ... below cEnd through the warp's ring, kDenseStages - 1 ahead
+        auto ring_stream = [&](int c0, int cEnd, AccT (&acc)[NA]) {
+            int4 *rg = ring + (threadIdx.x >> 5) * (kDenseStages * R * 32) + lane;
+            int ci = c0;
+#pragma unroll
+            for (int st = 0; st < kDenseStages - 1; ++st) {
+                if (ci < cEnd) {
+#pragma unroll
+                    for (int r = 0; r < R; ++r) async_copy16(rg + (st * R + r) * 32, rp[r] + ci);
+                }
+                asm volatile("cp.async.commit_group;" ::: "memory");
+                ci += stride;
+            }
+            int stage = 0;
+            for (int cc = c0; cc < cEnd; cc += stride) {
+                int ahead = stage + kDenseStages - 1;
+                if (ahead >= kDenseStages) ahead -= kDenseStages;
+                if (ci < cEnd) {
+#pragma unroll
+                    for (int r = 0; r < R; ++r) async_copy16(rg + (ahead * R + r) * 32, rp[r] + ci);
+                }
+                asm volatile("cp.async.commit_group;" ::: "memory");
+                ci += stride;
+                asm volatile("cp.async.wait_group %0;" :: "n"(kDenseStages - 1) : "memory");
+                int4 sr[R];
+#pragma unroll
+                for (int r = 0; r < R; ++r) sr[r] = rg[(stage * R + r) * 32];
+                accumulate_chunk<SV, P, R>(prm.one, sr, shCover, ld4, cc, acc);
+                if (++stage == kDenseStages) stage = 0;
+            }
+            asm volatile("cp.async.wait_group 0;" ::: "memory");
+        };
+        (void)ring_stream;
         if constexpr (Arith<SV>::kInt) {
             // sum_i max(S[v][i], cover[i]) in unsigned 32-bit partials (every term is in [0, 2^31)),
             // widened to 64 bits every segIters iterations; the gain is that sum minus f_p.
@@ -640,7 +692,9 @@ __device__ __forceinline__ void sweep_class(const GreedyParams<SV> &prm, int l, 
                 for (int i = 0; i < NA; ++i) acc[i] = 0u;
                 const int c0 = base + first;
                 const int cEnd = min(ld4, base + segLen);
-                if constexpr (kPrefetch) {
+                if constexpr (kRing) {
+                    ring_stream(c0, cEnd, acc);
+                } else if constexpr (kPrefetch) {
                     int4 cur[R], nxt[R];
                     if (c0 < cEnd) {
 #pragma unroll
@@ -681,7 +735,9 @@ __device__ __forceinline__ void sweep_class(const GreedyParams<SV> &prm, int l, 
             AccT acc[NA];
 #pragma unroll
             for (int i = 0; i < NA; ++i) acc[i] = 0.f;
-            if constexpr (kPrefetch) {
+            if constexpr (kRing) {
+                ring_stream(first, ld4, acc);
+            } else if constexpr (kPrefetch) {
                 int4 cur[R], nxt[R];
                 if (first < ld4) {
 #pragma unroll
@@ -739,12 +795,6 @@ __device__ __forceinline__ void sweep_class(const GreedyParams<SV> &prm, int l, 
         __syncwarp();
         if (lane == 0) { __threadfence(); atomicAdd(done, finished); }
     }
-}
-
-// 16 bytes global -> shared without passing through registers (completion: cp.async.wait_group).
-__device__ __forceinline__ void async_copy16(int4 *smemDst, const int4 *src)
-{
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" :: "r"((uint32_t)__cvta_generic_to_shared(smemDst)), "l"(src) : "memory");
 }
 
 // Threshold pass over one class.  shThr[i] = min over the P listed blocks of cover_p[i]: an element
@@ -1096,16 +1146,78 @@ __device__ __noinline__ void sweep_class_lazy(const GreedyParams<SV> &prm, int l
     }
 }
 
+// Shared-memory arrays a CTA needs to serve sweeps (beside the dynamic area that holds the coverage vectors).
+template <typename SV>
+struct SweepShared {
+    long long f[kMaxSweepBatch];
+    int32_t parts[kSparseMax];
+    typename Arith<SV>::GV theta[kLazyBlocks];
+    int ticket[kSweepThreads / 32];
+    typename Arith<SV>::GV part[kSweepThreads];
+};
+
+// One CTA (kSweepThreads threads) works on the scheduled sweep of class l until its tickets run out: stages the
+// coverage vectors (or the threshold vector) of the listed blocks in shCover and calls the pass the class asked for.
+// Several CTAs may serve the same sweep; they share its ticket counter rowCtr[l].
+template <typename SV>
+__device__ __forceinline__ void sweep_serve_class(const GreedyParams<SV> &prm, int l, int4 *shCover, SweepShared<SV> &sh)
+{
+    const ClassDesc c = prm.desc[l];
+    const int nR = prm.nR[l];
+    const int P = prm.sweepN[l];
+    const int CS = prm.sweepCS[l];
+    const int ld4 = c.ld >> 2;
+    const int32_t *parts = prm.sweepParts + (int64_t)l * kSparseMax;
+    if (prm.sweepMode[l]) {
+        // threshold pass: one vector in shared memory, the blocks' coverage stays in global memory
+        const int4 *thr = reinterpret_cast<const int4 *>(prm.thr + c.vOff / prm.W);
+        for (int i = threadIdx.x; i < ld4; i += blockDim.x) shCover[i] = thr[i];
+        const bool lazy = prm.sweepMode[l] == 2;
+        if (threadIdx.x < P) {
+            sh.parts[threadIdx.x] = parts[threadIdx.x];
+            if (lazy) sh.theta[threadIdx.x] = prm.sweepTheta[(int64_t)l * kLazyBlocks + threadIdx.x];
+        }
+        __syncthreads();
+        uint2 *queue = reinterpret_cast<uint2 *>(reinterpret_cast<char *>(shCover) + thr_bytes_aligned(c.ld * (int)sizeof(SV)) + (threadIdx.x >> 5) * kSparseWarpBytes);
+        if (lazy) {
+            if (P <= 32) sweep_class_lazy<SV, 1>(prm, l, c, nR, P, shCover, sh.parts, sh.theta, queue, &prm.rowCtr[l], nullptr, -1);
+            else sweep_class_lazy<SV, 2>(prm, l, c, nR, P, shCover, sh.parts, sh.theta, queue, &prm.rowCtr[l], nullptr, -1);
+        } else if (P <= 32) sweep_class_sparse<SV, 1>(prm, l, c, nR, P, shCover, sh.parts, queue, &prm.rowCtr[l], nullptr, -1);
+        else sweep_class_sparse<SV, 2>(prm, l, c, nR, P, shCover, sh.parts, queue, &prm.rowCtr[l], nullptr, -1);
+    } else {
+        const int4 *cov = reinterpret_cast<const int4 *>(prm.cover + c.vOff);
+        for (int i = threadIdx.x; i < P * ld4; i += blockDim.x) {
+            int p = i / ld4, cc = i - p * ld4;
+            shCover[i] = cov[(int64_t)parts[p] * ld4 + cc];
+        }
+        if (threadIdx.x < P) {
+            sh.parts[threadIdx.x] = parts[threadIdx.x];
+            if constexpr (Arith<SV>::kInt) sh.f[threadIdx.x] = prm.fval[(int64_t)l * prm.W + parts[threadIdx.x]];
+        }
+        __syncthreads();
+        switch (P) {
+        case 1: sweep_class<SV, 1, 8>(prm, l, c, nR, CS, shCover, sh.f, sh.parts, sh.ticket, sh.part, &prm.rowCtr[l], nullptr, -1); break;
+        case 2: sweep_class<SV, 2, 8>(prm, l, c, nR, CS, shCover, sh.f, sh.parts, sh.ticket, sh.part, &prm.rowCtr[l], nullptr, -1); break;
+        case 4: sweep_class<SV, 4, 8>(prm, l, c, nR, CS, shCover, sh.f, sh.parts, sh.ticket, sh.part, &prm.rowCtr[l], nullptr, -1); break;
+        default: {
+            const int covBytes = thr_bytes_aligned(8 * c.ld * (int)sizeof(SV));
+            if (prm.denseRing && covBytes + dense_ring_bytes(4) <= prm.smemBytes)
+                sweep_class<SV, 8, 4, true>(prm, l, c, nR, CS, shCover, sh.f, sh.parts, sh.ticket, sh.part, &prm.rowCtr[l], nullptr, -1,
+                                            reinterpret_cast<int4 *>(reinterpret_cast<char *>(shCover) + covBytes));
+            else
+                sweep_class<SV, 8, 4>(prm, l, c, nR, CS, shCover, sh.f, sh.parts, sh.ticket, sh.part, &prm.rowCtr[l], nullptr, -1);
+            break;
+        }
+        }
+    }
+    __syncthreads();
+}
+
 // The sweep of greedy step `step`, run by every CTA of the launch (kSweepThreads threads each).
 template <typename SV>
 __device__ __forceinline__ void sweep_step(const GreedyParams<SV> &prm, int step, int4 *shCover)
 {
-    using GV = typename Arith<SV>::GV;
-    __shared__ long long shF[kMaxSweepBatch];
-    __shared__ int32_t shParts[kSparseMax];
-    __shared__ GV shTheta[kLazyBlocks];
-    __shared__ int shTicket[kSweepThreads / 32];
-    __shared__ GV shPart[kSweepThreads];
+    __shared__ SweepShared<SV> shSweep;
     __shared__ int shGo;
     // three lists in rotation: this step reads list step%3, its picks fill (step+1)%3, and the one
     // after that is cleared here, a full step (and at least one barrier / launch boundary) before use
@@ -1137,48 +1249,7 @@ __device__ __forceinline__ void sweep_step(const GreedyParams<SV> &prm, int step
         if (go == INT_MAX) break;
         int s = start + go;
         if (s >= nS) s -= nS;
-        const int l = prm.sweepList[(int64_t)par * prm.L + s];
-        const ClassDesc c = prm.desc[l];
-        const int nR = prm.nR[l];
-        const int P = prm.sweepN[l];
-        const int CS = prm.sweepCS[l];
-        const int ld4 = c.ld >> 2;
-        const int32_t *parts = prm.sweepParts + (int64_t)l * kSparseMax;
-        if (prm.sweepMode[l]) {
-            // threshold pass: one vector in shared memory, the blocks' coverage stays in global memory
-            const int4 *thr = reinterpret_cast<const int4 *>(prm.thr + c.vOff / prm.W);
-            for (int i = threadIdx.x; i < ld4; i += blockDim.x) shCover[i] = thr[i];
-            const bool lazy = prm.sweepMode[l] == 2;
-            if (threadIdx.x < P) {
-                shParts[threadIdx.x] = parts[threadIdx.x];
-                if (lazy) shTheta[threadIdx.x] = prm.sweepTheta[(int64_t)l * kLazyBlocks + threadIdx.x];
-            }
-            __syncthreads();
-            uint2 *queue = reinterpret_cast<uint2 *>(reinterpret_cast<char *>(shCover) + thr_bytes_aligned(c.ld * (int)sizeof(SV)) + (threadIdx.x >> 5) * kSparseWarpBytes);
-            if (lazy) {
-                if (P <= 32) sweep_class_lazy<SV, 1>(prm, l, c, nR, P, shCover, shParts, shTheta, queue, &prm.rowCtr[l], nullptr, -1);
-                else sweep_class_lazy<SV, 2>(prm, l, c, nR, P, shCover, shParts, shTheta, queue, &prm.rowCtr[l], nullptr, -1);
-            } else if (P <= 32) sweep_class_sparse<SV, 1>(prm, l, c, nR, P, shCover, shParts, queue, &prm.rowCtr[l], nullptr, -1);
-            else sweep_class_sparse<SV, 2>(prm, l, c, nR, P, shCover, shParts, queue, &prm.rowCtr[l], nullptr, -1);
-        } else {
-            const int4 *cov = reinterpret_cast<const int4 *>(prm.cover + c.vOff);
-            for (int i = threadIdx.x; i < P * ld4; i += blockDim.x) {
-                int p = i / ld4, cc = i - p * ld4;
-                shCover[i] = cov[(int64_t)parts[p] * ld4 + cc];
-            }
-            if (threadIdx.x < P) {
-                shParts[threadIdx.x] = parts[threadIdx.x];
-                if constexpr (Arith<SV>::kInt) shF[threadIdx.x] = prm.fval[(int64_t)l * prm.W + parts[threadIdx.x]];
-            }
-            __syncthreads();
-            switch (P) {
-            case 1: sweep_class<SV, 1, 8>(prm, l, c, nR, CS, shCover, shF, shParts, shTicket, shPart, &prm.rowCtr[l], nullptr, -1); break;
-            case 2: sweep_class<SV, 2, 8>(prm, l, c, nR, CS, shCover, shF, shParts, shTicket, shPart, &prm.rowCtr[l], nullptr, -1); break;
-            case 4: sweep_class<SV, 4, 8>(prm, l, c, nR, CS, shCover, shF, shParts, shTicket, shPart, &prm.rowCtr[l], nullptr, -1); break;
-            default: sweep_class<SV, 8, 4>(prm, l, c, nR, CS, shCover, shF, shParts, shTicket, shPart, &prm.rowCtr[l], nullptr, -1); break;
-            }
-        }
-        __syncthreads();
+        sweep_serve_class(prm, prm.sweepList[(int64_t)par * prm.L + s], shCover, shSweep);
     }
 }
 
@@ -1848,6 +1919,53 @@ __global__ void __launch_bounds__(kSweepThreads, 1) greedy_async_kernel(const __
 }
 
 // ---------------------------------------------------------------------------------------------
+// The greedy loop with one CTA per class at a time (many classes: more classes than SMs, or classes too small
+// to be worth sharing).  Classes are independent in Algorithm 1, so a CTA draws a class from a counter and runs
+// it from its first pick to its last -- sweep with all its warps, then picks until the next sweep is due -- and
+// draws the next.  Nothing is shared between CTAs but that counter: no grid barrier, no hand-off, and while one
+// SM makes picks (latency-bound) the others stream, so the memory system stays busy without any phase structure.
+// Classes are drawn largest first (classOrder), which keeps the last CTAs from finishing long after the rest.
+template <typename SV>
+__global__ void __launch_bounds__(kSweepThreads, 1) greedy_owner_kernel(const __grid_constant__ GreedyParams<SV> prm)
+{
+    extern __shared__ __align__(128) int4 shCover[];
+    __shared__ SweepShared<SV> shSweep;
+    __shared__ int shClass;
+    __shared__ int shKeep[2];
+    unsigned long long tSweep = 0, tPick = 0, tThreshold = 0;
+    for (;;) {
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            const int k = atomicAdd(&prm.nSweep[0], 1);
+            shClass = k < prm.L ? prm.classOrder[k] : -1;
+        }
+        __syncthreads();
+        const int l = shClass;
+        if (l < 0) break;
+        if (prm.desc[l].M == 0) continue;
+        for (int round = 0; round <= prm.desc[l].M; ++round) {
+            if (*(volatile int32_t *)prm.status != 0) break;
+            unsigned long long t0 = 0;
+            if (blockIdx.x == 0 && threadIdx.x == 0) t0 = global_ns();
+            const bool thresholdPass = prm.sweepN[l] > 0 && prm.sweepMode[l] != 0;
+            if (prm.sweepN[l] > 0) sweep_serve_class(prm, l, shCover, shSweep);
+            __syncthreads();
+            if (blockIdx.x == 0 && threadIdx.x == 0) {
+                const unsigned long long t1 = global_ns();
+                tSweep += t1 - t0;
+                if (thresholdPass) tThreshold += t1 - t0;
+                t0 = t1;
+            }
+            pick_chain(prm, l, round, shCover, prm.smemBytes, 0, shKeep);
+            __syncthreads();
+            if (blockIdx.x == 0 && threadIdx.x == 0) tPick += global_ns() - t0;
+            if (shKeep[0] == 0 || shKeep[1] < 0) break;
+        }
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0) { prm.phaseNs[0] = tSweep; prm.phaseNs[1] = tPick; prm.phaseNs[13] = tThreshold; }
+}
+
+// ---------------------------------------------------------------------------------------------
 // Launch with programmatic stream serialization: the next kernel's CTAs may be placed while this
 // one drains; every kernel starts with cudaGridDependencySynchronize(), so data dependencies hold.
 template <typename... KArgs, typename... Args>
@@ -1932,6 +2050,13 @@ static rcd_status run_greedy(rcd_ctx *ctx, const Sizes &sz, const Workspace &ws,
         for (const auto &c : descHost) sorted.push_back(c.M);
         std::sort(sorted.begin(), sorted.end());
         prm.sizesSorted = ws.sizesSorted;
+        prm.classOrder = ws.classOrder;
+        {
+            std::vector<int32_t> order(descHost.size());
+            for (size_t i = 0; i < order.size(); ++i) order[i] = (int32_t)i;
+            std::stable_sort(order.begin(), order.end(), [&](int32_t a, int32_t b) { return descHost[(size_t)a].M > descHost[(size_t)b].M; });
+            RCD_CUDA(ctx, cudaMemcpyAsync(ws.classOrder, order.data(), order.size() * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+        }
         prm.nonEmpty = 0;
         prm.minM = 0;
         for (int32_t m : sorted) {
@@ -1947,6 +2072,12 @@ static rcd_status run_greedy(rcd_ctx *ctx, const Sizes &sz, const Workspace &ws,
     int64_t smem = (int64_t)batch * maxLd * (int64_t)sizeof(SV);
     if (prm.sparseMinMembers >= 0)                                   // threshold pass: one vector + the warps' rings and queues
         smem = std::max<int64_t>(smem, (int64_t)thr_bytes_aligned(maxLd * (int)sizeof(SV)) + kSparseQueueBytes);
+    // room for the rings of the 8-block dense pass behind its coverage vectors, where both fit
+    prm.denseRing = 0;
+    if (batch == 8 && ctx->cfg.dense_ring != 2) {
+        const int64_t withRing = (int64_t)thr_bytes_aligned(8 * maxLd * (int)sizeof(SV)) + dense_ring_bytes(4);
+        if (withRing <= smemCap) { smem = std::max<int64_t>(smem, withRing); prm.denseRing = 1; }
+    }
     if (smem > smemCap) smem = smemCap;
     if ((int64_t)maxLd * (int64_t)sizeof(SV) > smem)
         return fail(ctx, RCD_ERR_UNSUPPORTED,
@@ -1971,8 +2102,13 @@ static rcd_status run_greedy(rcd_ctx *ctx, const Sizes &sz, const Workspace &ws,
     const bool perSweep = ctx->cfg.profile >= 2;
     int path = ctx->cfg.greedy_path;
     if (perSweep || !ctx->cooperative) path = 1;
-    if (path == 0) path = (sz.L * 4 <= ctx->smCount) ? 3 : 2;
+    if (path == 0) path = (sz.L * 4 <= ctx->smCount) ? 3 : 4;
     if (path == 3 && ctx->smCount < 2) path = 2;
+    if (path == 4) {
+        RCD_CUDA(ctx, cudaFuncSetAttribute(greedy_owner_kernel<SV>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        prm.asyncMode = 2;
+        prm.sweepWarps = kSweepThreads / 32;                     // a class is swept by the warps of its own CTA
+    }
     if (path == 2 || path == 3) {
         // one cooperative launch needs one CTA per SM resident at once
         RCD_CUDA(ctx, cudaFuncSetAttribute(greedy_persistent_kernel<SV>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
@@ -2004,7 +2140,11 @@ static rcd_status run_greedy(rcd_ctx *ctx, const Sizes &sz, const Workspace &ws,
     // One cooperative launch for the whole loop when the device can hold one sweep CTA per SM at once;
     // per-sweep event timing (profile 2) needs the sweeps as separate launches.
     const bool persistent = path != 1;
-    if (persistent && path == 3) {
+    if (path == 4) {
+        // (an ordinary launch: the CTAs never wait for one another)
+        greedy_owner_kernel<SV><<<std::min<int>(ctx->smCount, sz.L), kSweepThreads, (size_t)smem, st>>>(prm);
+        ctx->kernelLaunches += 1;
+    } else if (persistent && path == 3) {
         void *args[] = {(void *)&prm};
         RCD_CUDA(ctx, cudaLaunchCooperativeKernel((const void *)greedy_async_kernel<SV>, dim3(ctx->smCount), dim3(kSweepThreads),
                                                   args, (size_t)smem, st));

@@ -116,6 +116,7 @@ struct Workspace {
     ClassSync *sync;        // [L] asynchronous kernel: hand-off words
     int32_t *tickets;       // [N + L] asynchronous kernel: one ticket counter per (class, sweep number), never reused
     int32_t *sizesSorted;   // [L] class sizes, ascending
+    int32_t *classOrder;    // [L] classes by descending size
     void *floorv;           // [L][kLazyBlocks] per block: every stored gain at or above it is exact (int64 / double)
     void *theta;            // [L][kLazyBlocks] per block: floor its next row-skipping pass will establish
     void *sweepTheta;       // [L][kLazyBlocks] floors of the blocks the class's next pass lists, in list order (int64 / fp32)

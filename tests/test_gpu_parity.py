@@ -99,7 +99,7 @@ def check_exact(rcd, orc, wl, variant="incremental", **cfg):
     return a, o, v, ref
 
 
-@pytest.mark.parametrize("path", [0, 1, 2, 3])  # chosen by the library / two launches per round / one launch with rounds / asynchronous
+@pytest.mark.parametrize("path", [0, 1, 2, 3, 4])  # chosen by the library / two launches per round / one launch with rounds / asynchronous / one CTA per class
 @pytest.mark.parametrize("batch", [1, 2, 4, 8])
 def test_partition_c1_exact(rcd, orc, batch, path):
     from paper_2211_00839_b200.workloads import make_workload
@@ -129,7 +129,7 @@ def test_partition_int8_ragged_classes(rcd, orc, seed):
     caps = np.array([1, 2.5, 1, 4, 0.5, 3, 1, 1, 2], dtype=np.float64)
     wl = Workload("ragged", "int8", np.ascontiguousarray(feats[perm]), np.ascontiguousarray(labels[perm]), caps,
                   len(sizes), len(caps))
-    for batch, path in ((8, 0), (1, 0), (8, 1), (8, 2), (8, 3), (2, 3)):
+    for batch, path in ((8, 0), (1, 0), (8, 1), (8, 2), (8, 3), (2, 3), (8, 4), (4, 4)):
         check_exact(rcd, orc, wl, sweep_batch_max=batch, greedy_path=path)
 
 
@@ -156,7 +156,7 @@ def test_partition_c5_reduced_exact(rcd, orc):
     check_exact(rcd, orc, wl)
 
 
-@pytest.mark.parametrize("path", [2, 3])
+@pytest.mark.parametrize("path", [2, 3, 4])
 def test_partition_many_small_classes_every_loop_form(rcd, orc, path):
     """More classes than pick CTAs of the asynchronous loop (a pick CTA then serves several classes), of
     unequal sizes so that classes finish at different times; W = 64 with threshold passes."""
@@ -198,7 +198,7 @@ def ragged_float_workload(sizes, d, W, seed):
                     len(sizes), W)
 
 
-@pytest.mark.parametrize("path", [2, 3])
+@pytest.mark.parametrize("path", [2, 3, 4])
 def test_float_partition_is_reproducible_with_ragged_classes(rcd, path):
     """fp32 gains depend on how a pass splits its columns, so the shape of a class's sweeps must not depend on
     when OTHER classes finish: classes of very unequal sizes (the small ones finish while the large ones
@@ -274,7 +274,7 @@ def test_partition_c3_reduced_float(rcd, orc):
     check_float(rcd, orc, wl)
 
 
-@pytest.mark.parametrize("batch,path", [(1, 0), (8, 0), (8, 1), (8, 2), (8, 3)])
+@pytest.mark.parametrize("batch,path", [(1, 0), (8, 0), (8, 1), (8, 2), (8, 3), (8, 4)])
 def test_partition_c4_reduced_float(rcd, orc, batch, path):
     from paper_2211_00839_b200.workloads import make_workload
     wl = make_workload("C4", L=5, M=500, d=256)
@@ -291,7 +291,7 @@ def run_with_profile(rcd, wl, **cfg):
         return a.cpu().numpy(), o.cpu().numpy(), v.cpu().numpy(), ctx.profile()
 
 
-@pytest.mark.parametrize("path", [0, 1, 2, 3])
+@pytest.mark.parametrize("path", [0, 1, 2, 3, 4])
 def test_threshold_passes_int8_exact(rcd, orc, path):
     """Classes large enough that the sweeps switch to threshold passes: same picks as the oracle, and
     the same as with dense passes only."""
@@ -308,7 +308,8 @@ def test_threshold_passes_int8_exact(rcd, orc, path):
 
 @pytest.mark.parametrize("knobs", [dict(greedy_path=3, async_group=1), dict(greedy_path=3, async_group=2, async_help_min=1),
                                    dict(greedy_path=3, async_help_min=400), dict(threshold_from=1), dict(threshold_from=2, threshold_hit_shift=3),
-                                   dict(greedy_path=2, threshold_from=1, threshold_hit_shift=7), dict(greedy_path=1, threshold_from=3)])
+                                   dict(greedy_path=2, threshold_from=1, threshold_hit_shift=7), dict(greedy_path=1, threshold_from=3),
+                                   dict(greedy_path=4, threshold_from=2, sweep_batch_max=4)])
 def test_scheduling_knobs_never_change_a_result(rcd, orc, knobs):
     """Serving order of the asynchronous loop and the start / back-off rule of the threshold passes only move
     work around: assignment, pick order and block values stay those of the oracle."""
@@ -341,7 +342,7 @@ def test_threshold_passes_float(rcd, orc):
 
 # ----------------------------------------------------------------------------- exact lazy evaluation (row-skipping passes)
 
-@pytest.mark.parametrize("path", [0, 1, 2, 3])
+@pytest.mark.parametrize("path", [0, 1, 2, 3, 4])
 def test_lazy_evaluation_int8_exact(rcd, orc, path):
     """Row-skipping threshold passes (stored gains as upper bounds, a floor per block): rows are skipped, some picks
     miss and are answered by a pass over every row, and every pick is still the oracle's."""
@@ -373,7 +374,7 @@ def test_lazy_evaluation_many_blocks_and_ragged_classes_exact(rcd, orc, lazy_fro
         keep[ids[:int(rng.integers(0, 200))]] = False
     wl = Workload("ragged-lazy", "int8", np.ascontiguousarray(base.features[keep]), np.ascontiguousarray(base.labels[keep]),
                   base.capacities, base.L, base.W)
-    for path in (2, 3):
+    for path in (2, 3, 4):
         check_exact(rcd, orc, wl, greedy_path=path, lazy_mode=1, lazy_from=lazy_from)
 
 
