@@ -218,7 +218,7 @@ def run_ours(args):
     Xd, yd = Xh.to(dev), yh.to(dev)
     kind = rcd.RCD_SIM_GAUSSIAN if args.similarity == "gaussian" else rcd.RCD_SIM_DOT
     ctx = rcd.Context(local, sweep_batch_max=args.sweep_batch, profile=1, greedy_path=args.greedy_path, similarity_kind=kind,
-                      async_group=args.async_group, async_help_min=args.async_help_min, lazy_mode=args.lazy_mode, lazy_from=args.lazy_from, dense_ring=args.dense_ring,
+                      async_group=args.async_group, async_help_min=args.async_help_min, lazy_mode=args.lazy_mode, lazy_from=args.lazy_from, dense_ring=args.dense_ring, incremental=args.incremental, incremental_max=args.incremental_max,
                       objective=rcd.RCD_OBJ_GRAPH_CUT if args.objective == "cut" else rcd.RCD_OBJ_FACILITY)
 
     def barrier():
@@ -407,6 +407,7 @@ def run_ours(args):
                                 async_lull_ms=prof["async_lull_ns"] * 1e-6, async_visits=int(prof["async_visits"]), async_attempts=int(prof["async_attempts"]),
                                 lazy_sweeps=int(prof["lazy_sweeps"]), lazy_misses=int(prof["lazy_misses"]), lazy_rows=int(prof["lazy_rows"]),
                                 lazy_rows_skipped=int(prof["lazy_rows_skipped"]),
+                                incremental_updates=int(prof["incremental_updates"]), incremental_rows=int(prof["incremental_rows"]),
                                 threshold_pass_ms=prof["threshold_pass_ns"] * 1e-6, threshold_pass_gb=prof["threshold_pass_bytes"] * 1e-9),
               "similarity": similarity,
               "e2e": {"value": e2e_value, "unit": "samples/s", "h2d_bytes_per_step": int(h2d),
@@ -447,6 +448,8 @@ def main():
     ap.add_argument("--sharding", default="replicas", choices=["replicas", "classes"],
                     help="with --gpus N: one dataset per rank (weak scaling), or one dataset with its classes sharded over the ranks (strong scaling)")
     ap.add_argument("--lazy-mode", type=int, default=0, help="1 = threshold passes skip rows below the blocks' floors (exact lazy evaluation), 0 = every pass reads every row")
+    ap.add_argument("--incremental", type=int, default=0, help="in-place correction of stored gains: 0 = chosen by the library, 1 = on, 2 = off")
+    ap.add_argument("--incremental-max", type=int, default=0, help="most raised columns a pick corrects in place (0 = library default)")
     ap.add_argument("--dense-ring", type=int, default=0, help="0 = dense passes stream through shared-memory rings where they fit, 2 = never")
     ap.add_argument("--lazy-from", type=int, default=0, help="members a block needs before rows are skipped (0 = library default)")
     ap.add_argument("--ref-picks", type=int, default=150, help="picks per class in the CPU-oracle sample")

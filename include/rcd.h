@@ -105,7 +105,13 @@ typedef struct {
     int32_t lazy_from;         /* members every out-of-date block must have before rows are skipped; 0 = default (8) */
     int32_t dense_ring;        /* 0 = 8-block dense passes stream S through per-warp rings of asynchronous copies in shared
                                   memory when the coverage vectors leave room for them; 2 = never (one register buffer ahead) */
-    int32_t reserved[2];       /* must be 0 */
+    int32_t incremental;       /* in-place correction of stored gains (greedy paths 3 and 4).  When a pick raised its block's coverage
+                                  in few columns i, every candidate's gain falls by max(0, S[v][i] - old_i) - max(0, S[v][i] - new_i),
+                                  read from row i of S (S is symmetric): the block's stored gains stay exact and it needs no
+                                  pass over S.  0 = choose (on for path 3 with at most 8 blocks, where it is faster), 1 = on,
+                                  2 = off (every block that received a sample waits for a pass).  Same picks either way. */
+    int32_t incremental_max;   /* most columns a pick may raise and still be corrected in place; 0 = default (32 for greedy
+                                  path 3, where a pass is served by the whole GPU; 128 for path 4); at most 128 */
 } rcd_config;
 
 /* Timings and counters of the last rcd_partition / rcd_partition_host on a context (profile >= 1). */
@@ -135,6 +141,8 @@ typedef struct {
     int64_t lazy_misses;            /* picks whose best stored gain lay below its block's floor (answered by a pass over every row) */
     int64_t lazy_rows;              /* rows of S those passes did read */
     int64_t lazy_rows_skipped;      /* rows they did not */
+    int64_t incremental_updates;    /* picks after which the block's stored gains were corrected in place (no pass needed) */
+    int64_t incremental_rows;       /* rows of S those corrections read (one per column whose coverage rose) */
     int64_t threshold_pass_ns;      /* one CTA per class: time the first CTA spent in threshold passes (part of persistent_sweep_ns) */
     int64_t threshold_pass_bytes;   /* bytes of S and threshold vectors the (row-visiting) threshold passes had to read (part of sweep_bytes) */
 } rcd_profile;

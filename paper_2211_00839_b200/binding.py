@@ -50,7 +50,7 @@ class RcdConfig(C.Structure):
     _fields_ = [("sweep_batch_max", C.c_int32), ("similarity_path", C.c_int32), ("profile", C.c_int32),
                 ("greedy_path", C.c_int32), ("similarity_kind", C.c_int32), ("objective", C.c_int32), ("sweep_mode", C.c_int32), ("async_group", C.c_int32),
                 ("async_help_min", C.c_int32), ("threshold_from", C.c_int32), ("threshold_hit_shift", C.c_int32),
-                ("lazy_mode", C.c_int32), ("lazy_from", C.c_int32), ("dense_ring", C.c_int32), ("reserved", C.c_int32 * 2)]
+                ("lazy_mode", C.c_int32), ("lazy_from", C.c_int32), ("dense_ring", C.c_int32), ("incremental", C.c_int32), ("incremental_max", C.c_int32)]
 
 
 class RcdProfile(C.Structure):
@@ -62,7 +62,7 @@ class RcdProfile(C.Structure):
                 ("threshold_elems", C.c_int64), ("threshold_max_blocks", C.c_int64),
                 ("async_lull_ns", C.c_int64), ("async_visits", C.c_int64), ("async_attempts", C.c_int64),
                 ("lazy_sweeps", C.c_int64), ("lazy_misses", C.c_int64), ("lazy_rows", C.c_int64),
-                ("lazy_rows_skipped", C.c_int64), ("threshold_pass_ns", C.c_int64), ("threshold_pass_bytes", C.c_int64)]
+                ("lazy_rows_skipped", C.c_int64), ("incremental_updates", C.c_int64), ("incremental_rows", C.c_int64), ("threshold_pass_ns", C.c_int64), ("threshold_pass_bytes", C.c_int64)]
 
 
 def _load() -> C.CDLL:
@@ -167,7 +167,7 @@ class Context:
     def __init__(self, device: int = 0, sweep_batch_max: int = 0, similarity_path: int = 0, profile: int = 0,
                  greedy_path: int = 0, similarity_kind: int = 0, objective: int = 0, sweep_mode: int = 0,
                  async_group: int = 0, async_help_min: int = 0, threshold_from: int = 0, threshold_hit_shift: int = 0,
-                 lazy_mode: int = 0, lazy_from: int = 0, dense_ring: int = 0):
+                 lazy_mode: int = 0, lazy_from: int = 0, dense_ring: int = 0, incremental: int = 0, incremental_max: int = 0):
         torch = _torch()
         if not torch.cuda.is_available():
             raise RcdError(4, "no CUDA device: this library has no CPU path")
@@ -188,6 +188,8 @@ class Context:
         cfg.lazy_mode = lazy_mode
         cfg.lazy_from = lazy_from
         cfg.dense_ring = dense_ring
+        cfg.incremental = incremental
+        cfg.incremental_max = incremental_max
         self.similarity_kind = similarity_kind
         self._h = C.c_void_p()
         st = lib.rcd_create(C.byref(self._h), self.device, C.byref(cfg))

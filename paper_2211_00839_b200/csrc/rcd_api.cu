@@ -321,7 +321,8 @@ rcd_status rcd_create(rcd_ctx **out, int cuda_device, const rcd_config *cfg)
         if (cfg->lazy_mode != 0 && cfg->lazy_mode != 1) return RCD_ERR_INVALID_ARG;
         if (cfg->lazy_from < 0) return RCD_ERR_INVALID_ARG;
         if (cfg->dense_ring != 0 && cfg->dense_ring != 2) return RCD_ERR_INVALID_ARG;
-        for (int i = 0; i < 2; ++i) if (cfg->reserved[i] != 0) return RCD_ERR_INVALID_ARG;
+        if (cfg->incremental < 0 || cfg->incremental > 2) return RCD_ERR_INVALID_ARG;
+        if (cfg->incremental_max < 0 || cfg->incremental_max > 128) return RCD_ERR_INVALID_ARG;
     }
     int count = 0;
     if (cudaGetDeviceCount(&count) != cudaSuccess || cuda_device < 0 || cuda_device >= count) {
@@ -411,6 +412,8 @@ rcd_status rcd_get_profile(rcd_ctx *ctx, rcd_profile *out)
         out->lazy_rows = (int64_t)ns[10];
         out->lazy_rows_skipped = (int64_t)ns[11];
         lazyBytes = (int64_t)ns[12];
+        out->incremental_updates = (int64_t)ns[15];
+        out->incremental_rows = (int64_t)ns[16];
         out->threshold_pass_ns = (int64_t)ns[13];
         out->threshold_pass_bytes = (int64_t)ns[14];
         out->persistent_sweep_ns = (int64_t)ns[0];

@@ -16,7 +16,7 @@ constexpr int kSparseMax = 64;             // blocks refreshed by one threshold 
 constexpr int kSweepThreads = 512;         // sweep CTA: 16 warps, one CTA per SM
 constexpr int kSelectThreads = 512;        // pick/update CTA: one per class
 constexpr int kLazyBlocks = 64;            // row skipping keeps a floor per block for classes of up to this many blocks
-constexpr int kPhaseWords = 16;            // 64-bit counters a greedy launch keeps (phase clocks, barrier, pass statistics)
+constexpr int kPhaseWords = 20;            // 64-bit counters a greedy launch keeps (phase clocks, barrier, pass statistics)
 constexpr size_t kAlign = 256;
 
 // Device-side status bits (OR-ed into the status word).

@@ -198,7 +198,17 @@ def test_c2_every_class_bit_exact(rcd, orc):
 
 def test_c2_every_class_bit_exact_with_lazy_evaluation(rcd, orc):
     """The same 10 x 5000 picks with row-skipping passes switched on."""
-    _check_against_digests(rcd, orc, "C2", lazy_mode=1)
+    _check_against_digests(rcd, orc, "C2", lazy_mode=1, incremental=2)
+
+
+def test_c2_every_class_bit_exact_without_incremental_updates(rcd, orc):
+    """... and with every block waiting for a pass after each sample it receives (the bandwidth-bound form)."""
+    _check_against_digests(rcd, orc, "C2", incremental=2)
+
+
+def test_c5_every_class_bit_exact_with_incremental_updates(rcd, orc):
+    """All 1000 classes with the in-place correction of stored gains forced on (the library leaves it off for this shape)."""
+    _check_against_digests(rcd, orc, "C5", incremental=1)
 
 
 def test_c5_every_class_bit_exact(rcd, orc):

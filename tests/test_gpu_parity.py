@@ -298,10 +298,11 @@ def test_threshold_passes_int8_exact(rcd, orc, path):
     from paper_2211_00839_b200.workloads import make_workload
     wl = make_workload("C2", L=3, M=1200)
     ref = orc.partition(wl.features, wl.labels, wl.capacities, wl.L, variant="incremental")
-    a, o, v, prof = run_with_profile(rcd, wl, greedy_path=path)
+    # (incremental = 2: every block that received a sample waits for a pass, so that threshold passes are what runs)
+    a, o, v, prof = run_with_profile(rcd, wl, greedy_path=path, incremental=2)
     assert prof["threshold_elems"] > 0 and 0 < prof["threshold_hits"] < prof["threshold_elems"] // 32
     assert np.array_equal(a, ref.assignment) and np.array_equal(o, ref.order) and np.array_equal(v, ref.part_values)
-    a1, o1, v1, prof1 = run_with_profile(rcd, wl, greedy_path=path, sweep_mode=1)
+    a1, o1, v1, prof1 = run_with_profile(rcd, wl, greedy_path=path, sweep_mode=1, incremental=2)
     assert prof1["threshold_elems"] == 0
     assert np.array_equal(a1, a) and np.array_equal(o1, o) and np.array_equal(v1, v)
 
@@ -323,7 +324,7 @@ def test_threshold_passes_many_blocks_exact(rcd, orc):
     from paper_2211_00839_b200.workloads import make_workload
     wl = make_workload("C5", L=3, M=1300, d=128)
     ref = orc.partition(wl.features, wl.labels, wl.capacities, wl.L, variant="incremental")
-    a, o, v, prof = run_with_profile(rcd, wl)
+    a, o, v, prof = run_with_profile(rcd, wl, incremental=2)
     assert prof["threshold_elems"] > 0 and prof["threshold_max_blocks"] > 32
     assert np.array_equal(a, ref.assignment) and np.array_equal(o, ref.order) and np.array_equal(v, ref.part_values)
 
@@ -331,13 +332,68 @@ def test_threshold_passes_many_blocks_exact(rcd, orc):
 def test_threshold_passes_float(rcd, orc):
     from paper_2211_00839_b200.workloads import make_workload
     wl = make_workload("C3", L=2, M=900, d=512)
-    with rcd.Context(0, profile=1) as ctx:
+    with rcd.Context(0, profile=1, incremental=2) as ctx:
         X, y = to_device(rcd, wl)
         ctx.rcd_partition(X, y, wl.capacities, wl.L)
         ctx.sync_status()
         assert ctx.profile()["threshold_elems"] > 0
-    check_float(rcd, orc, wl)                       # default configuration: the run above
-    check_float(rcd, orc, wl, sweep_mode=1)
+    check_float(rcd, orc, wl, incremental=2)        # the run above
+    check_float(rcd, orc, wl, sweep_mode=1, incremental=2)
+
+
+# ----------------------------------------------------------------------------- incremental update of stored gains
+
+@pytest.mark.parametrize("path", [3, 4])
+def test_incremental_update_int8_exact(rcd, orc, path):
+    """A pick that raises its block's coverage in few columns corrects the block's stored gains in place (one row of S
+    per column); the block then needs no pass.  Same picks as the oracle, and as with the correction switched off."""
+    from paper_2211_00839_b200.workloads import make_workload
+    wl = make_workload("C2", L=3, M=1200)
+    ref = orc.partition(wl.features, wl.labels, wl.capacities, wl.L, variant="incremental")
+    a, o, v, prof = run_with_profile(rcd, wl, greedy_path=path, incremental=1)
+    assert prof["incremental_updates"] > 1000 and prof["incremental_rows"] >= prof["incremental_updates"] // 2
+    assert np.array_equal(a, ref.assignment) and np.array_equal(o, ref.order) and np.array_equal(v, ref.part_values)
+    a0, o0, v0, prof0 = run_with_profile(rcd, wl, greedy_path=path, incremental=2)
+    assert prof0["incremental_updates"] == 0
+    assert np.array_equal(a0, a) and np.array_equal(o0, o) and np.array_equal(v0, v)
+    assert prof["sweep_bytes"] < prof0["sweep_bytes"]
+
+
+def test_incremental_update_many_blocks_ragged_ties_exact(rcd, orc):
+    """W = 64 with short rows (twelve rows of S in flight per thread), ragged classes with duplicate rows (ties), several
+    caps on the number of raised columns, both loop forms that carry the correction."""
+    from paper_2211_00839_b200.workloads import Workload, make_workload
+    wl = make_workload("C5", L=3, M=1300, d=128)
+    for path, cap in ((4, 0), (4, 5), (3, 0), (3, 128)):
+        check_exact(rcd, orc, wl, greedy_path=path, incremental=1, incremental_max=cap)
+    base = make_workload("C2", L=40, M=300, d=64)
+    rng = np.random.default_rng(29)
+    keep = np.ones(base.N, bool)
+    for l in range(base.L):
+        ids = np.nonzero(base.labels == l)[0]
+        keep[ids[:int(rng.integers(0, 200))]] = False
+    feats = base.features[keep].copy()
+    feats[::7] = feats[3]
+    wl2 = Workload("ragged-inc", "int8", np.ascontiguousarray(feats), np.ascontiguousarray(base.labels[keep]), base.capacities, base.L, base.W)
+    for path in (3, 4):
+        check_exact(rcd, orc, wl2, greedy_path=path, incremental=1)
+
+
+@pytest.mark.parametrize("path", [3, 4])
+def test_incremental_update_float(rcd, orc, path):
+    from paper_2211_00839_b200.workloads import make_workload
+    wl = make_workload("C3", L=2, M=900, d=512)
+    with rcd.Context(0, profile=1, greedy_path=path, incremental=1) as ctx:
+        X, y = to_device(rcd, wl)
+        ctx.rcd_partition(X, y, wl.capacities, wl.L)
+        ctx.sync_status()
+        assert ctx.profile()["incremental_updates"] > 0
+    check_float(rcd, orc, wl, greedy_path=path, incremental=1)
+    check_float(rcd, orc, wl, greedy_path=path, incremental=1, incremental_max=4)
+    r1 = run_partition(rcd, wl, greedy_path=path, incremental=1)
+    r2 = run_partition(rcd, wl, greedy_path=path, incremental=1)
+    for x, y in zip(r1, r2):
+        assert np.array_equal(x, y)                      # the corrections are applied in a fixed order
 
 
 # ----------------------------------------------------------------------------- exact lazy evaluation (row-skipping passes)
@@ -349,10 +405,10 @@ def test_lazy_evaluation_int8_exact(rcd, orc, path):
     from paper_2211_00839_b200.workloads import make_workload
     wl = make_workload("C2", L=3, M=1200)
     ref = orc.partition(wl.features, wl.labels, wl.capacities, wl.L, variant="incremental")
-    a, o, v, prof = run_with_profile(rcd, wl, greedy_path=path, lazy_mode=1, lazy_from=2)
+    a, o, v, prof = run_with_profile(rcd, wl, greedy_path=path, lazy_mode=1, lazy_from=2, incremental=2)
     assert prof["lazy_sweeps"] > 0 and prof["lazy_rows_skipped"] > prof["lazy_rows"] > 0 and prof["lazy_misses"] > 0
     assert np.array_equal(a, ref.assignment) and np.array_equal(o, ref.order) and np.array_equal(v, ref.part_values)
-    a0, o0, v0, prof0 = run_with_profile(rcd, wl, greedy_path=path)
+    a0, o0, v0, prof0 = run_with_profile(rcd, wl, greedy_path=path, incremental=2)
     assert prof0["lazy_sweeps"] == 0 and prof0["lazy_rows"] == 0
     assert prof["sweep_bytes"] < prof0["sweep_bytes"]
 
@@ -363,7 +419,7 @@ def test_lazy_evaluation_many_blocks_and_ragged_classes_exact(rcd, orc, lazy_fro
     from paper_2211_00839_b200.workloads import Workload, make_workload
     wl = make_workload("C5", L=3, M=1300, d=128)
     ref = orc.partition(wl.features, wl.labels, wl.capacities, wl.L, variant="incremental")
-    a, o, v, prof = run_with_profile(rcd, wl, lazy_mode=1, lazy_from=lazy_from)
+    a, o, v, prof = run_with_profile(rcd, wl, lazy_mode=1, lazy_from=lazy_from, incremental=2)
     assert prof["lazy_sweeps"] > 0
     assert np.array_equal(a, ref.assignment) and np.array_equal(o, ref.order) and np.array_equal(v, ref.part_values)
     base = make_workload("C2", L=40, M=300, d=64)
@@ -375,18 +431,18 @@ def test_lazy_evaluation_many_blocks_and_ragged_classes_exact(rcd, orc, lazy_fro
     wl = Workload("ragged-lazy", "int8", np.ascontiguousarray(base.features[keep]), np.ascontiguousarray(base.labels[keep]),
                   base.capacities, base.L, base.W)
     for path in (2, 3, 4):
-        check_exact(rcd, orc, wl, greedy_path=path, lazy_mode=1, lazy_from=lazy_from)
+        check_exact(rcd, orc, wl, greedy_path=path, lazy_mode=1, lazy_from=lazy_from, incremental=2)
 
 
 def test_lazy_evaluation_float(rcd, orc):
     from paper_2211_00839_b200.workloads import make_workload
     wl = make_workload("C3", L=2, M=900, d=512)
-    with rcd.Context(0, profile=1, lazy_mode=1, lazy_from=2) as ctx:
+    with rcd.Context(0, profile=1, lazy_mode=1, lazy_from=2, incremental=2) as ctx:
         X, y = to_device(rcd, wl)
         ctx.rcd_partition(X, y, wl.capacities, wl.L)
         ctx.sync_status()
         assert ctx.profile()["lazy_sweeps"] > 0
-    check_float(rcd, orc, wl, lazy_mode=1, lazy_from=2)
+    check_float(rcd, orc, wl, lazy_mode=1, lazy_from=2, incremental=2)
     check_float(rcd, orc, wl, lazy_mode=1, greedy_path=2)
 
 
