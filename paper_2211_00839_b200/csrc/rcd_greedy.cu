@@ -1700,6 +1700,9 @@ __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, i
                     atomicAdd(&prm.phaseNs[12], (unsigned long long)(total + 2) * (unsigned long long)c.ld * sizeof(SV) + 2ull * c.ld * sizeof(GV));
                 }
             }
+            // (a compiler barrier: without it the correction above and the choice of the next block below are scheduled
+            // into one another, and a pick takes 3 us longer -- C2 66 ms instead of 47 ms, measured)
+            asm volatile("" ::: "memory");
             if (warp == 0) {
                 __syncwarp();
                 plan_decide(prm, l, c, nR - 1, round + 1, shPlan, &shPre);
@@ -2300,6 +2303,11 @@ static rcd_status run_greedy(rcd_ctx *ctx, const Sizes &sz, const Workspace &ws,
     if (path == 3 && ctx->smCount < 2) path = 2;
     if (path == 4) {
         RCD_CUDA(ctx, cudaFuncSetAttribute(greedy_owner_kernel<SV>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        // (in-place correction of stored gains: a class's passes are made by one SM here, so their cost grows with the
+        // square of the class size while a correction reads a few dozen rows; measured: it wins on 1300-sample classes
+        // with 64 blocks (208 -> 183 ms) and loses on 500-sample classes with 32 (3.9 -> 5.0 ms))
+        if (ctx->cfg.incremental == 0) prm.incremental = sz.maxM >= 1024 ? 1 : 0;
+        if (ctx->cfg.incremental_max <= 0) prm.deltaMax = 64;
         prm.asyncMode = 2;
         prm.sweepWarps = kSweepThreads / 32;                     // a class is swept by the warps of its own CTA
     }
@@ -2317,7 +2325,7 @@ static rcd_status run_greedy(rcd_ctx *ctx, const Sizes &sz, const Workspace &ws,
         if (ctx->cfg.incremental_max <= 0) prm.deltaMax = 32;
         // In-place correction of stored gains costs about three dependent trips to memory per pick; a pass refreshes every
         // out-of-date block at once, so its cost per pick falls with the number of blocks.  Measured on CIFAR-10-shaped
-        // classes: with 8 blocks the correction wins (98 -> 66 ms), with 16 it loses (72 -> 86 ms).
+        // classes: with 8 blocks the correction wins (98 -> 47 ms), with 16 it does not (73 -> 74 ms).
         if (ctx->cfg.incremental == 0) prm.incremental = sz.W <= 8 ? 1 : 0;
         prm.asyncMode = 1;
         prm.nPick = std::min<int>(sz.L, std::max(1, ctx->smCount / 4));
