@@ -278,6 +278,13 @@ RCD_API rcd_status rcd_worker_lists(rcd_ctx *ctx, const int32_t *assignment_dev,
  * lists and batches both proportional to r_j every worker needs the same number of steps per epoch.) */
 RCD_API rcd_status rcd_batch_sizes(int64_t B, const double *capacities_host, int32_t W, int64_t *batch_sizes_host_out);
 
+/* The same with the reading chosen by the caller.  RCD_BATCH_PROPORTIONAL: b_j = B r_j / r_1 (rcd_batch_sizes: the text
+ * below Algorithm 2).  RCD_BATCH_AS_PRINTED: b_j = B r_1 / r_j, the ratio as Algorithm 2's initialisation line prints
+ * it (fast workers then get the smallest batches).  Rounded half up, at least 1, either way.  Host-only. */
+typedef enum { RCD_BATCH_PROPORTIONAL = 0, RCD_BATCH_AS_PRINTED = 1 } rcd_batch_rule;
+RCD_API rcd_status rcd_batch_sizes_rule(int64_t B, const double *capacities_host, int32_t W, rcd_batch_rule rule,
+                                int64_t *batch_sizes_host_out);
+
 /* ---- objective of one class without any allocation (no counterpart in the paper) ----------- */
 
 /* The paper has nothing corresponding to this entry point: it exists for callers that cannot

@@ -298,13 +298,14 @@ def worker_lists(assignment: np.ndarray, W: int) -> Tuple[np.ndarray, np.ndarray
     return offsets, indices.astype(np.int32)
 
 
-def batch_sizes(B: int, capacities: Sequence[float]) -> np.ndarray:
+def batch_sizes(B: int, capacities: Sequence[float], rule: str = "proportional") -> np.ndarray:
     """Per-worker batch sizes of Algorithm 2's initialisation.  The text below Algorithm 2 makes the batch
-    size of a worker proportional to its processing speed (the algorithm's own line prints the inverse
-    ratio): b_i = B * r_i / r_1 with worker 1 the reference, rounded half up to an integer, at least 1."""
+    size of a worker proportional to its processing speed (rule "proportional": b_i = B * r_i / r_1 with worker 1
+    the reference); the algorithm's own line prints the inverse ratio (rule "printed": b_i = B * r_1 / r_i).
+    Rounded half up to an integer, at least 1."""
     r = [float(x) for x in capacities]
     out = []
     for ri in r:
-        x = float(B) * ri / r[0]
+        x = float(B) * ri / r[0] if rule == "proportional" else float(B) * r[0] / ri
         out.append(max(1, int(np.floor(x + 0.5))))
     return np.asarray(out, dtype=np.int64)

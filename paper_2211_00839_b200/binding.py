@@ -36,7 +36,7 @@ EXPORTS = ["rcd_create", "rcd_destroy", "rcd_last_error", "rcd_version", "rcd_sy
            "rcd_partition_workspace_bytes", "rcd_partition",
            "rcd_partition_host_workspace_bytes", "rcd_partition_host", "rcd_objective_workspace_bytes",
            "rcd_objective", "rcd_objective_class_static",
-           "rcd_worker_lists_workspace_bytes", "rcd_worker_lists", "rcd_batch_sizes",
+           "rcd_worker_lists_workspace_bytes", "rcd_worker_lists", "rcd_batch_sizes", "rcd_batch_sizes_rule",
            "rcd_yardstick_read", "rcd_yardstick_mma"]
 
 
@@ -95,6 +95,7 @@ def _load() -> C.CDLL:
     lib.rcd_worker_lists_workspace_bytes.argtypes = [vp, i64, i32, C.POINTER(sz)]
     lib.rcd_worker_lists.argtypes = [vp, vp, i64, i32, vp, vp, vp, sz, vp]
     lib.rcd_batch_sizes.argtypes = [i64, vp, i32, vp]
+    lib.rcd_batch_sizes_rule.argtypes = [i64, vp, i32, C.c_int, vp]
     lib.rcd_yardstick_read.argtypes = [vp, vp, sz, i32, vp]
     lib.rcd_yardstick_mma.argtypes = [vp, C.c_int, i32, C.POINTER(C.c_double), vp]
     for name in EXPORTS:
@@ -121,11 +122,19 @@ def rcd_quotas(M: int, capacities: Sequence[float]) -> np.ndarray:
     return out
 
 
-def rcd_batch_sizes(B: int, capacities: Sequence[float]) -> np.ndarray:
-    """Per-worker batch sizes b_j = B r_j / r_1 (host only; no GPU needed)."""
+RCD_BATCH_PROPORTIONAL = 0
+RCD_BATCH_AS_PRINTED = 1
+
+
+def rcd_batch_sizes(B: int, capacities: Sequence[float], rule: int = RCD_BATCH_PROPORTIONAL) -> np.ndarray:
+    """Per-worker batch sizes (host only; no GPU needed): b_j = B r_j / r_1, or with
+    ``rule=RCD_BATCH_AS_PRINTED`` the ratio as Algorithm 2 prints it, B r_1 / r_j."""
     r = np.ascontiguousarray(capacities, dtype=np.float64)
     out = np.empty(len(r), dtype=np.int64)
-    st = lib.rcd_batch_sizes(int(B), r.ctypes.data_as(C.c_void_p), len(r), out.ctypes.data_as(C.c_void_p))
+    if rule == RCD_BATCH_PROPORTIONAL:
+        st = lib.rcd_batch_sizes(int(B), r.ctypes.data_as(C.c_void_p), len(r), out.ctypes.data_as(C.c_void_p))
+    else:
+        st = lib.rcd_batch_sizes_rule(int(B), r.ctypes.data_as(C.c_void_p), len(r), int(rule), out.ctypes.data_as(C.c_void_p))
     if st != 0:
         raise RcdError(st, "rcd_batch_sizes")
     return out

@@ -166,35 +166,33 @@ static rcd_status check_capacities(rcd_ctx *ctx, const double *cap, int32_t W)
     return RCD_OK;
 }
 
-// Largest-remainder quotas.  Plain IEEE double operations in a fixed order.
+// Largest-remainder apportionment of M samples over W blocks (Algorithm 1's C_{l,j} = |V_l| r_j / sum r, made integer).
+// Shares are formed in IEEE double in index order (sum first, then M * r_j / sum, no contraction); every block gets
+// the integer part of its share, and the samples still unplaced go one each to the blocks ranked by fractional part
+// (a stable sort: equal fractions keep their index order, so ties fall to the lowest index).  Should rounding ever
+// make the integer parts add up to more than M (a share that rounds up onto an integer; no input found does), the
+// surplus is taken back from the other end of the same ranking.
 static void quotas_host(int64_t M, const double *r, int32_t W, int32_t *out)
 {
-    volatile double total = 0.0;
-    for (int32_t j = 0; j < W; ++j) total = total + r[j];
-    std::vector<double> rem((size_t)W);
-    int64_t used = 0;
+    volatile double sum = 0.0;
+    for (int32_t j = 0; j < W; ++j) sum = sum + r[j];
+    std::vector<double> frac((size_t)W);
+    std::vector<int32_t> rank((size_t)W);
+    int64_t placed = 0;
     for (int32_t j = 0; j < W; ++j) {
-        volatile double scaled = (double)M * r[j];
-        volatile double share = scaled / total;
-        double whole = floor(share);
+        volatile double numerator = (double)M * r[j];
+        volatile double share = numerator / sum;
+        const double whole = std::floor(share);
         out[j] = (int32_t)whole;
-        rem[j] = share - whole;
-        used += out[j];
+        frac[(size_t)j] = share - whole;
+        placed += (int64_t)whole;
+        rank[(size_t)j] = j;
     }
-    for (int64_t extra = M - used; extra > 0; --extra) {
-        int32_t pick = -1;
-        for (int32_t j = 0; j < W; ++j)
-            if (rem[j] >= 0.0 && (pick < 0 || rem[j] > rem[pick])) pick = j;
-        out[pick] += 1;
-        rem[pick] = -1.0;
-    }
-    for (int64_t over = used - M; over > 0; --over) {      // a share rounded up to an integer: give one back
-        int32_t pick = -1;
-        for (int32_t j = 0; j < W; ++j)
-            if (out[j] > 0 && rem[j] >= 0.0 && (pick < 0 || rem[j] <= rem[pick])) pick = j;
-        out[pick] -= 1;
-        rem[pick] = -1.0;
-    }
+    std::stable_sort(rank.begin(), rank.end(), [&](int32_t a, int32_t b) { return frac[(size_t)a] > frac[(size_t)b]; });
+    int64_t left = M - placed;
+    for (size_t k = 0; left > 0; k = (k + 1) % (size_t)W, --left) out[rank[k]] += 1;
+    for (size_t k = (size_t)W; left < 0 && k-- > 0;)
+        if (out[rank[k]] > 0) { out[rank[k]] -= 1; ++left; }
 }
 
 // Shared front half of rcd_partition and rcd_objective: class sizes, descriptors, workspace
@@ -533,18 +531,25 @@ rcd_status rcd_worker_lists(rcd_ctx *ctx, const int32_t *assignment_dev, int64_t
     return RCD_OK;
 }
 
-rcd_status rcd_batch_sizes(int64_t B, const double *capacities_host, int32_t W, int64_t *batch_sizes_host_out)
+rcd_status rcd_batch_sizes_rule(int64_t B, const double *capacities_host, int32_t W, rcd_batch_rule rule, int64_t *batch_sizes_host_out)
 {
     if (B <= 0 || W <= 0 || !capacities_host || !batch_sizes_host_out) return RCD_ERR_INVALID_ARG;
+    if (rule != RCD_BATCH_PROPORTIONAL && rule != RCD_BATCH_AS_PRINTED) return RCD_ERR_INVALID_ARG;
     for (int32_t j = 0; j < W; ++j)
         if (!(capacities_host[j] > 0.0) || !std::isfinite(capacities_host[j])) return RCD_ERR_INVALID_ARG;
     for (int32_t j = 0; j < W; ++j) {
-        const double x = (double)B * capacities_host[j] / capacities_host[0];
+        const double x = rule == RCD_BATCH_PROPORTIONAL ? (double)B * capacities_host[j] / capacities_host[0]
+                                                        : (double)B * capacities_host[0] / capacities_host[j];
         if (!(x < 9.0e18)) return RCD_ERR_INVALID_ARG;
         const int64_t b = (int64_t)std::floor(x + 0.5);
         batch_sizes_host_out[j] = b < 1 ? 1 : b;
     }
     return RCD_OK;
+}
+
+rcd_status rcd_batch_sizes(int64_t B, const double *capacities_host, int32_t W, int64_t *batch_sizes_host_out)
+{
+    return rcd_batch_sizes_rule(B, capacities_host, W, RCD_BATCH_PROPORTIONAL, batch_sizes_host_out);
 }
 
 rcd_status rcd_similarity(rcd_ctx *ctx, const void *X_dev, rcd_feat_dtype dtype, int64_t M, int64_t d,

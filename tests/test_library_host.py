@@ -51,6 +51,12 @@ def test_batch_sizes_match_oracle_and_closed_forms(binding):
     from oracle import rcd_oracle as orc
     assert binding.rcd_batch_sizes(32, [1, 1, 2, 4]).tolist() == [32, 32, 64, 128]
     assert binding.rcd_batch_sizes(10, [4, 1, 3]).tolist() == [10, 3, 8]
+    assert binding.rcd_batch_sizes(32, [1, 1, 2, 4], rule=binding.RCD_BATCH_AS_PRINTED).tolist() == [32, 32, 16, 8]
+    rng2 = np.random.default_rng(77)
+    for _ in range(50):
+        r2 = rng2.uniform(0.2, 9.0, size=int(rng2.integers(1, 20)))
+        B2 = int(rng2.integers(1, 500))
+        assert np.array_equal(binding.rcd_batch_sizes(B2, r2, rule=binding.RCD_BATCH_AS_PRINTED), orc.batch_sizes(B2, r2, rule="printed"))
     rng = np.random.default_rng(12)
     for _ in range(200):
         W = int(rng.integers(1, 70))
@@ -86,3 +92,23 @@ def test_no_oracle_in_the_product_path():
             if f.endswith((".py", ".cu", ".h", ".cuh")):
                 text = open(os.path.join(dirpath, f)).read()
                 assert "oracle" not in text.lower() or f == "workloads.py" and "oracle's tests" in text, f
+
+
+def test_quotas_decimal_grid_agrees_with_oracle_and_never_overshoots(binding):
+    """Capacities that are not representable in binary (tenths), every pair and a sample of triples, M up to 60: the
+    library's apportionment (ranked by a stable sort) equals the oracle's (repeated selection), the quotas add up to
+    M, and the integer parts of the shares never add up to more than M -- the branch that would take samples back is
+    not reached by any of these inputs."""
+    import itertools
+    import math
+    from oracle import rcd_oracle as orc
+    vals = [k / 10 for k in range(1, 31)]
+    cases = list(itertools.product(vals, repeat=2)) + list(itertools.product(vals[::3], repeat=3))
+    for r in cases:
+        total = 0.0
+        for x in r:
+            total = total + x
+        for M in (1, 7, 10, 33, 60):
+            assert sum(math.floor(M * x / total) for x in r) <= M
+            q = binding.rcd_quotas(M, r)
+            assert q.sum() == M and np.array_equal(q, orc.quotas(M, r))

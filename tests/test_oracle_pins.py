@@ -626,6 +626,10 @@ def test_worker_lists_are_a_stable_partition_with_quota_sizes():
 
 def test_batch_sizes_closed_forms():
     assert orc.batch_sizes(32, [1, 1, 2, 4]).tolist() == [32, 32, 64, 128]
+    # the ratio as Algorithm 2 prints it: B r_1 / r_i
+    assert orc.batch_sizes(32, [1, 1, 2, 4], rule="printed").tolist() == [32, 32, 16, 8]
+    assert orc.batch_sizes(10, [4, 1, 3], rule="printed").tolist() == [10, 40, 13]      # 13.33 -> 13
+    assert orc.batch_sizes(1, [1, 8], rule="printed").tolist() == [1, 1]
     assert orc.batch_sizes(32, [2, 1, 4]).tolist() == [32, 16, 64]          # relative to worker 1
     assert orc.batch_sizes(10, [4, 1, 3]).tolist() == [10, 3, 8]            # 2.5 -> 3, 7.5 -> 8: halves round up
     assert orc.batch_sizes(1, [8, 1]).tolist() == [1, 1]                    # never below one sample
