@@ -269,8 +269,7 @@ static rcd_status prepare(rcd_ctx *ctx, const void *features, rcd_feat_dtype dty
         int64_t run = 0;
         for (int32_t l = 0; l < L; ++l) {
             prefix[(size_t)l] = (int32_t)run;
-            const int64_t nt = (P.desc[(size_t)l].M + 127) / 128;
-            run += nt * (nt + 1) / 2;
+            run += sim_tiles(P.desc[(size_t)l].M);
             if (run > 0x7fffffffLL) return fail(ctx, RCD_ERR_UNSUPPORTED, "too many similarity tiles");
         }
         prefix[(size_t)L] = (int32_t)run;
@@ -574,7 +573,7 @@ rcd_status rcd_similarity(rcd_ctx *ctx, const void *X_dev, rcd_feat_dtype dtype,
     cls.L = (int32_t)batch;
     cls.maxM = M;
     cls.tilePrefixDev = nullptr;
-    cls.uniTiles = (int32_t)(((M + 127) / 128) * ((M + 127) / 128 + 1) / 2);
+    cls.uniTiles = (int32_t)sim_tiles(M);
     cls.upperTiles = batch * (int64_t)cls.uniTiles;
     ctx->kernelLaunches = 0;
     ctx->tcLaunches = 0;

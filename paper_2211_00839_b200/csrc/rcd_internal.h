@@ -72,7 +72,7 @@ struct SimClasses {
     DescSource src;
     int32_t L;
     int64_t maxM;
-    // tensor-core kernel: 128 x 128 tiles on or above the diagonal, listed class after class
+    // tensor-core kernel: 128 x 256 tiles that reach the diagonal or lie above it, listed class after class
     const int32_t *tilePrefixDev;   // [L+1] first tile index of every class (null: equal classes)
     int32_t uniTiles;               // tiles per class when the classes are equal
     int64_t upperTiles;             // tiles in all
@@ -151,6 +151,16 @@ inline int32_t pad4(int64_t m) { return (int32_t)((m + 3) / 4 * 4); }
 // elements, so that every row starts on a 32-byte boundary (one memory sector): the 16-byte pieces that
 // the sweeps copy then pair up into whole sectors.
 inline int32_t pad_row(int64_t m) { return (int32_t)((m + 7) / 8 * 8); }
+
+// Tiles the tensor-core similarity kernel computes for a class of M samples: 128 rows x 256 columns each, those that
+// reach the diagonal or lie above it (row block tm pairs with the column blocks from tm / 2 on).
+inline int64_t sim_tiles(int64_t M)
+{
+    const int64_t rowBlocks = (M + 127) / 128, colBlocks = (M + 255) / 256;
+    int64_t n = 0;
+    for (int64_t tm = 0; tm < rowBlocks; ++tm) n += colBlocks - tm / 2;
+    return n;
+}
 
 // Lays the workspace out at `base` (may be null to measure).  Returns total bytes.
 size_t layout_workspace(void *base, rcd_feat_dtype dtype, const Sizes &sz, Workspace *ws);

@@ -1,13 +1,16 @@
 // Tensor-core similarity kernel for sm_100a:  S_l = X_l X_l^T  per class (Section 3.1: similarities
 // from the feature vectors; int8 -> int32 exact, bf16 -> fp32).
 //
-// Persistent CTAs (one per SM) walk the 128 x 128 tiles on or above the diagonal of every class;
-// S is symmetric, so each off-diagonal tile is computed once and written twice (itself and its
-// mirror image), which halves the tensor work and the operand traffic.  Both operands are rows of
+// Persistent CTAs (one per SM) walk tiles of 128 rows x 256 columns of every class, those that reach the
+// diagonal or lie above it; S is symmetric, so each 128 x 128 block above the diagonal is computed once
+// and written twice (itself and its mirror image), which halves the tensor work and the operand traffic
+// (a tile whose left half lies below the diagonal computes its right half only).  The tile is twice as wide
+// as it is high because the kernel is bound by operand traffic from L2 at 128 x 128 (512 bytes of operands
+// per 32 768 multiply-adds and k-step): 128 x 256 moves 768 bytes per 65 536.  Both operands are rows of
 // the class-sorted feature matrix (K-major), brought in 128-byte k-slabs by TMA (cp.async.bulk.tensor,
 // 128-byte swizzle, out-of-range rows and columns filled with zeros) into a 4-stage shared-memory
 // ring; one thread issues tcgen05.mma (kind::i8, or kind::f16 with bf16 inputs) into one of two
-// accumulator buffers in tensor memory, so the next tile's MMAs run while four warps read the
+// 256-column accumulator buffers in tensor memory, so the next tile's MMAs run while four warps read the
 // previous accumulator back with tcgen05.ld, transpose 32 x 32 blocks through shared memory and
 // write S with coalesced 128-bit stores (pad columns as zeros).
 //
@@ -24,13 +27,13 @@ namespace rcd {
 namespace {
 
 constexpr int kTileM = 128;
-constexpr int kTileN = 128;
+constexpr int kTileN = 256;
 constexpr int kSlabBytes = 128;                         // k-slab per stage and operand row
 constexpr int kStages = 4;
-constexpr int kOperandBytes = kTileM * kSlabBytes;      // 16 KB
-constexpr int kStageBytes = 2 * kOperandBytes;          // A + B
+constexpr int kOperandBytes = kTileM * kSlabBytes;      // 16 KB: 128 rows of one k-slab
+constexpr int kStageBytes = 3 * kOperandBytes;          // A (128 rows) + B (256 rows)
 constexpr int kTcThreads = 192;
-constexpr int kTmemCols = 256;                           // two accumulator buffers of 128 columns
+constexpr int kTmemCols = 512;                           // two accumulator buffers of 256 columns
 constexpr uint32_t kSpinLimit = 1u << 22;               // polls of ~64 ns: a quarter of a second
 
 struct __align__(8) TcShared {
@@ -130,9 +133,11 @@ __device__ __forceinline__ void mbar_arrive(uint64_t *bar)
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" :: "r"(smem_addr(bar)) : "memory");
 }
 
-// Tile idx of the launch -> (class, row tile, column tile).  Only tiles on or above the diagonal
-// are listed (S is symmetric); a class with nt row tiles owns nt*(nt+1)/2 consecutive indices.
-struct TileCoord { int l, tm, tn; };
+// Tile idx of the launch -> (class, row block tm of 128 rows, column block sn of 256 columns).  A class lists, row
+// block after row block, the tiles with sn >= tm / 2: those that contain a 128 x 128 block on or above the diagonal.
+// skip = 128 when the left half of the tile lies below the diagonal (tm odd, sn = tm / 2): that half is the mirror
+// image of a block another tile computes, so only the right half is computed.
+struct TileCoord { int l, tm, sn, skip; };
 __device__ __forceinline__ TileCoord decode_tile(const DescSource &src, const int32_t *__restrict__ prefix, int L, int uniTiles, int idx)
 {
     TileCoord t;
@@ -150,10 +155,16 @@ __device__ __forceinline__ TileCoord decode_tile(const DescSource &src, const in
         local = idx - t.l * uniTiles;
     }
     const ClassDesc c = src.get(t.l);
-    int rowLen = (c.M + kTileM - 1) / kTileM;
+    const int colBlocks = (c.M + kTileN - 1) / kTileN;
     t.tm = 0;
-    while (local >= rowLen) { local -= rowLen; --rowLen; ++t.tm; }
-    t.tn = t.tm + local;
+    for (;;) {
+        const int rowLen = colBlocks - t.tm / 2;
+        if (local < rowLen) break;
+        local -= rowLen;
+        ++t.tm;
+    }
+    t.sn = t.tm / 2 + local;
+    t.skip = (2 * t.sn < t.tm) ? kTileM : 0;
     return t;
 }
 
@@ -194,16 +205,16 @@ __global__ void __launch_bounds__(kTcThreads, 1) sim_tc_kernel(const __grid_cons
             for (int idx = blockIdx.x; idx < totalTiles && ok; idx += gridDim.x) {
                 const TileCoord t = decode_tile(src, tilePrefix, L, uniTiles, idx);
                 const ClassDesc c = src.get(t.l);
-                const int rowA = c.row0 + t.tm * kTileM, rowB = c.row0 + t.tn * kTileN;
-                const bool diag = (t.tm == t.tn);        // A and B are the same rows: one copy serves both
+                const int rowA = c.row0 + t.tm * kTileM, rowB = c.row0 + t.sn * kTileN + t.skip;
+                const int halves = (kTileN - t.skip) / kTileM;         // 128-row pieces of B to bring in: 2, or 1
                 for (int kb = 0; kb < numSlabs; ++kb, ++it) {
                     const int s = it % kStages;
                     if (!mbar_wait(&sh.empty[s], ((it / kStages) & 1) ^ 1, &sh)) { ok = false; break; }
                     unsigned char *a = tiles + (size_t)s * kStageBytes;
-                    mbar_expect_tx(&sh.full[s], diag ? kOperandBytes : kStageBytes);
+                    mbar_expect_tx(&sh.full[s], (1 + halves) * kOperandBytes);
                     const int k0 = kb * (kInt8 ? kSlabBytes : kSlabBytes / 2);         // element coordinate
                     tma_load_2d(a, &map, k0, rowA, &sh.full[s]);
-                    if (!diag) tma_load_2d(a + kOperandBytes, &map, k0, rowB, &sh.full[s]);
+                    for (int h = 0; h < halves; ++h) tma_load_2d(a + (1 + h) * kOperandBytes, &map, k0, rowB + h * kTileM, &sh.full[s]);
                 }
             }
             // after an abort: let the copies already issued land before the CTA leaves
@@ -218,14 +229,14 @@ __global__ void __launch_bounds__(kTcThreads, 1) sim_tc_kernel(const __grid_cons
         // ---------------- MMA issuer ----------------
         if (lane == 0) {
             // instruction descriptor: D format, A/B format, K-major operands, N and M of the tile
-            const uint32_t idesc = (kInt8 ? (2u << 4) | (1u << 7) | (1u << 10)       // S32 accumulate, S8 x S8
-                                          : (1u << 4) | (1u << 7) | (1u << 10))      // F32 accumulate, BF16 x BF16
-                                   | ((uint32_t)(kTileN >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
+            const uint32_t idescBase = (kInt8 ? (2u << 4) | (1u << 7) | (1u << 10)   // S32 accumulate, S8 x S8
+                                              : (1u << 4) | (1u << 7) | (1u << 10))  // F32 accumulate, BF16 x BF16
+                                       | ((uint32_t)(kTileM >> 4) << 24);
             uint32_t it = 0, nt = 0;
             bool ok = true;
             for (int idx = blockIdx.x; idx < totalTiles && ok; idx += gridDim.x, ++nt) {
                 const TileCoord t = decode_tile(src, tilePrefix, L, uniTiles, idx);
-                const bool diag = (t.tm == t.tn);
+                const uint32_t idesc = idescBase | ((uint32_t)((kTileN - t.skip) >> 3) << 17);   // N = 256, or 128 for a half tile
                 const uint32_t buf = nt & 1;
                 // the epilogue must have drained this accumulator buffer (two tiles ago)
                 if (!mbar_wait(&sh.accEmpty[buf], ((nt >> 1) & 1) ^ 1, &sh)) { ok = false; break; }
@@ -237,7 +248,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) sim_tc_kernel(const __grid_cons
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const uint32_t aAddr = smem_addr(tiles + (size_t)s * kStageBytes);
                     const uint64_t descA = make_smem_desc(aAddr);
-                    const uint64_t descB = diag ? descA : make_smem_desc(aAddr + kOperandBytes);
+                    const uint64_t descB = make_smem_desc(aAddr + kOperandBytes);
 #pragma unroll
                     for (int k = 0; k < kSlabBytes / 32; ++k)          // one MMA consumes 32 bytes of k per row
                         mma_issue<kInt8>(tmemD, descA + (uint64_t)(2 * k), descB + (uint64_t)(2 * k), idesc, (kb > 0 || k > 0) ? 1u : 0u);
@@ -254,24 +265,27 @@ __global__ void __launch_bounds__(kTcThreads, 1) sim_tc_kernel(const __grid_cons
         for (int idx = blockIdx.x; idx < totalTiles; idx += gridDim.x, ++nt) {
             const TileCoord t = decode_tile(src, tilePrefix, L, uniTiles, idx);
             const ClassDesc c = src.get(t.l);
-            const int rowA = t.tm * kTileM, rowB = t.tn * kTileN;      // class-local
-            const bool diag = (t.tm == t.tn);
+            const int rowA = t.tm * kTileM, colB = t.sn * kTileN + t.skip;   // class-local: first row, first column computed
             const uint32_t buf = nt & 1;
             if (!mbar_wait(&sh.accFull[buf], (nt >> 1) & 1, &sh)) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             if (*(volatile int32_t *)&sh.abort) break;
             uint32_t *Sl = S + c.sOff;
             const int cg = (lane & 7) * 4;                             // this lane's 4 columns of a 32-wide block
+            const int nCb = (kTileN - t.skip) / 32;
 #pragma unroll 1
-            for (int cb = 0; cb < kTileN / 32; ++cb) {
+            for (int cb = 0; cb < nCb; ++cb) {
+                // the 128 x 128 block this column block belongs to lies on the diagonal (stored once) or above it
+                // (stored twice: itself and its mirror image)
+                const bool diag = (colB + cb * 32) / kTileM == t.tm;
                 uint32_t v[32];
                 tmem_load_32cols(tmemBase + buf * kTileN + ((uint32_t)(q * 32) << 16) + (uint32_t)(cb * 32), v);
 #pragma unroll
                 for (int j = 0; j < 32; ++j) stage32[ew][lane][j] = v[j];         // lane = row inside the quarter
                 __syncwarp();
-                // block rows -> S[rowA + ..][rowB + ..]: 8 lanes cover 32 columns with 128-bit stores, 4 rows per pass
+                // block rows -> S[rowA + ..][colB + ..]: 8 lanes cover 32 columns with 128-bit stores, 4 rows per pass
                 {
-                    const int col = rowB + cb * 32 + cg;
+                    const int col = colB + cb * 32 + cg;
 #pragma unroll
                     for (int pass = 0; pass < 8; ++pass) {
                         const int r = pass * 4 + (lane >> 3);
@@ -286,13 +300,13 @@ __global__ void __launch_bounds__(kTcThreads, 1) sim_tc_kernel(const __grid_cons
                         }
                     }
                 }
-                // the mirrored block -> S[rowB + ..][rowA + ..] (tiles below the diagonal are never computed)
+                // the mirrored block -> S[colB + ..][rowA + ..] (blocks below the diagonal are never computed)
                 if (!diag) {
                     const int col = rowA + q * 32 + cg;
 #pragma unroll
                     for (int pass = 0; pass < 8; ++pass) {
                         const int jj = pass * 4 + (lane >> 3);
-                        const int row = rowB + cb * 32 + jj;
+                        const int row = colB + cb * 32 + jj;
                         if (row < c.M && col < c.ld) {
                             uint4 o;
                             o.x = col + 0 < c.M ? stage32[ew][cg + 0][jj] : 0u;
