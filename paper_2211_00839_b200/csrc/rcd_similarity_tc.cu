@@ -10,11 +10,13 @@
 // the class-sorted feature matrix (K-major), brought in 128-byte k-slabs by TMA (cp.async.bulk.tensor,
 // 128-byte swizzle, out-of-range rows and columns filled with zeros) into a 4-stage shared-memory
 // ring; one thread issues tcgen05.mma (kind::i8, or kind::f16 with bf16 inputs) into one of two
-// 256-column accumulator buffers in tensor memory, so the next tile's MMAs run while four warps read the
+// 256-column accumulator buffers in tensor memory, so the next tile's MMAs run while eight warps read the
 // previous accumulator back with tcgen05.ld, transpose 32 x 32 blocks through shared memory and
 // write S with coalesced 128-bit stores (pad columns as zeros).
 //
-// Warp roles: 0 = TMA producer, 1 = TMEM allocation + MMA issue, 2..5 = epilogue.
+// Warp roles: 0 = TMA producer, 1 = TMEM allocation + MMA issue, 2..9 = epilogue (two warps per quarter of the
+// tensor-memory lanes, one taking the even 32-column blocks of a tile and one the odd ones; the load of a warp's
+// next block from tensor memory is in flight while it writes the current one).
 // Every wait on an mbarrier is bounded: on expiry the CTA records kDevTimeout in the status
 // word, stops issuing work, still waits (bounded) for the copies it has in flight, releases its
 // tensor memory and returns.
@@ -32,7 +34,8 @@ constexpr int kSlabBytes = 128;                         // k-slab per stage and 
 constexpr int kStages = 4;
 constexpr int kOperandBytes = kTileM * kSlabBytes;      // 16 KB: 128 rows of one k-slab
 constexpr int kStageBytes = 3 * kOperandBytes;          // A (128 rows) + B (256 rows)
-constexpr int kTcThreads = 192;
+constexpr int kEpiWarps = 8;                            // two per quarter of the TMEM lanes
+constexpr int kTcThreads = 64 + 32 * kEpiWarps;
 constexpr int kTmemCols = 512;                           // two accumulator buffers of 256 columns
 constexpr uint32_t kSpinLimit = 1u << 22;               // polls of ~64 ns: a quarter of a second
 
@@ -125,6 +128,10 @@ __device__ __forceinline__ void tmem_load_32cols(uint32_t taddr, uint32_t (&v)[3
                    "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
                    "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
                  : "r"(taddr) : "memory");
+}
+// The registers of an earlier tmem_load_32cols hold their values only after this wait.
+__device__ __forceinline__ void tmem_load_wait()
+{
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
@@ -137,7 +144,7 @@ __device__ __forceinline__ void mbar_arrive(uint64_t *bar)
 // block after row block, the tiles with sn >= tm / 2: those that contain a 128 x 128 block on or above the diagonal.
 // skip = 128 when the left half of the tile lies below the diagonal (tm odd, sn = tm / 2): that half is the mirror
 // image of a block another tile computes, so only the right half is computed.
-struct TileCoord { int l, tm, sn, skip; };
+struct TileCoord { int l, tm, sn, skip, n; };         // n: columns computed, from column sn * 256 + skip on
 __device__ __forceinline__ TileCoord decode_tile(const DescSource &src, const int32_t *__restrict__ prefix, int L, int uniTiles, int idx)
 {
     TileCoord t;
@@ -165,6 +172,9 @@ __device__ __forceinline__ TileCoord decode_tile(const DescSource &src, const in
     }
     t.sn = t.tm / 2 + local;
     t.skip = (2 * t.sn < t.tm) ? kTileM : 0;
+    // no further than the rows of S reach, pad columns included (in steps of 32 columns: the epilogue's block, and a
+    // legal N of the MMA)
+    t.n = min(kTileN - t.skip, (c.ld - (t.sn * kTileN + t.skip) + 31) & ~31);
     return t;
 }
 
@@ -178,13 +188,13 @@ __global__ void __launch_bounds__(kTcThreads, 1) sim_tc_kernel(const __grid_cons
     // operand stages need 1024-byte alignment for the 128-byte swizzle pattern
     unsigned char *tiles = reinterpret_cast<unsigned char *>(((uintptr_t)smemRaw + 1023) & ~(uintptr_t)1023);
     __shared__ TcShared sh;
-    __shared__ uint32_t stage32[4][32][33];             // per epilogue warp: one 32 x 32 block, padded
+    __shared__ uint32_t stage32[kEpiWarps][32][33];             // per epilogue warp: one 32 x 32 block, padded
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(&sh.accFull[b], 1); mbar_init(&sh.accEmpty[b], 4); }
+        for (int b = 0; b < 2; ++b) { mbar_init(&sh.accFull[b], 1); mbar_init(&sh.accEmpty[b], kEpiWarps); }
         sh.abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -206,7 +216,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) sim_tc_kernel(const __grid_cons
                 const TileCoord t = decode_tile(src, tilePrefix, L, uniTiles, idx);
                 const ClassDesc c = src.get(t.l);
                 const int rowA = c.row0 + t.tm * kTileM, rowB = c.row0 + t.sn * kTileN + t.skip;
-                const int halves = (kTileN - t.skip) / kTileM;         // 128-row pieces of B to bring in: 2, or 1
+                const int halves = (t.n + kTileM - 1) / kTileM;         // 128-row pieces of B to bring in: 2, or 1
                 for (int kb = 0; kb < numSlabs; ++kb, ++it) {
                     const int s = it % kStages;
                     if (!mbar_wait(&sh.empty[s], ((it / kStages) & 1) ^ 1, &sh)) { ok = false; break; }
@@ -236,7 +246,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) sim_tc_kernel(const __grid_cons
             bool ok = true;
             for (int idx = blockIdx.x; idx < totalTiles && ok; idx += gridDim.x, ++nt) {
                 const TileCoord t = decode_tile(src, tilePrefix, L, uniTiles, idx);
-                const uint32_t idesc = idescBase | ((uint32_t)((kTileN - t.skip) >> 3) << 17);   // N = 256, or 128 for a half tile
+                const uint32_t idesc = idescBase | ((uint32_t)(t.n >> 3) << 17);   // N = 256, less for a half tile or at the class's edge
                 const uint32_t buf = nt & 1;
                 // the epilogue must have drained this accumulator buffer (two tiles ago)
                 if (!mbar_wait(&sh.accEmpty[buf], ((nt >> 1) & 1) ^ 1, &sh)) { ok = false; break; }
@@ -261,6 +271,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) sim_tc_kernel(const __grid_cons
         // ---------------- epilogue: TMEM -> registers -> shared (transpose) -> global ----------------
         const int q = warp & 3;                                        // TMEM lane quarter this warp may read
         const int ew = warp - 2;
+        const int half = ew >> 2;                                      // which column blocks of the tile: even or odd
         uint32_t nt = 0;
         for (int idx = blockIdx.x; idx < totalTiles; idx += gridDim.x, ++nt) {
             const TileCoord t = decode_tile(src, tilePrefix, L, uniTiles, idx);
@@ -272,17 +283,21 @@ __global__ void __launch_bounds__(kTcThreads, 1) sim_tc_kernel(const __grid_cons
             if (*(volatile int32_t *)&sh.abort) break;
             uint32_t *Sl = S + c.sOff;
             const int cg = (lane & 7) * 4;                             // this lane's 4 columns of a 32-wide block
-            const int nCb = (kTileN - t.skip) / 32;
+            const int nCb = t.n / 32;
+            const uint32_t tmemRow = tmemBase + buf * kTileN + ((uint32_t)(q * 32) << 16);
+            uint32_t v[32];
+            if (half < nCb) tmem_load_32cols(tmemRow + (uint32_t)(half * 32), v);
 #pragma unroll 1
-            for (int cb = 0; cb < nCb; ++cb) {
+            for (int cb = half; cb < nCb; cb += kEpiWarps / 4) {
                 // the 128 x 128 block this column block belongs to lies on the diagonal (stored once) or above it
                 // (stored twice: itself and its mirror image)
                 const bool diag = (colB + cb * 32) / kTileM == t.tm;
-                uint32_t v[32];
-                tmem_load_32cols(tmemBase + buf * kTileN + ((uint32_t)(q * 32) << 16) + (uint32_t)(cb * 32), v);
+                tmem_load_wait();
 #pragma unroll
                 for (int j = 0; j < 32; ++j) stage32[ew][lane][j] = v[j];         // lane = row inside the quarter
                 __syncwarp();
+                // the next block of this warp travels from tensor memory while this one is written out
+                if (cb + kEpiWarps / 4 < nCb) tmem_load_32cols(tmemRow + (uint32_t)((cb + kEpiWarps / 4) * 32), v);
                 // block rows -> S[rowA + ..][colB + ..]: 8 lanes cover 32 columns with 128-bit stores, 4 rows per pass
                 {
                     const int col = colB + cb * 32 + cg;
