@@ -504,6 +504,16 @@ __device__ __forceinline__ int4 ld_stream(const int4 *p)
     return v;
 }
 
+// The same load as a volatile statement: it stays where it is written (the compiler neither sinks it into the
+// branch that uses its result nor merges it with a neighbour), so that several of them are in flight at once.
+__device__ __forceinline__ int4 ld_stream_here(const int4 *p)
+{
+    int4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.s32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+
 // Barrier over the `threads` threads of one team of warps (named barriers 1..15; 0 is the CTA's).
 __device__ __forceinline__ void team_sync(int id, int threads)
 {
@@ -1636,7 +1646,7 @@ __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, i
                         for (int q = 0; q < 12; ++q) {
                             const int col = list[e0 + q < total ? e0 + q : e0].x;
                             const int4 *rp = reinterpret_cast<const int4 *>(Sl + (int64_t)col * c.ld);
-                            x[q] = i < ld4 ? ld_stream(rp + i) : make_int4(0, 0, 0, 0);
+                            x[q] = i < ld4 ? ld_stream_here(rp + i) : make_int4(0, 0, 0, 0);
                         }
 #pragma unroll
                         for (int q = 0; q < 12; ++q) {
@@ -1659,7 +1669,7 @@ __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, i
 #pragma unroll
                             for (int k = 0; k < 3; ++k) {
                                 const int i = (int)threadIdx.x + k * kSelectThreads;
-                                x[q][k] = i < ld4 ? ld_stream(rp + i) : make_int4(0, 0, 0, 0);
+                                x[q][k] = i < ld4 ? ld_stream_here(rp + i) : make_int4(0, 0, 0, 0);
                             }
                         }
 #pragma unroll
