@@ -1428,10 +1428,14 @@ __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, i
         for (int i = threadIdx.x; i < ld4; i += kSelectThreads) thrAcc[i] = top;
     }
     int chainLen = 0;
+    __shared__ int shRaised;                               // integer path: raised columns of the pick in hand
+    __shared__ unsigned long long shStat[3];               // corrections of this chain: how many, rows of S, bytes (thread 0 only)
+    if (threadIdx.x == 0) shStat[0] = shStat[1] = shStat[2] = 0ull;
     __shared__ PlanGlobals shPre;
     if (threadIdx.x == 0) shPre = plan_globals(prm, l);     // (in flight under the first argmax; read after its barriers)
 
     for (;;) {
+        if (threadIdx.x == 0) shRaised = 0;                 // (read last before the previous pick's final barrier; used after two more)
         const GV *G = prm.gains + c.vOff + (int64_t)j * c.ld;
         // v* = argmax over the unassigned samples, ties -> lowest class-local index.  Walks all
         // samples with independent, coalesced loads (pos[v] < 0 marks an assigned sample).
@@ -1593,14 +1597,36 @@ __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, i
                 if (i < ld4) {
                     const int4 r = scratch[i], o = scratch[ld4 + i];
                     const int4 m = max_int4<SV>(o, r);
-                    cov[i] = m;
                     if (thrAcc) thrAcc[i] = min_int4<SV>(thrAcc[i], m);
                     const unsigned b = (rose<SV>(r.x, o.x) ? 1u : 0u) | (rose<SV>(r.y, o.y) ? 2u : 0u) |
                                        (rose<SV>(r.z, o.z) ? 4u : 0u) | (rose<SV>(r.w, o.w) ? 8u : 0u);
+                    if (b) cov[i] = m;                            // (elsewhere the vector keeps its value)
                     mask |= b << (4 * k);
                     cnt += __popc(b);
                 }
             }
+            int4 *list = scratch + 6 * ld4;                      // (column, old coverage, new coverage, -)
+            int total;
+            bool few;
+            if constexpr (Arith<SV>::kInt) {
+                // integer corrections are exact in any order: the threads that found raised columns append them
+                int at = cnt ? atomicAdd(&shRaised, cnt) : 0;
+#pragma unroll
+                for (int k = 0; k < 3; ++k) {
+                    const int i = (int)threadIdx.x + k * kSelectThreads;
+                    const unsigned b = (mask >> (4 * k)) & 15u;
+                    if (b) {
+                        const int4 r = scratch[i], o = scratch[ld4 + i];
+                        if ((b & 1u) && at < kDeltaMax) list[at++] = make_int4(4 * i + 0, o.x, r.x, 0);
+                        if ((b & 2u) && at < kDeltaMax) list[at++] = make_int4(4 * i + 1, o.y, r.y, 0);
+                        if ((b & 4u) && at < kDeltaMax) list[at++] = make_int4(4 * i + 2, o.z, r.z, 0);
+                        if ((b & 8u) && at < kDeltaMax) list[at++] = make_int4(4 * i + 3, o.w, r.w, 0);
+                    }
+                }
+                __syncthreads();
+                total = shRaised;
+                few = total <= prm.deltaMax;
+            } else {
             // where this thread's columns go in the list: an exclusive prefix sum over the CTA, so that the list (and with it
             // the order of the floating-point corrections) does not depend on timing
             int incl = cnt;
@@ -1610,15 +1636,14 @@ __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, i
             }
             if (lane == 31) shV[warp] = incl;                    // (the argmax is over: its per-warp array is free)
             __syncthreads();
-            int base = 0, total = 0;
+            int base = 0; total = 0;
 #pragma unroll
             for (int w = 0; w < kSelectThreads / 32; ++w) {
                 const int t = shV[w];
                 if (w < warp) base += t;
                 total += t;
             }
-            int4 *list = scratch + 6 * ld4;                      // (column, old coverage, new coverage, -)
-            const bool few = total <= prm.deltaMax;
+            few = total <= prm.deltaMax;
             if (few) {
                 int at = base + incl - cnt;
 #pragma unroll
@@ -1635,6 +1660,8 @@ __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, i
                 }
             }
             __syncthreads();
+            }
+            unsigned changed = 0;                                // bit k: the correction moved one of this thread's gains of piece k
             if (few) {
                 const SV *Sl = prm.S + c.sOff;
                 if (ld4 <= kSelectThreads) {
@@ -1652,10 +1679,10 @@ __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, i
                         for (int q = 0; q < 12; ++q) {
                             if (e0 + q < total) {
                                 const int4 ent = list[e0 + q];              // (shared memory, the same word for every thread)
-                                gj[0][0] -= delta_term<SV>(x[q].x, ent.y, ent.z);
-                                gj[0][1] -= delta_term<SV>(x[q].y, ent.y, ent.z);
-                                gj[0][2] -= delta_term<SV>(x[q].z, ent.y, ent.z);
-                                gj[0][3] -= delta_term<SV>(x[q].w, ent.y, ent.z);
+                                const auto d0 = delta_term<SV>(x[q].x, ent.y, ent.z), d1 = delta_term<SV>(x[q].y, ent.y, ent.z);
+                                const auto d2 = delta_term<SV>(x[q].z, ent.y, ent.z), d3 = delta_term<SV>(x[q].w, ent.y, ent.z);
+                                gj[0][0] -= d0; gj[0][1] -= d1; gj[0][2] -= d2; gj[0][3] -= d3;
+                                changed |= (d0 != 0 || d1 != 0 || d2 != 0 || d3 != 0) ? 1u : 0u;
                             }
                         }
                     }
@@ -1669,7 +1696,7 @@ __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, i
 #pragma unroll
                             for (int k = 0; k < 3; ++k) {
                                 const int i = (int)threadIdx.x + k * kSelectThreads;
-                                x[q][k] = i < ld4 ? ld_stream_here(rp + i) : make_int4(0, 0, 0, 0);
+                                x[q][k] = (i < ld4 && e0 + q < total) ? ld_stream_here(rp + i) : make_int4(0, 0, 0, 0);
                             }
                         }
 #pragma unroll
@@ -1678,10 +1705,10 @@ __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, i
                                 const int4 ent = list[e0 + q];
 #pragma unroll
                                 for (int k = 0; k < 3; ++k) {
-                                    gj[k][0] -= delta_term<SV>(x[q][k].x, ent.y, ent.z);
-                                    gj[k][1] -= delta_term<SV>(x[q][k].y, ent.y, ent.z);
-                                    gj[k][2] -= delta_term<SV>(x[q][k].z, ent.y, ent.z);
-                                    gj[k][3] -= delta_term<SV>(x[q][k].w, ent.y, ent.z);
+                                    const auto d0 = delta_term<SV>(x[q][k].x, ent.y, ent.z), d1 = delta_term<SV>(x[q][k].y, ent.y, ent.z);
+                                    const auto d2 = delta_term<SV>(x[q][k].z, ent.y, ent.z), d3 = delta_term<SV>(x[q][k].w, ent.y, ent.z);
+                                    gj[k][0] -= d0; gj[k][1] -= d1; gj[k][2] -= d2; gj[k][3] -= d3;
+                                    changed |= (d0 != 0 || d1 != 0 || d2 != 0 || d3 != 0) ? (1u << k) : 0u;
                                 }
                             }
                         }
@@ -1691,7 +1718,7 @@ __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, i
 #pragma unroll
                     for (int k = 0; k < 3; ++k) {
                         const int i = (int)threadIdx.x + k * kSelectThreads;
-                        if (i < ld4) {
+                        if (i < ld4 && ((changed >> k) & 1u)) {        // (most gains keep their value: nothing to store)
                             if constexpr (Arith<SV>::kInt) {
                                 reinterpret_cast<longlong2 *>(Gj + 4 * i)[0] = make_longlong2(gj[k][0], gj[k][1]);
                                 reinterpret_cast<longlong2 *>(Gj + 4 * i)[1] = make_longlong2(gj[k][2], gj[k][3]);
@@ -1705,9 +1732,9 @@ __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, i
                     // block j is up to date again
                     shPlan.open[j] = (uint8_t)1;
                     prm.valid[(int64_t)l * prm.W + j] = 1;
-                    atomicAdd(&prm.phaseNs[15], 1ull);
-                    atomicAdd(&prm.phaseNs[16], (unsigned long long)total);
-                    atomicAdd(&prm.phaseNs[12], (unsigned long long)(total + 2) * (unsigned long long)c.ld * sizeof(SV) + 2ull * c.ld * sizeof(GV));
+                    shStat[0] += 1ull;
+                    shStat[1] += (unsigned long long)total;
+                    shStat[2] += (unsigned long long)(total + 2) * (unsigned long long)c.ld * sizeof(SV) + 2ull * c.ld * sizeof(GV);
                 }
             }
             // (a compiler barrier: without it the correction above and the choice of the next block below are scheduled
@@ -1736,6 +1763,11 @@ __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, i
         nR -= 1;
         j = shPlan.nextJ;
         if (nR == 0 || j < 0 || shPlan.needSweep) break;
+    }
+    if (threadIdx.x == 0 && shStat[0]) {
+        atomicAdd(&prm.phaseNs[15], shStat[0]);
+        atomicAdd(&prm.phaseNs[16], shStat[1]);
+        atomicAdd(&prm.phaseNs[12], shStat[2]);
     }
     if (keep && threadIdx.x == 0) { keep[0] = nR; keep[1] = j; }     // (j = -1 after an inconsistency: the class is given up)
     if (!res) plan_store_lazy(prm, l, shPlan);                       // (a CTA that owns its class keeps this state in shared memory)
