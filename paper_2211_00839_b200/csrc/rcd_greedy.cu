@@ -1428,19 +1428,57 @@ __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, i
         for (int i = threadIdx.x; i < ld4; i += kSelectThreads) thrAcc[i] = top;
     }
     int chainLen = 0;
-    __shared__ int shRaised;                               // integer path: raised columns of the pick in hand
+    __shared__ int shRaised[2];                            // integer path: raised columns of the pick in hand (slot: pick parity)
+    // The next v* of a block, noted ahead of time.  When the stored gains of block p are corrected in place they all stand
+    // in registers, so every warp notes its best unassigned candidate among them.  At p's next turn the best of those is
+    // the argmax, unless it has been assigned meanwhile (the stored gains of p do not change in between): then no stored
+    // gain is loaded and the pick needs neither of the argmax's two barriers.  Blocks 0..kCacheBlocks-1; the notes sit
+    // behind the list of raised columns.
+    constexpr int kCacheBlocks = 8;
+    constexpr int kWarps = kSelectThreads / 32;
+    __shared__ uint8_t shNoted[kCacheBlocks];
+    GV *noteG = reinterpret_cast<GV *>(scratch + 6 * ld4 + kDeltaMax);             // [kCacheBlocks][kWarps]
+    int *noteV = reinterpret_cast<int *>(noteG + kCacheBlocks * kWarps);
+    const bool notes = kDelta && deltaAllowed && prm.lazyFrom < 0 &&
+                       (int64_t)6 * c.ld * (int64_t)sizeof(SV) + (int64_t)kDeltaMax * 16 +
+                       (int64_t)kCacheBlocks * kWarps * (int64_t)(sizeof(GV) + sizeof(int)) <= scratchBytes;
+    if (threadIdx.x < kCacheBlocks) shNoted[threadIdx.x] = 0;       // (a pass may have rewritten any block's stored gains)
+    if (threadIdx.x == 0) shRaised[0] = shRaised[1] = 0;
+    __syncthreads();
     __shared__ unsigned long long shStat[3];               // corrections of this chain: how many, rows of S, bytes (thread 0 only)
     if (threadIdx.x == 0) shStat[0] = shStat[1] = shStat[2] = 0ull;
     __shared__ PlanGlobals shPre;
     if (threadIdx.x == 0) shPre = plan_globals(prm, l);     // (in flight under the first argmax; read after its barriers)
 
     for (;;) {
-        if (threadIdx.x == 0) shRaised = 0;                 // (read last before the previous pick's final barrier; used after two more)
+        const int par = chainLen & 1;
+        if (threadIdx.x == 0) shRaised[par ^ 1] = 0;        // (the next pick's slot: read last before the previous pick's final barrier)
         const GV *G = prm.gains + c.vOff + (int64_t)j * c.ld;
         // v* = argmax over the unassigned samples, ties -> lowest class-local index.  Walks all
         // samples with independent, coalesced loads (pos[v] < 0 marks an assigned sample).
         GV bestG = 0;
         int bestV = INT_MAX;
+        bool fast = false;                                  // v* comes from the notes: no argmax
+        if constexpr (kDelta) {
+            if (notes && j < kCacheBlocks && shNoted[j]) {
+                bestG = lane < kWarps ? noteG[j * kWarps + lane] : (GV)0;
+                bestV = lane < kWarps ? noteV[j * kWarps + lane] : INT_MAX;
+                for (int off = 16; off > 0; off >>= 1) {
+                    GV oG = __shfl_xor_sync(0xffffffffu, bestG, off);
+                    int oV = __shfl_xor_sync(0xffffffffu, bestV, off);
+                    if (oV != INT_MAX && (bestV == INT_MAX || oG > bestG || (oG == bestG && oV < bestV))) { bestG = oG; bestV = oV; }
+                }
+                fast = bestV != INT_MAX && (res ? shPos[bestV] : pos[bestV]) >= 0;
+                if (!fast) { bestG = 0; bestV = INT_MAX; }
+            }
+        }
+        if (fast) {
+            if (res && chainLen == 0 && threadIdx.x == 0) __threadfence();
+            if (pendDst) {
+                fold_pending<SV>(pendDst, scratch, ld4, thrAcc);
+                pendDst = nullptr;
+            }
+        } else {
         // batches of kArgmaxBatch samples per thread: all loads of a batch are issued before the
         // first comparison, so a class of up to kArgmaxBatch * kSelectThreads samples costs one
         // memory round trip
@@ -1515,7 +1553,8 @@ __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, i
             __syncwarp();
         }
         __syncthreads();
-        if (shPick == kPickMiss) {
+        }
+        if (!fast && shPick == kPickMiss) {
             // (the chain ends here: its last act is to schedule the pass this block needs)
             if (warp == 0) plan_decide(prm, l, c, nR, round + 1, shPlan, &shPre);
             __syncthreads();
@@ -1524,7 +1563,18 @@ __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, i
         }
         if (threadIdx.x == 0 && chainLen < kSparseMax) shChain[chainLen] = j;
         ++chainLen;
-        const int vstar = shPick;
+        const int vstar = fast ? bestV : shPick;
+        // (fast: thread 0 books the pick in the plan after the next barrier, so the room still counts this sample)
+        const int roomAfter = fast ? shPlan.room[j] - 1 : shPlan.room[j];
+        auto book_fast = [&]() {                             // thread 0, fast picks: what warp 0 does after an argmax
+            shPlan.f[j] += (FV)bestG;
+            shPlan.room[j] = roomAfter;
+            shPlan.open[j] = (uint8_t)((roomAfter > 0 ? 1 : 0) | 2);
+            const int64_t at = (int64_t)l * prm.W + j;
+            prm.valid[at] = 0;
+            prm.fval[at] = shPlan.f[j];
+            prm.cnt[at] = shPlan.quota[j] - roomAfter;
+        };
         if (vstar == INT_MAX || vstar < 0 || vstar >= c.M) {
             if (threadIdx.x == 0) atomicOr(prm.status, kDevBadState);
             j = -1;
@@ -1535,9 +1585,11 @@ __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, i
         const int4 *row = reinterpret_cast<const int4 *>(prm.S + c.sOff + (int64_t)vstar * c.ld);
         int4 *cov = reinterpret_cast<int4 *>(prm.cover + c.vOff + (int64_t)j * c.ld);
         if (threadIdx.x == kSelectThreads - 32) {
-            const int64_t at = (int64_t)l * prm.W + j;
-            prm.fval[at] = shPlan.f[j];
-            prm.cnt[at] = shPlan.quota[j] - shPlan.room[j];
+            if (!fast) {
+                const int64_t at = (int64_t)l * prm.W + j;
+                prm.fval[at] = shPlan.f[j];
+                prm.cnt[at] = shPlan.quota[j] - shPlan.room[j];
+            }
             if (res) {
                 // everything this needs is in shared memory: stores only, nothing to wait for
                 const int global = shPerm[vstar];
@@ -1562,7 +1614,7 @@ __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, i
             prm.nR[l] = nR - 1;
             if (nR == 1) atomicSub(&prm.nSweep[3], 1);        // one class fewer to finish
         }
-        if (kDelta && deltaAllowed && nR > 1 && shPlan.room[j] > 0) {
+        if (kDelta && deltaAllowed && nR > 1 && roomAfter > 0) {
             // Incremental update: fold row v* into the coverage vector now, find the columns it raised, and if they are
             // few correct the stored gains of block j by one row of S per column; the block then stays up to date.
             for (int i = threadIdx.x; i < ld4; i += kSelectThreads) {
@@ -1610,7 +1662,7 @@ __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, i
             bool few;
             if constexpr (Arith<SV>::kInt) {
                 // integer corrections are exact in any order: the threads that found raised columns append them
-                int at = cnt ? atomicAdd(&shRaised, cnt) : 0;
+                int at = cnt ? atomicAdd(&shRaised[par], cnt) : 0;
 #pragma unroll
                 for (int k = 0; k < 3; ++k) {
                     const int i = (int)threadIdx.x + k * kSelectThreads;
@@ -1624,7 +1676,7 @@ __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, i
                     }
                 }
                 __syncthreads();
-                total = shRaised;
+                total = shRaised[par];
                 few = total <= prm.deltaMax;
             } else {
             // where this thread's columns go in the list: an exclusive prefix sum over the CTA, so that the list (and with it
@@ -1661,6 +1713,7 @@ __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, i
             }
             __syncthreads();
             }
+            if (fast && threadIdx.x == 0) book_fast();
             unsigned changed = 0;                                // bit k: the correction moved one of this thread's gains of piece k
             if (few) {
                 const SV *Sl = prm.S + c.sOff;
@@ -1737,6 +1790,31 @@ __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, i
                     shStat[2] += (unsigned long long)(total + 2) * (unsigned long long)c.ld * sizeof(SV) + 2ull * c.ld * sizeof(GV);
                 }
             }
+            if (notes && j < kCacheBlocks) {
+                if (few) {
+                    // the corrected gains stand in registers: this warp's best unassigned candidate among them
+                    GV ng = 0;
+                    int nv = INT_MAX;
+#pragma unroll
+                    for (int k = 0; k < 3; ++k) {
+                        const int i = (int)threadIdx.x + k * kSelectThreads;
+                        if (i < ld4) {
+#pragma unroll
+                            for (int q = 0; q < 4; ++q) {
+                                const int v = 4 * i + q;
+                                if (v < c.M && (res ? shPos[v] : pos[v]) >= 0 && (nv == INT_MAX || gj[k][q] > ng)) { ng = gj[k][q]; nv = v; }
+                            }
+                        }
+                    }
+                    for (int off = 16; off > 0; off >>= 1) {
+                        GV oG = __shfl_xor_sync(0xffffffffu, ng, off);
+                        int oV = __shfl_xor_sync(0xffffffffu, nv, off);
+                        if (oV != INT_MAX && (nv == INT_MAX || oG > ng || (oG == ng && oV < nv))) { ng = oG; nv = oV; }
+                    }
+                    if (lane == 0) { noteG[j * kWarps + warp] = ng; noteV[j * kWarps + warp] = nv; }
+                }
+                if (threadIdx.x == 0) shNoted[j] = few ? 1 : 0;
+            }
             // (a compiler barrier: without it the correction above and the choice of the next block below are scheduled
             // into one another, and a pick takes 3 us longer -- C2 66 ms instead of 47 ms, measured)
             asm volatile("" ::: "memory");
@@ -1745,7 +1823,15 @@ __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, i
                 plan_decide(prm, l, c, nR - 1, round + 1, shPlan, &shPre);
             }
         } else {
-            if (warp == 0) plan_decide(prm, l, c, nR - 1, round + 1, shPlan, &shPre);
+            if (fast) {
+                __syncthreads();                            // (everybody has read the room of block j)
+                if (threadIdx.x == 0) book_fast();
+            }
+            if (threadIdx.x == 0 && notes && j < kCacheBlocks) shNoted[j] = 0;     // (the block's stored gains are out of date)
+            if (warp == 0) {
+                __syncwarp();
+                plan_decide(prm, l, c, nR - 1, round + 1, shPlan, &shPre);
+            }
             // cover_j <- max(cover_j, S[v*][.])
             if (defer) {
                 for (int i = threadIdx.x; i < ld4; i += kSelectThreads) {
