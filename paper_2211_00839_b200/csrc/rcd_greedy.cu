@@ -1584,12 +1584,10 @@ __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, i
         // everybody else meanwhile starts fetching row v* and the coverage vector.
         const int4 *row = reinterpret_cast<const int4 *>(prm.S + c.sOff + (int64_t)vstar * c.ld);
         int4 *cov = reinterpret_cast<int4 *>(prm.cover + c.vOff + (int64_t)j * c.ld);
-        if (threadIdx.x == kSelectThreads - 32) {
-            if (!fast) {
-                const int64_t at = (int64_t)l * prm.W + j;
-                prm.fval[at] = shPlan.f[j];
-                prm.cnt[at] = shPlan.quota[j] - shPlan.room[j];
-            }
+        // (one thread: the sample leaves the candidate list.  After an argmax its barriers lie between this and every read
+        // of the list; a fast pick has none, and a warp that runs ahead must not change what the others still test their
+        // noted candidate against: there it waits for the pick's next barrier)
+        auto book_sample = [&]() {
             if (res) {
                 // everything this needs is in shared memory: stores only, nothing to wait for
                 const int global = shPerm[vstar];
@@ -1613,6 +1611,12 @@ __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, i
             }
             prm.nR[l] = nR - 1;
             if (nR == 1) atomicSub(&prm.nSweep[3], 1);        // one class fewer to finish
+        };
+        if (threadIdx.x == kSelectThreads - 32 && !fast) {
+            const int64_t at = (int64_t)l * prm.W + j;
+            prm.fval[at] = shPlan.f[j];
+            prm.cnt[at] = shPlan.quota[j] - shPlan.room[j];
+            book_sample();
         }
         if (kDelta && deltaAllowed && nR > 1 && roomAfter > 0) {
             // Incremental update: fold row v* into the coverage vector now, find the columns it raised, and if they are
@@ -1714,6 +1718,7 @@ __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, i
             __syncthreads();
             }
             if (fast && threadIdx.x == 0) book_fast();
+            if (fast && threadIdx.x == kSelectThreads - 32) book_sample();
             unsigned changed = 0;                                // bit k: the correction moved one of this thread's gains of piece k
             if (few) {
                 const SV *Sl = prm.S + c.sOff;
@@ -1802,7 +1807,8 @@ __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, i
 #pragma unroll
                             for (int q = 0; q < 4; ++q) {
                                 const int v = 4 * i + q;
-                                if (v < c.M && (res ? shPos[v] : pos[v]) >= 0 && (nv == INT_MAX || gj[k][q] > ng)) { ng = gj[k][q]; nv = v; }
+                                // (v* may or may not have left the list yet: named explicitly)
+                                if (v < c.M && v != vstar && (res ? shPos[v] : pos[v]) >= 0 && (nv == INT_MAX || gj[k][q] > ng)) { ng = gj[k][q]; nv = v; }
                             }
                         }
                     }
@@ -1826,6 +1832,7 @@ __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, i
             if (fast) {
                 __syncthreads();                            // (everybody has read the room of block j)
                 if (threadIdx.x == 0) book_fast();
+                if (threadIdx.x == kSelectThreads - 32) book_sample();
             }
             if (threadIdx.x == 0 && notes && j < kCacheBlocks) shNoted[j] = 0;     // (the block's stored gains are out of date)
             if (warp == 0) {
