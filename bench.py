@@ -425,6 +425,7 @@ def run_ours(args):
                                 lazy_sweeps=int(prof["lazy_sweeps"]), lazy_misses=int(prof["lazy_misses"]), lazy_rows=int(prof["lazy_rows"]),
                                 lazy_rows_skipped=int(prof["lazy_rows_skipped"]),
                                 incremental_updates=int(prof["incremental_updates"]), incremental_rows=int(prof["incremental_rows"]),
+                                noted_picks=int(prof["noted_picks"]),
                                 threshold_pass_ms=prof["threshold_pass_ns"] * 1e-6, threshold_pass_gb=prof["threshold_pass_bytes"] * 1e-9),
               "similarity": similarity,
               "e2e": {"value": e2e_value, "unit": "samples/s", "h2d_bytes_per_step": int(h2d),

@@ -146,6 +146,7 @@ typedef struct {
     int64_t incremental_rows;       /* rows of S those corrections read (one per column whose coverage rose) */
     int64_t threshold_pass_ns;      /* one CTA per class: time the first CTA spent in threshold passes (part of persistent_sweep_ns) */
     int64_t threshold_pass_bytes;   /* bytes of S and threshold vectors the (row-visiting) threshold passes had to read (part of sweep_bytes) */
+    int64_t noted_picks;            /* picks whose v* was noted when the block's stored gains were last corrected (no argmax over stored gains) */
 } rcd_profile;
 
 typedef struct rcd_ctx rcd_ctx;

@@ -62,7 +62,7 @@ class RcdProfile(C.Structure):
                 ("threshold_elems", C.c_int64), ("threshold_max_blocks", C.c_int64),
                 ("async_lull_ns", C.c_int64), ("async_visits", C.c_int64), ("async_attempts", C.c_int64),
                 ("lazy_sweeps", C.c_int64), ("lazy_misses", C.c_int64), ("lazy_rows", C.c_int64),
-                ("lazy_rows_skipped", C.c_int64), ("incremental_updates", C.c_int64), ("incremental_rows", C.c_int64), ("threshold_pass_ns", C.c_int64), ("threshold_pass_bytes", C.c_int64)]
+                ("lazy_rows_skipped", C.c_int64), ("incremental_updates", C.c_int64), ("incremental_rows", C.c_int64), ("threshold_pass_ns", C.c_int64), ("threshold_pass_bytes", C.c_int64), ("noted_picks", C.c_int64)]
 
 
 def _load() -> C.CDLL:

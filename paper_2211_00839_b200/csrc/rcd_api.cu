@@ -411,6 +411,7 @@ rcd_status rcd_get_profile(rcd_ctx *ctx, rcd_profile *out)
         lazyBytes = (int64_t)ns[12];
         out->incremental_updates = (int64_t)ns[15];
         out->incremental_rows = (int64_t)ns[16];
+        out->noted_picks = (int64_t)ns[17];
         out->threshold_pass_ns = (int64_t)ns[13];
         out->threshold_pass_bytes = (int64_t)ns[14];
         out->persistent_sweep_ns = (int64_t)ns[0];

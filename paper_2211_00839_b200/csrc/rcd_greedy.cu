@@ -1445,8 +1445,8 @@ __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, i
     if (threadIdx.x < kCacheBlocks) shNoted[threadIdx.x] = 0;       // (a pass may have rewritten any block's stored gains)
     if (threadIdx.x == 0) shRaised[0] = shRaised[1] = 0;
     __syncthreads();
-    __shared__ unsigned long long shStat[3];               // corrections of this chain: how many, rows of S, bytes (thread 0 only)
-    if (threadIdx.x == 0) shStat[0] = shStat[1] = shStat[2] = 0ull;
+    __shared__ unsigned long long shStat[4];               // corrections of this chain: how many, rows of S, bytes; picks from a note (thread 0 only)
+    if (threadIdx.x == 0) shStat[0] = shStat[1] = shStat[2] = shStat[3] = 0ull;
     __shared__ PlanGlobals shPre;
     if (threadIdx.x == 0) shPre = plan_globals(prm, l);     // (in flight under the first argmax; read after its barriers)
 
@@ -1567,6 +1567,7 @@ __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, i
         // (fast: thread 0 books the pick in the plan after the next barrier, so the room still counts this sample)
         const int roomAfter = fast ? shPlan.room[j] - 1 : shPlan.room[j];
         auto book_fast = [&]() {                             // thread 0, fast picks: what warp 0 does after an argmax
+            shStat[3] += 1ull;
             shPlan.f[j] += (FV)bestG;
             shPlan.room[j] = roomAfter;
             shPlan.open[j] = (uint8_t)((roomAfter > 0 ? 1 : 0) | 2);
@@ -1858,6 +1859,7 @@ __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, i
         if (nR == 0 || j < 0 || shPlan.needSweep) break;
     }
     if (threadIdx.x == 0 && shStat[0]) {
+        if (shStat[3]) atomicAdd(&prm.phaseNs[17], shStat[3]);
         atomicAdd(&prm.phaseNs[15], shStat[0]);
         atomicAdd(&prm.phaseNs[16], shStat[1]);
         atomicAdd(&prm.phaseNs[12], shStat[2]);
