@@ -352,6 +352,7 @@ def test_incremental_update_int8_exact(rcd, orc, path):
     ref = orc.partition(wl.features, wl.labels, wl.capacities, wl.L, variant="incremental")
     a, o, v, prof = run_with_profile(rcd, wl, greedy_path=path, incremental=1)
     assert prof["incremental_updates"] > 1000 and prof["incremental_rows"] >= prof["incremental_updates"] // 2
+    assert prof["noted_picks"] > prof["incremental_updates"] // 2      # most picks take v* from the note of the last correction
     assert np.array_equal(a, ref.assignment) and np.array_equal(o, ref.order) and np.array_equal(v, ref.part_values)
     a0, o0, v0, prof0 = run_with_profile(rcd, wl, greedy_path=path, incremental=2)
     assert prof0["incremental_updates"] == 0
@@ -394,6 +395,31 @@ def test_incremental_update_float(rcd, orc, path):
     r2 = run_partition(rcd, wl, greedy_path=path, incremental=1)
     for x, y in zip(r1, r2):
         assert np.array_equal(x, y)                      # the corrections are applied in a fixed order
+
+
+@pytest.mark.parametrize("path", [3, 4])
+def test_noted_candidates_ties_and_many_classes(rcd, orc, path):
+    """Picks that take v* from the note made at the block's last correction (eight blocks per class): duplicate samples
+    make equal gains (the lowest index must win, also when the noted sample of one block is taken by another block first),
+    ragged classes, more classes than SMs in the one-CTA-per-class form; twice, with identical results."""
+    from paper_2211_00839_b200.workloads import Workload, make_workload
+    L = 12 if path == 3 else 200
+    base = make_workload("C2", L=L, M=260, d=64, seed=77)
+    rng = np.random.default_rng(31)
+    keep = np.ones(base.N, bool)
+    for l in range(base.L):
+        ids = np.nonzero(base.labels == l)[0]
+        keep[ids[:int(rng.integers(0, 120))]] = False
+    feats = base.features[keep].copy()
+    feats[::5] = feats[2]                                # a fifth of all samples are copies of one: ties everywhere
+    feats[1::11] = feats[4]
+    wl = Workload("noted", "int8", np.ascontiguousarray(feats), np.ascontiguousarray(base.labels[keep]), base.capacities, base.L, base.W)
+    ref = orc.partition(wl.features, wl.labels, wl.capacities, wl.L, variant="incremental")
+    a, o, v, prof = run_with_profile(rcd, wl, greedy_path=path, incremental=1)
+    assert prof["noted_picks"] > 0
+    assert np.array_equal(a, ref.assignment) and np.array_equal(o, ref.order) and np.array_equal(v, ref.part_values)
+    a2, o2, v2, prof2 = run_with_profile(rcd, wl, greedy_path=path, incremental=1)
+    assert np.array_equal(a2, a) and np.array_equal(o2, o) and np.array_equal(v2, v) and prof2["noted_picks"] == prof["noted_picks"]
 
 
 # ----------------------------------------------------------------------------- exact lazy evaluation (row-skipping passes)
