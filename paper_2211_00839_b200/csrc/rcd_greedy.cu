@@ -2015,6 +2015,14 @@ __device__ __forceinline__ int4 ld_volatile16(const void *p)
     return v;
 }
 __device__ __forceinline__ int32_t ld_volatile32(const int32_t *p) { return *(const volatile int32_t *)p; }
+// The second read of a class's epoch (the first one and everything read in between count only if it returns the same
+// even value): an acquire load at GPU scope.
+__device__ __forceinline__ int32_t ld_acquire32(const int32_t *p)
+{
+    int32_t v;
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
 
 
 template <typename SV>
@@ -2039,6 +2047,9 @@ __device__ __forceinline__ void async_pick_cta(const GreedyParams<SV> &prm, int4
                     e = sy.x;
                     *(volatile int32_t *)&prm.sync[l].epoch = e + 1;    // the class is mine until I publish again
                     if (!owner) __threadfence();                        // (an owner's chain fences after its first loads)
+                } else if (!(sy.x & 1) && sy.z > sy.y) {
+                    // more row groups reported done than the sweep has: a sweep CTA acted on a torn or stale word
+                    atomicOr(prm.status, kDevBadState);
                 }
                 shEpoch = e;
             }
@@ -2187,7 +2198,7 @@ __device__ __forceinline__ void async_sweep_cta(const GreedyParams<SV> &prm, int
             const int e1 = shInfo[9];
             const int teams = (kSweepThreads / 32) / (mode ? 1 : CS);
             const int first = atomicAdd(prm.tickets + c.row0 + l + (e1 >> 1), teams);
-            const int e2 = ld_volatile32(&prm.sync[l].epoch);
+            const int e2 = ld_acquire32(&prm.sync[l].epoch);
             shInfo[0] = (e1 == e2 && !(e1 & 1) && first < shInfo[6]) ? 1 : 0;
             if (clocked) shClk[2] += 1ull << 32;                   // attempts (high half), visits (low half)
             shInfo[1] = first;
