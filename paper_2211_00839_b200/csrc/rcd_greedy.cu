@@ -251,6 +251,27 @@ __device__ void plan_decide(const GreedyParams<SV> &prm, int l, const ClassDesc 
         return;
     }
 
+    if constexpr (Arith<SV>::kInt) {
+        if (W <= 32) {
+            // At most one block per lane and nothing out of date (the usual case once stored gains are corrected in place):
+            // the next block is the argmin of f over the non-full blocks, lowest index on ties, and no pass is due.
+            const uint8_t o = lane < W ? sh.open[lane] : (uint8_t)0;
+            const bool cand = (o & 1) != 0;
+            const unsigned candMask = __ballot_sync(0xffffffffu, cand);
+            const unsigned staleMask = __ballot_sync(0xffffffffu, cand && (o & 2));
+            if (candMask != 0 && staleMask == 0) {
+                const long long fl = cand ? (long long)sh.f[lane] : 0;
+                const int hi = cand ? (int)(fl >> 32) : INT_MAX;
+                const unsigned lo = (unsigned)fl;
+                const int mhi = __reduce_min_sync(0xffffffffu, hi);
+                const unsigned mlo = __reduce_min_sync(0xffffffffu, (cand && hi == mhi) ? lo : 0xffffffffu);
+                const unsigned eq = __ballot_sync(0xffffffffu, cand && hi == mhi && lo == mlo);
+                const int jnext = __ffs(eq) - 1;
+                if (lane == 0) { prm.jstar[l] = jnext; prm.sweepN[l] = 0; sh.nextJ = jnext; sh.needSweep = 0; }
+                return;
+            }
+        }
+    }
     // j* = argmin over non-full blocks of f, ties -> lowest index
     FV bestF = 0;
     int bestP = INT_MAX;
@@ -1359,6 +1380,19 @@ __device__ __forceinline__ bool rose(int r, int o)
     else return __int_as_float(r) > __int_as_float(o);
 }
 
+// Maximum of a 64-bit key over the warp (two 32-bit warp reductions: high words, then low words among the lanes that
+// hold the greatest high word).
+__device__ __forceinline__ unsigned long long warp_max_u64(unsigned long long k)
+{
+    const unsigned hi = (unsigned)(k >> 32), lo = (unsigned)k;
+    const unsigned mhi = __reduce_max_sync(0xffffffffu, hi);
+    const unsigned mlo = __reduce_max_sync(0xffffffffu, hi == mhi ? lo : 0u);
+    return ((unsigned long long)mhi << 32) | mlo;
+}
+// Integer notes are one key: gain << 13 | (8191 - index).  A greater key is a greater gain, or the same gain at a lower
+// index; 0 means none.  (Notes exist for classes of at most 6144 samples, whose gains stay far below 2^50.)
+__device__ __forceinline__ unsigned long long note_key(long long gain, int v) { return ((unsigned long long)gain << 13) | (unsigned long long)(8191 - v); }
+
 // kDelta: compiled with the incremental update of stored gains.
 template <typename SV, bool kDelta = false>
 __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, int round, int4 *scratch, int scratchBytes,
@@ -1461,12 +1495,17 @@ __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, i
         bool fast = false;                                  // v* comes from the notes: no argmax
         if constexpr (kDelta) {
             if (notes && j < kCacheBlocks && shNoted[j]) {
-                bestG = lane < kWarps ? noteG[j * kWarps + lane] : (GV)0;
-                bestV = lane < kWarps ? noteV[j * kWarps + lane] : INT_MAX;
-                for (int off = 16; off > 0; off >>= 1) {
-                    GV oG = __shfl_xor_sync(0xffffffffu, bestG, off);
-                    int oV = __shfl_xor_sync(0xffffffffu, bestV, off);
-                    if (oV != INT_MAX && (bestV == INT_MAX || oG > bestG || (oG == bestG && oV < bestV))) { bestG = oG; bestV = oV; }
+                if constexpr (Arith<SV>::kInt) {
+                    const unsigned long long key = warp_max_u64(lane < kWarps ? (unsigned long long)noteG[j * kWarps + lane] : 0ull);
+                    if (key) { bestG = (GV)(key >> 13); bestV = 8191 - (int)(key & 8191ull); }
+                } else {
+                    bestG = lane < kWarps ? noteG[j * kWarps + lane] : (GV)0;
+                    bestV = lane < kWarps ? noteV[j * kWarps + lane] : INT_MAX;
+                    for (int off = 16; off > 0; off >>= 1) {
+                        GV oG = __shfl_xor_sync(0xffffffffu, bestG, off);
+                        int oV = __shfl_xor_sync(0xffffffffu, bestV, off);
+                        if (oV != INT_MAX && (bestV == INT_MAX || oG > bestG || (oG == bestG && oV < bestV))) { bestG = oG; bestV = oV; }
+                    }
                 }
                 fast = bestV != INT_MAX && (res ? shPos[bestV] : pos[bestV]) >= 0;
                 if (!fast) { bestG = 0; bestV = INT_MAX; }
@@ -1799,6 +1838,25 @@ __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, i
             if (notes && j < kCacheBlocks) {
                 if (few) {
                     // the corrected gains stand in registers: this warp's best unassigned candidate among them
+                    if constexpr (Arith<SV>::kInt) {
+                        unsigned long long nk = 0ull;
+#pragma unroll
+                        for (int k = 0; k < 3; ++k) {
+                            const int i = (int)threadIdx.x + k * kSelectThreads;
+                            if (i < ld4) {
+#pragma unroll
+                                for (int q = 0; q < 4; ++q) {
+                                    const int v = 4 * i + q;
+                                    if (v < c.M && v != vstar && (res ? shPos[v] : pos[v]) >= 0) {
+                                        const unsigned long long kk = note_key(gj[k][q], v);
+                                        if (kk > nk) nk = kk;
+                                    }
+                                }
+                            }
+                        }
+                        nk = warp_max_u64(nk);
+                        if (lane == 0) noteG[j * kWarps + warp] = (GV)nk;
+                    } else {
                     GV ng = 0;
                     int nv = INT_MAX;
 #pragma unroll
@@ -1819,6 +1877,7 @@ __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, i
                         if (oV != INT_MAX && (nv == INT_MAX || oG > ng || (oG == ng && oV < nv))) { ng = oG; nv = oV; }
                     }
                     if (lane == 0) { noteG[j * kWarps + warp] = ng; noteV[j * kWarps + warp] = nv; }
+                    }
                 }
                 if (threadIdx.x == 0) shNoted[j] = few ? 1 : 0;
             }
