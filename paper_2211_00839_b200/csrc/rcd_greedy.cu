@@ -237,6 +237,20 @@ __device__ __forceinline__ int classes_alongside(const GreedyParams<SV> &prm, in
     return n;
 }
 
+// Order-preserving images in unsigned integers (a < b exactly when image(a) < image(b); -0.0 is taken as +0.0).
+__device__ __forceinline__ unsigned long long ordered_u64(long long x) { return (unsigned long long)x ^ 0x8000000000000000ull; }
+__device__ __forceinline__ unsigned long long ordered_u64(double x)
+{
+    const unsigned long long b = (unsigned long long)__double_as_longlong(x + 0.0);
+    return b ^ ((b >> 63) ? ~0ull : 0x8000000000000000ull);
+}
+__device__ __forceinline__ unsigned ordered_u32(float x)
+{
+    const unsigned b = __float_as_uint(x + 0.0f);
+    return b ^ ((b >> 31) ? 0xffffffffu : 0x80000000u);
+}
+__device__ __forceinline__ float from_ordered_u32(unsigned o) { return __uint_as_float(o ^ ((o >> 31) ? 0x80000000u : 0xffffffffu)); }
+
 template <typename SV>
 __device__ void plan_decide(const GreedyParams<SV> &prm, int l, const ClassDesc &c, int nR, int nextStep,
                             PlanShared<typename Arith<SV>::FV> &sh, const PlanGlobals *pre = nullptr)
@@ -251,7 +265,7 @@ __device__ void plan_decide(const GreedyParams<SV> &prm, int l, const ClassDesc 
         return;
     }
 
-    if constexpr (Arith<SV>::kInt) {
+    {
         if (W <= 32) {
             // At most one block per lane and nothing out of date (the usual case once stored gains are corrected in place):
             // the next block is the argmin of f over the non-full blocks, lowest index on ties, and no pass is due.
@@ -260,10 +274,10 @@ __device__ void plan_decide(const GreedyParams<SV> &prm, int l, const ClassDesc 
             const unsigned candMask = __ballot_sync(0xffffffffu, cand);
             const unsigned staleMask = __ballot_sync(0xffffffffu, cand && (o & 2));
             if (candMask != 0 && staleMask == 0) {
-                const long long fl = cand ? (long long)sh.f[lane] : 0;
-                const int hi = cand ? (int)(fl >> 32) : INT_MAX;
-                const unsigned lo = (unsigned)fl;
-                const int mhi = __reduce_min_sync(0xffffffffu, hi);
+                const unsigned long long fo = cand ? ordered_u64(sh.f[lane]) : ~0ull;     // (same order as f itself)
+                const unsigned hi = (unsigned)(fo >> 32);
+                const unsigned lo = (unsigned)fo;
+                const unsigned mhi = __reduce_min_sync(0xffffffffu, hi);
                 const unsigned mlo = __reduce_min_sync(0xffffffffu, (cand && hi == mhi) ? lo : 0xffffffffu);
                 const unsigned eq = __ballot_sync(0xffffffffu, cand && hi == mhi && lo == mlo);
                 const int jnext = __ffs(eq) - 1;
@@ -1389,9 +1403,14 @@ __device__ __forceinline__ unsigned long long warp_max_u64(unsigned long long k)
     const unsigned mlo = __reduce_max_sync(0xffffffffu, hi == mhi ? lo : 0u);
     return ((unsigned long long)mhi << 32) | mlo;
 }
-// Integer notes are one key: gain << 13 | (8191 - index).  A greater key is a greater gain, or the same gain at a lower
-// index; 0 means none.  (Notes exist for classes of at most 6144 samples, whose gains stay far below 2^50.)
+// A (gain, index) pair as one key, for classes of at most 8192 samples: a greater key is a greater gain, or the same gain
+// at a lower index; 0 means none.  Integer gains (never negative, far below 2^50 for such classes): gain << 13 |
+// (8191 - index).  fp32 gains: order-preserving image of the gain << 32 | (8191 - index).
 __device__ __forceinline__ unsigned long long note_key(long long gain, int v) { return ((unsigned long long)gain << 13) | (unsigned long long)(8191 - v); }
+__device__ __forceinline__ unsigned long long note_key(float gain, int v) { return ((unsigned long long)ordered_u32(gain) << 32) | (unsigned long long)(8191 - v); }
+__device__ __forceinline__ int key_index(unsigned long long key) { return 8191 - (int)(key & 8191ull); }
+__device__ __forceinline__ void key_gain(unsigned long long key, long long &g) { g = (long long)(key >> 13); }
+__device__ __forceinline__ void key_gain(unsigned long long key, float &g) { g = from_ordered_u32((unsigned)(key >> 32)); }
 
 // kDelta: compiled with the incremental update of stored gains.
 template <typename SV, bool kDelta = false>
@@ -1403,6 +1422,7 @@ __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, i
     __shared__ PlanShared<FV> shPlan;
     __shared__ GV shG[kSelectThreads / 32];
     __shared__ int shV[kSelectThreads / 32];
+    __shared__ unsigned long long shKey[kSelectThreads / 32];
     __shared__ int shPick;
     const ClassDesc c = prm.desc[l];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -1471,11 +1491,10 @@ __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, i
     constexpr int kCacheBlocks = 8;
     constexpr int kWarps = kSelectThreads / 32;
     __shared__ uint8_t shNoted[kCacheBlocks];
-    GV *noteG = reinterpret_cast<GV *>(scratch + 6 * ld4 + kDeltaMax);             // [kCacheBlocks][kWarps]
-    int *noteV = reinterpret_cast<int *>(noteG + kCacheBlocks * kWarps);
-    const bool notes = kDelta && deltaAllowed && prm.lazyFrom < 0 &&
+    unsigned long long *noteK = reinterpret_cast<unsigned long long *>(scratch + 6 * ld4 + kDeltaMax);   // [kCacheBlocks][kWarps] keys
+    const bool notes = kDelta && deltaAllowed && prm.lazyFrom < 0 && c.M <= 8192 &&
                        (int64_t)6 * c.ld * (int64_t)sizeof(SV) + (int64_t)kDeltaMax * 16 +
-                       (int64_t)kCacheBlocks * kWarps * (int64_t)(sizeof(GV) + sizeof(int)) <= scratchBytes;
+                       (int64_t)kCacheBlocks * kWarps * (int64_t)sizeof(unsigned long long) <= scratchBytes;
     if (threadIdx.x < kCacheBlocks) shNoted[threadIdx.x] = 0;       // (a pass may have rewritten any block's stored gains)
     if (threadIdx.x == 0) shRaised[0] = shRaised[1] = 0;
     __syncthreads();
@@ -1495,18 +1514,8 @@ __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, i
         bool fast = false;                                  // v* comes from the notes: no argmax
         if constexpr (kDelta) {
             if (notes && j < kCacheBlocks && shNoted[j]) {
-                if constexpr (Arith<SV>::kInt) {
-                    const unsigned long long key = warp_max_u64(lane < kWarps ? (unsigned long long)noteG[j * kWarps + lane] : 0ull);
-                    if (key) { bestG = (GV)(key >> 13); bestV = 8191 - (int)(key & 8191ull); }
-                } else {
-                    bestG = lane < kWarps ? noteG[j * kWarps + lane] : (GV)0;
-                    bestV = lane < kWarps ? noteV[j * kWarps + lane] : INT_MAX;
-                    for (int off = 16; off > 0; off >>= 1) {
-                        GV oG = __shfl_xor_sync(0xffffffffu, bestG, off);
-                        int oV = __shfl_xor_sync(0xffffffffu, bestV, off);
-                        if (oV != INT_MAX && (bestV == INT_MAX || oG > bestG || (oG == bestG && oV < bestV))) { bestG = oG; bestV = oV; }
-                    }
-                }
+                const unsigned long long key = warp_max_u64(lane < kWarps ? noteK[j * kWarps + lane] : 0ull);
+                if (key) { key_gain(key, bestG); bestV = key_index(key); }
                 fast = bestV != INT_MAX && (res ? shPos[bestV] : pos[bestV]) >= 0;
                 if (!fast) { bestG = 0; bestV = INT_MAX; }
             }
@@ -1548,25 +1557,41 @@ __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, i
             fold_pending<SV>(pendDst, scratch, ld4, thrAcc);
             pendDst = nullptr;
         }
-        for (int off = 16; off > 0; off >>= 1) {
-            GV oG = __shfl_xor_sync(0xffffffffu, bestG, off);
-            int oV = __shfl_xor_sync(0xffffffffu, bestV, off);
-            if (oV != INT_MAX && (bestV == INT_MAX || oG > bestG || (oG == bestG && oV < bestV))) { bestG = oG; bestV = oV; }
-        }
-        if (lane == 0) { shG[warp] = bestG; shV[warp] = bestV; }
-        __syncthreads();
-        if (warp == 0) {
-            bestG = lane < kSelectThreads / 32 ? shG[lane] : (GV)0;
-            bestV = lane < kSelectThreads / 32 ? shV[lane] : INT_MAX;
-            // The least of the warps' best stored gains: at least one unassigned sample per warp lies at or above it,
-            // so a later row-skipping pass with this floor recomputes the few dozen best-placed candidates of the block.
-            FV low = bestV != INT_MAX ? (FV)bestG : highest_value<FV>();
+        // (gain, index) as one key where the class is small enough and no floors are kept (row-skipping passes off): the
+        // two reductions are then two warp-wide maxima each instead of shuffle ladders over pairs
+        const bool packed = c.M <= 8192 && prm.lazyFrom < 0;
+        if (packed) {
+            const unsigned long long key = warp_max_u64(bestV != INT_MAX ? note_key(bestG, bestV) : 0ull);
+            if (lane == 0) shKey[warp] = key;
+        } else {
             for (int off = 16; off > 0; off >>= 1) {
                 GV oG = __shfl_xor_sync(0xffffffffu, bestG, off);
                 int oV = __shfl_xor_sync(0xffffffffu, bestV, off);
-                const FV oLow = __shfl_xor_sync(0xffffffffu, low, off);
-                if (oLow < low) low = oLow;
                 if (oV != INT_MAX && (bestV == INT_MAX || oG > bestG || (oG == bestG && oV < bestV))) { bestG = oG; bestV = oV; }
+            }
+            if (lane == 0) { shG[warp] = bestG; shV[warp] = bestV; }
+        }
+        __syncthreads();
+        if (warp == 0) {
+            // The least of the warps' best stored gains: at least one unassigned sample per warp lies at or above it,
+            // so a later row-skipping pass with this floor recomputes the few dozen best-placed candidates of the block.
+            FV low = lowest_value<FV>();
+            if (packed) {
+                const unsigned long long key = warp_max_u64(lane < kSelectThreads / 32 ? shKey[lane] : 0ull);
+                bestG = 0;
+                bestV = INT_MAX;
+                if (key) { key_gain(key, bestG); bestV = key_index(key); }
+            } else {
+                bestG = lane < kSelectThreads / 32 ? shG[lane] : (GV)0;
+                bestV = lane < kSelectThreads / 32 ? shV[lane] : INT_MAX;
+                low = bestV != INT_MAX ? (FV)bestG : highest_value<FV>();
+                for (int off = 16; off > 0; off >>= 1) {
+                    GV oG = __shfl_xor_sync(0xffffffffu, bestG, off);
+                    int oV = __shfl_xor_sync(0xffffffffu, bestV, off);
+                    const FV oLow = __shfl_xor_sync(0xffffffffu, low, off);
+                    if (oLow < low) low = oLow;
+                    if (oV != INT_MAX && (bestV == INT_MAX || oG > bestG || (oG == bestG && oV < bestV))) { bestG = oG; bestV = oV; }
+                }
             }
             if (lane == 0) {
                 shPick = bestV;
@@ -1838,27 +1863,7 @@ __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, i
             if (notes && j < kCacheBlocks) {
                 if (few) {
                     // the corrected gains stand in registers: this warp's best unassigned candidate among them
-                    if constexpr (Arith<SV>::kInt) {
-                        unsigned long long nk = 0ull;
-#pragma unroll
-                        for (int k = 0; k < 3; ++k) {
-                            const int i = (int)threadIdx.x + k * kSelectThreads;
-                            if (i < ld4) {
-#pragma unroll
-                                for (int q = 0; q < 4; ++q) {
-                                    const int v = 4 * i + q;
-                                    if (v < c.M && v != vstar && (res ? shPos[v] : pos[v]) >= 0) {
-                                        const unsigned long long kk = note_key(gj[k][q], v);
-                                        if (kk > nk) nk = kk;
-                                    }
-                                }
-                            }
-                        }
-                        nk = warp_max_u64(nk);
-                        if (lane == 0) noteG[j * kWarps + warp] = (GV)nk;
-                    } else {
-                    GV ng = 0;
-                    int nv = INT_MAX;
+                    unsigned long long nk = 0ull;
 #pragma unroll
                     for (int k = 0; k < 3; ++k) {
                         const int i = (int)threadIdx.x + k * kSelectThreads;
@@ -1867,17 +1872,15 @@ __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, i
                             for (int q = 0; q < 4; ++q) {
                                 const int v = 4 * i + q;
                                 // (v* may or may not have left the list yet: named explicitly)
-                                if (v < c.M && v != vstar && (res ? shPos[v] : pos[v]) >= 0 && (nv == INT_MAX || gj[k][q] > ng)) { ng = gj[k][q]; nv = v; }
+                                if (v < c.M && v != vstar && (res ? shPos[v] : pos[v]) >= 0) {
+                                    const unsigned long long kk = note_key(gj[k][q], v);
+                                    if (kk > nk) nk = kk;
+                                }
                             }
                         }
                     }
-                    for (int off = 16; off > 0; off >>= 1) {
-                        GV oG = __shfl_xor_sync(0xffffffffu, ng, off);
-                        int oV = __shfl_xor_sync(0xffffffffu, nv, off);
-                        if (oV != INT_MAX && (nv == INT_MAX || oG > ng || (oG == ng && oV < nv))) { ng = oG; nv = oV; }
-                    }
-                    if (lane == 0) { noteG[j * kWarps + warp] = ng; noteV[j * kWarps + warp] = nv; }
-                    }
+                    nk = warp_max_u64(nk);
+                    if (lane == 0) noteK[j * kWarps + warp] = nk;
                 }
                 if (threadIdx.x == 0) shNoted[j] = few ? 1 : 0;
             }
