@@ -43,7 +43,7 @@ __global__ void __launch_bounds__(kCutThreads, 2) cut_chain_kernel(CutParams<SV>
     using FV = typename CutArith<SV>::FV;
     __shared__ FV shF[kCutMaxBlocks];
     __shared__ int32_t shRoom[kCutMaxBlocks];
-    __shared__ FV shG[kCutThreads / 32];
+    __shared__ unsigned long long shG[kCutThreads / 32];      // order-preserving images of the warps' best gains
     __shared__ int shV[kCutThreads / 32];
     __shared__ int shPick, shBlock;
     const int l = blockIdx.x;
@@ -79,11 +79,9 @@ __global__ void __launch_bounds__(kCutThreads, 2) cut_chain_kernel(CutParams<SV>
             int bestP = INT_MAX;
             for (int p = lane; p < W; p += 32)
                 if (shRoom[p] > 0 && (bestP == INT_MAX || shF[p] < bestF)) { bestF = shF[p]; bestP = p; }
-            for (int off = 16; off > 0; off >>= 1) {
-                FV oF = __shfl_xor_sync(0xffffffffu, bestF, off);
-                int oP = __shfl_xor_sync(0xffffffffu, bestP, off);
-                if (oP != INT_MAX && (bestP == INT_MAX || oF < bestF || (oF == bestF && oP < bestP))) { bestF = oF; bestP = oP; }
-            }
+            // (three warp-wide reductions on an order-preserving image of f: least f, lowest index among equals)
+            unsigned long long of = ordered_u64(bestF);
+            warp_argmin_ordered(of, bestP);
             if (lane == 0) shBlock = bestP;
         }
         __syncthreads();
@@ -101,21 +99,17 @@ __global__ void __launch_bounds__(kCutThreads, 2) cut_chain_kernel(CutParams<SV>
             const FV g = base[u] - 2 * tj[u];
             if (pos[u] >= 0 && (bestV == INT_MAX || g > bestG)) { bestG = g; bestV = u; }
         }
-        for (int off = 16; off > 0; off >>= 1) {
-            FV oG = __shfl_xor_sync(0xffffffffu, bestG, off);
-            int oV = __shfl_xor_sync(0xffffffffu, bestV, off);
-            if (oV != INT_MAX && (bestV == INT_MAX || oG > bestG || (oG == bestG && oV < bestV))) { bestG = oG; bestV = oV; }
-        }
-        if (lane == 0) { shG[warp] = bestG; shV[warp] = bestV; }
+        // greatest gain, lowest index among equals: over the warp, then over the warps' results
+        unsigned long long og = ordered_u64(bestG);
+        warp_argmax_ordered(og, bestV);
+        if (lane == 0) { shG[warp] = og; shV[warp] = bestV; }
         __syncthreads();
         if (warp == 0) {
-            bestG = lane < kCutThreads / 32 ? shG[lane] : (FV)0;
+            og = lane < kCutThreads / 32 ? shG[lane] : 0ull;
             bestV = lane < kCutThreads / 32 ? shV[lane] : INT_MAX;
-            for (int off = 16; off > 0; off >>= 1) {
-                FV oG = __shfl_xor_sync(0xffffffffu, bestG, off);
-                int oV = __shfl_xor_sync(0xffffffffu, bestV, off);
-                if (oV != INT_MAX && (bestV == INT_MAX || oG > bestG || (oG == bestG && oV < bestV))) { bestG = oG; bestV = oV; }
-            }
+            warp_argmax_ordered(og, bestV);
+            if constexpr (std::is_same<FV, double>::value) bestG = from_ordered_u64_d(og);
+            else bestG = from_ordered_u64_ll(og);
             if (lane == 0) {
                 shPick = bestV;
                 if (bestV != INT_MAX) {

@@ -237,20 +237,6 @@ __device__ __forceinline__ int classes_alongside(const GreedyParams<SV> &prm, in
     return n;
 }
 
-// Order-preserving images in unsigned integers (a < b exactly when image(a) < image(b); -0.0 is taken as +0.0).
-__device__ __forceinline__ unsigned long long ordered_u64(long long x) { return (unsigned long long)x ^ 0x8000000000000000ull; }
-__device__ __forceinline__ unsigned long long ordered_u64(double x)
-{
-    const unsigned long long b = (unsigned long long)__double_as_longlong(x + 0.0);
-    return b ^ ((b >> 63) ? ~0ull : 0x8000000000000000ull);
-}
-__device__ __forceinline__ unsigned ordered_u32(float x)
-{
-    const unsigned b = __float_as_uint(x + 0.0f);
-    return b ^ ((b >> 31) ? 0xffffffffu : 0x80000000u);
-}
-__device__ __forceinline__ float from_ordered_u32(unsigned o) { return __uint_as_float(o ^ ((o >> 31) ? 0x80000000u : 0xffffffffu)); }
-
 template <typename SV>
 __device__ void plan_decide(const GreedyParams<SV> &prm, int l, const ClassDesc &c, int nR, int nextStep,
                             PlanShared<typename Arith<SV>::FV> &sh, const PlanGlobals *pre = nullptr)
@@ -1394,15 +1380,6 @@ __device__ __forceinline__ bool rose(int r, int o)
     else return __int_as_float(r) > __int_as_float(o);
 }
 
-// Maximum of a 64-bit key over the warp (two 32-bit warp reductions: high words, then low words among the lanes that
-// hold the greatest high word).
-__device__ __forceinline__ unsigned long long warp_max_u64(unsigned long long k)
-{
-    const unsigned hi = (unsigned)(k >> 32), lo = (unsigned)k;
-    const unsigned mhi = __reduce_max_sync(0xffffffffu, hi);
-    const unsigned mlo = __reduce_max_sync(0xffffffffu, hi == mhi ? lo : 0u);
-    return ((unsigned long long)mhi << 32) | mlo;
-}
 // A (gain, index) pair as one key, for classes of at most 8192 samples: a greater key is a greater gain, or the same gain
 // at a lower index; 0 means none.  Integer gains (never negative, far below 2^50 for such classes): gain << 13 |
 // (8191 - index).  fp32 gains: order-preserving image of the gain << 32 | (8191 - index).

@@ -239,4 +239,56 @@ rcd_status launch_objective(rcd_ctx *ctx, rcd_feat_dtype dtype, const Sizes &sz,
                             const int32_t *assignment, void *partValues, void *total, void *scratch,
                             cudaStream_t st);
 
+
+#ifdef __CUDACC__
+// ---- warp-wide reductions of (value, index) pairs by 32-bit redux instead of shuffle ladders ----
+// Order-preserving images in unsigned integers (a < b exactly when image(a) < image(b); -0.0 is taken as +0.0).
+__device__ __forceinline__ unsigned long long ordered_u64(long long x) { return (unsigned long long)x ^ 0x8000000000000000ull; }
+__device__ __forceinline__ unsigned long long ordered_u64(double x)
+{
+    const unsigned long long b = (unsigned long long)__double_as_longlong(x + 0.0);
+    return b ^ ((b >> 63) ? ~0ull : 0x8000000000000000ull);
+}
+__device__ __forceinline__ unsigned ordered_u32(float x)
+{
+    const unsigned b = __float_as_uint(x + 0.0f);
+    return b ^ ((b >> 31) ? 0xffffffffu : 0x80000000u);
+}
+__device__ __forceinline__ float from_ordered_u32(unsigned o) { return __uint_as_float(o ^ ((o >> 31) ? 0x80000000u : 0xffffffffu)); }
+
+// Maximum of a 64-bit key over the warp (two 32-bit warp reductions: high words, then low words among the lanes that
+// hold the greatest high word).
+__device__ __forceinline__ unsigned long long warp_max_u64(unsigned long long k)
+{
+    const unsigned hi = (unsigned)(k >> 32), lo = (unsigned)k;
+    const unsigned mhi = __reduce_max_sync(0xffffffffu, hi);
+    const unsigned mlo = __reduce_max_sync(0xffffffffu, hi == mhi ? lo : 0u);
+    return ((unsigned long long)mhi << 32) | mlo;
+}
+// Arg-maximum of (ordered image of the value, index) pairs over the warp: the greatest value, and among the lanes that
+// hold it the lowest index; lanes without a candidate pass index INT_MAX.  Three warp-wide reductions.
+__device__ __forceinline__ void warp_argmax_ordered(unsigned long long &ord, int &idx)
+{
+    const bool has = idx != 0x7fffffff;
+    const unsigned hi = has ? (unsigned)(ord >> 32) : 0u, lo = has ? (unsigned)ord : 0u;
+    const unsigned mhi = __reduce_max_sync(0xffffffffu, hi);
+    const unsigned mlo = __reduce_max_sync(0xffffffffu, (has && hi == mhi) ? lo : 0u);
+    const int mi = __reduce_min_sync(0xffffffffu, (has && hi == mhi && lo == mlo) ? idx : 0x7fffffff);
+    ord = ((unsigned long long)mhi << 32) | mlo;
+    idx = mi;
+}
+// The same for the least value (lowest index among equals).
+__device__ __forceinline__ void warp_argmin_ordered(unsigned long long &ord, int &idx)
+{
+    unsigned long long inv = ~ord;
+    warp_argmax_ordered(inv, idx);
+    ord = ~inv;
+}
+__device__ __forceinline__ long long from_ordered_u64_ll(unsigned long long o) { return (long long)(o ^ 0x8000000000000000ull); }
+__device__ __forceinline__ double from_ordered_u64_d(unsigned long long o)
+{
+    return __longlong_as_double((long long)(o ^ ((o >> 63) ? 0x8000000000000000ull : ~0ull)));
+}
+#endif
+
 }  // namespace rcd
