@@ -108,7 +108,7 @@ typedef struct {
     int32_t incremental;       /* in-place correction of stored gains (greedy paths 3 and 4).  When a pick raised its block's coverage
                                   in few columns i, every candidate's gain falls by max(0, S[v][i] - old_i) - max(0, S[v][i] - new_i),
                                   read from row i of S (S is symmetric): the block's stored gains stay exact and it needs no
-                                  pass over S.  0 = choose (on for path 3 with at most 8 blocks and for path 4 with classes of 1024 samples or
+                                  pass over S.  0 = choose (on for path 3 with at most 16 blocks and for path 4 with classes of 1024 samples or
                                   more: where it was measured faster), 1 = on,
                                   2 = off (every block that received a sample waits for a pass).  Same picks either way. */
     int32_t incremental_max;   /* most columns a pick may raise and still be corrected in place; 0 = default (32 for greedy

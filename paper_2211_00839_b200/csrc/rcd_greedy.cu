@@ -1465,7 +1465,7 @@ __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, i
     // the argmax, unless it has been assigned meanwhile (the stored gains of p do not change in between): then no stored
     // gain is loaded and the pick needs neither of the argmax's two barriers.  Blocks 0..kCacheBlocks-1; the notes sit
     // behind the list of raised columns.
-    constexpr int kCacheBlocks = 8;
+    constexpr int kCacheBlocks = 16;
     constexpr int kWarps = kSelectThreads / 32;
     __shared__ uint8_t shNoted[kCacheBlocks];
     unsigned long long *noteK = reinterpret_cast<unsigned long long *>(scratch + 6 * ld4 + kDeltaMax);   // [kCacheBlocks][kWarps] keys
@@ -2512,8 +2512,9 @@ static rcd_status run_greedy(rcd_ctx *ctx, const Sizes &sz, const Workspace &ws,
         if (ctx->cfg.incremental_max <= 0) prm.deltaMax = 32;
         // In-place correction of stored gains costs about three dependent trips to memory per pick; a pass refreshes every
         // out-of-date block at once, so its cost per pick falls with the number of blocks.  Measured on CIFAR-10-shaped
-        // classes: with 8 blocks the correction wins (98 -> 47 ms), with 16 it does not (73 -> 74 ms).
-        if (ctx->cfg.incremental == 0) prm.incremental = sz.W <= 8 ? 1 : 0;
+        // classes: with 8 blocks the correction wins (99 -> 35 ms), with 16 it wins a little once the picks take their v* from
+        // the notes (72.6 -> 70.7 ms); with 32 blocks and small classes it loses.
+        if (ctx->cfg.incremental == 0) prm.incremental = sz.W <= 16 ? 1 : 0;
         prm.asyncMode = 1;
         prm.nPick = std::min<int>(sz.L, std::max(1, ctx->smCount / 4));
         prm.sweepWarps = (ctx->smCount - prm.nPick) * (kSweepThreads / 32);

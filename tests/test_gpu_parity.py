@@ -399,7 +399,7 @@ def test_incremental_update_float(rcd, orc, path):
 
 @pytest.mark.parametrize("path", [3, 4])
 def test_noted_candidates_ties_and_many_classes(rcd, orc, path):
-    """Picks that take v* from the note made at the block's last correction (eight blocks per class): duplicate samples
+    """Picks that take v* from the note made at the block's last correction (up to sixteen blocks per class keep notes): duplicate samples
     make equal gains (the lowest index must win, also when the noted sample of one block is taken by another block first),
     ragged classes, more classes than SMs in the one-CTA-per-class form; twice, with identical results."""
     from paper_2211_00839_b200.workloads import Workload, make_workload
