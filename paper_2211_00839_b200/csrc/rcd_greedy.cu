@@ -1845,11 +1845,15 @@ __device__ __forceinline__ void pick_chain(const GreedyParams<SV> &prm, int l, i
                     for (int k = 0; k < 3; ++k) {
                         const int i = (int)threadIdx.x + k * kSelectThreads;
                         if (i < ld4) {
+                            // (resident list: the four marks of this piece in one 16-byte read)
+                            int4 mk = make_int4(0, 0, 0, 0);
+                            if (res) mk = reinterpret_cast<const int4 *>(shPos)[i];
+                            const int mark[4] = {mk.x, mk.y, mk.z, mk.w};
 #pragma unroll
                             for (int q = 0; q < 4; ++q) {
                                 const int v = 4 * i + q;
                                 // (v* may or may not have left the list yet: named explicitly)
-                                if (v < c.M && v != vstar && (res ? shPos[v] : pos[v]) >= 0) {
+                                if (v < c.M && v != vstar && (res ? mark[q] : pos[v]) >= 0) {
                                     const unsigned long long kk = note_key(gj[k][q], v);
                                     if (kk > nk) nk = kk;
                                 }
